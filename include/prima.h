@@ -1,0 +1,177 @@
+/*
+ * prima.h -- C ABI of the B200 layer-window decoder for Q4_K models.
+ *
+ * The library executes the per-token forward pass of a contiguous WINDOW of transformer layers,
+ * the unit of work one device performs per round in pipelined-ring parallelism (paper Section 3.1,
+ * "Pipelined-ring parallelism (PRP) with prefetching"; Appendix A.12, "Mmap- and prefetch-based
+ * PRP": an 80-layer model on 4 devices with window 10 runs layers 1-10/11-20/21-30/31-40 in round
+ * one and 41-50/.../71-80 in round two).  What enters and leaves a window is the hidden state,
+ * e fp32 values per token, 4e bytes (Appendix A.3, network communication latency and device copy
+ * time).  Each layer keeps its own fp16 KV cache, which grows by 2(h_k e_k + h_v e_v) bytes per
+ * token and is read in full, 2(h_k e_k + h_v e_v) n_kv bytes, at every step (Appendix A.3, KV
+ * cache copy time and device loading time).  The input layer is a lookup table and the output
+ * layer produces the logits (Appendix A.3, computation latency).  Draft tokens of speculative
+ * decoding are verified by one batched pass of n_tok tokens (Appendix A.9 "Run Prima.cpp with
+ * Speculative Decoding"; Appendix A.12 "Speculative decoding").
+ *
+ * Weights are stored in the 4.5-bit Q4_K block format the paper names (Section 4; Appendix A.3,
+ * the set Q of quantisation types).  The paper does not print the bit layout; this library
+ * defines it as follows.  A super-block covers 256 consecutive weights of one row and is 144
+ * bytes, little endian:
+ *     bytes 0-1    d     IEEE binary16
+ *     bytes 2-3    dmin  IEEE binary16
+ *     bytes 4-15   s[0..11]: eight 6-bit scales sc_j and eight 6-bit mins m_j, j = 0..7
+ *                    j < 4 : sc_j = s[j] & 63                      m_j = s[j+4] & 63
+ *                    j >= 4: sc_j = (s[j+4] & 15) | (s[j-4] >> 6) << 4
+ *                            m_j  = (s[j+4] >> 4) | (s[j]   >> 6) << 4
+ *     bytes 16-143 qs[0..127]: byte qs[32p+i] (p = 0..3, i = 0..31) holds weight 64p+i in its low
+ *                  nibble and weight 64p+32+i in its high nibble
+ *     weight k = d * sc_j * q_k - dmin * m_j,  j = k / 32.
+ * A matrix W[rows x cols] is rows * (cols/256) super-blocks, row-major; cols % 256 == 0.
+ *
+ * Conventions.  Every function returns PRIMA_OK (0) or a negative error code; nothing throws,
+ * aborts or traps the GPU.  "dev" pointers are CUDA device pointers on the context's device,
+ * "host" pointers are ordinary host memory.  All work is queued on the context's stream; calls
+ * return without waiting unless stated.  The library owns the memory it allocates (weights in its
+ * own tiled layout, KV cache, scratch); the caller owns every buffer it passes in.
+ */
+#ifndef PRIMA_H
+#define PRIMA_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PRIMA_OK 0
+#define PRIMA_ERR_ARG (-1)        /* bad argument; nothing was modified or launched            */
+#define PRIMA_ERR_STATE (-2)      /* a needed tensor has not been loaded                        */
+#define PRIMA_ERR_CUDA (-3)       /* a CUDA call failed; see prima_last_error                   */
+#define PRIMA_ERR_NOMEM (-4)      /* device allocation failed                                   */
+#define PRIMA_ERR_DEVICE (-5)     /* a kernel reported a failed self-check (status word)        */
+
+#define PRIMA_Q4K_BLOCK_BYTES 144
+#define PRIMA_Q4K_BLOCK_WEIGHTS 256
+#define PRIMA_MAX_N_TOK 8
+
+/* tensor ids for prima_load_q4k_weights */
+enum {
+  PRIMA_ATTN_NORM = 0, /* fp32 [hidden]                 per layer */
+  PRIMA_WQ = 1,        /* Q4_K [n_q_heads*head_dim x hidden]       */
+  PRIMA_WK = 2,        /* Q4_K [n_kv_heads*head_dim x hidden]      */
+  PRIMA_WV = 3,        /* Q4_K [n_kv_heads*head_dim x hidden]      */
+  PRIMA_WO = 4,        /* Q4_K [hidden x n_q_heads*head_dim]       */
+  PRIMA_FFN_NORM = 5,  /* fp32 [hidden]                            */
+  PRIMA_W_GATE = 6,    /* Q4_K [ffn x hidden]                      */
+  PRIMA_W_UP = 7,      /* Q4_K [ffn x hidden]                      */
+  PRIMA_W_DOWN = 8,    /* Q4_K [hidden x ffn]                      */
+  PRIMA_OUT_NORM = 9,  /* fp32 [hidden]                 layer = -1 */
+  PRIMA_W_HEAD = 10,   /* Q4_K [vocab x hidden]         layer = -1 */
+  PRIMA_TOK_EMBD = 11  /* Q4_K [vocab x hidden]         layer = -1 */
+};
+
+typedef struct prima_ctx prima_ctx; /* opaque, owned by the library */
+
+/* Model shape; plain data, copied by prima_ctx_create. */
+typedef struct {
+  int32_t n_layers;
+  int32_t hidden;      /* e; multiple of 256                                                    */
+  int32_t n_q_heads;   /* H                                                                     */
+  int32_t n_kv_heads;  /* G; H % G == 0, H / G <= 8                                             */
+  int32_t head_dim;    /* must be 128                                                           */
+  int32_t ffn;         /* F; multiple of 256                                                    */
+  int32_t vocab;       /* V                                                                     */
+  int32_t kv_capacity; /* positions per layer in the fp16 KV cache                              */
+  int32_t max_n_tok;   /* largest n_tok of a step, 1..PRIMA_MAX_N_TOK                           */
+  float rms_eps;
+  float rope_theta;
+  int32_t rope_mode;   /* 0: rotate pairs (i, i + head_dim/2); 1: pairs (2i, 2i+1)              */
+  int32_t device;      /* CUDA ordinal                                                          */
+} prima_model_config;
+
+/* Create a context on cfg->device.  `cuda_stream` is a cudaStream_t (or NULL for the default
+ * stream) on which all work of this context is queued.  Allocates scratch buffers; the KV cache
+ * of a layer and its weights are allocated when first loaded.  Errors: PRIMA_ERR_ARG for an
+ * inconsistent shape, PRIMA_ERR_NOMEM / PRIMA_ERR_CUDA otherwise; *out is NULL on error. */
+int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx** out);
+
+/* Wait for the stream, then free every device buffer the context allocated. */
+int prima_ctx_destroy(prima_ctx* ctx);
+
+/* Load one tensor (the paper's model is a file of such tensors; Section 3.1).  Q4_K tensors:
+ * `data` holds rows*(cols/256)*144 bytes in the layout above; norm tensors: fp32[cols], rows = 1.
+ * `data` may be host or device memory; the library copies it into its own layout before
+ * returning (this call synchronises the stream), the caller may free `data` afterwards.
+ * layer = -1 for PRIMA_OUT_NORM / PRIMA_W_HEAD / PRIMA_TOK_EMBD.  A shape that disagrees with the
+ * config, cols % 256 != 0, a wrong nbytes, an unknown id or a layer out of range return
+ * PRIMA_ERR_ARG and leave the context unchanged. */
+int prima_load_q4k_weights(prima_ctx* ctx, int layer, int tensor_id, const void* data,
+                           int64_t rows, int64_t cols, int64_t nbytes);
+
+/* Run layers [layer_begin, layer_end) (one window of the ring schedule) on n_tok tokens at cache
+ * positions pos .. pos+n_tok-1.  hidden_in / hidden_out: dev, fp32, [n_tok x hidden] row-major,
+ * may alias.  Per layer: RMSNorm, Q/K/V projections, rotary embedding, append of K and V to the
+ * fp16 cache, grouped-query attention over positions 0..pos+t for token t (causal inside the
+ * step), output projection and residual, RMSNorm, SwiGLU feed-forward and residual.  Windows of
+ * one step must be issued in ascending layer order; any split of the layer range into windows
+ * gives bit-identical results.  Errors (no launch): a layer of the range is not fully loaded
+ * (PRIMA_ERR_STATE); bad range, pos < 0, pos + n_tok > kv_capacity, n_tok outside 1..max_n_tok,
+ * NULL pointers (PRIMA_ERR_ARG). */
+int prima_forward_window(prima_ctx* ctx, int layer_begin, int layer_end, const float* hidden_in,
+                         float* hidden_out, int pos, int n_tok);
+
+/* Output layer: logits[t][v] = W_head . RMSNorm(hidden[t]; out_norm).  hidden: dev fp32
+ * [n_tok x hidden]; logits: dev fp32 [n_tok x vocab]. */
+int prima_logits(prima_ctx* ctx, const float* hidden, int n_tok, float* logits);
+
+/* Input layer (lookup table): hidden_out[t] = dequantised row tokens[t] of PRIMA_TOK_EMBD.
+ * tokens: host int32[n_tok]; hidden_out: dev fp32 [n_tok x hidden]. */
+int prima_embed(prima_ctx* ctx, const int32_t* tokens, int n_tok, float* hidden_out);
+
+/* Greedy choice per token: index of the largest logit, lowest index on ties.  logits: dev fp32
+ * [n_tok x vocab]; tokens_out: host int32[n_tok].  Waits for the result. */
+int prima_argmax(prima_ctx* ctx, const float* logits, int n_tok, int32_t* tokens_out);
+
+/* Write / read fp16 cache entries of one layer.  k, v: host, [n_pos][n_kv_heads][head_dim]
+ * binary16 bit patterns.  Both calls synchronise.  Used to prefill a context and by tests. */
+int prima_kv_load(prima_ctx* ctx, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v);
+int prima_kv_read(prima_ctx* ctx, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v);
+
+/* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word and
+ * PRIMA_ERR_CUDA if the stream reports an error. */
+int prima_sync(prima_ctx* ctx);
+
+/* Text of the most recent error of this context (never NULL; "" if none).  With ctx == NULL,
+ * the most recent error of a context-free call on this thread. */
+const char* prima_last_error(prima_ctx* ctx);
+
+/* Number of kernels this context has launched since it was created (for accounting). */
+int64_t prima_launch_count(prima_ctx* ctx);
+
+/* ---- context-free exports of the two primitives (tests and micro-benchmarks) ---------------- */
+
+/* Dequantise n_superblocks blocks (dev, standard 144-byte layout) to fp32 (dev, 256 per block).
+ * The result is the exact value d*sc*q - dmin*m rounded once to binary32.  `stream` is a
+ * cudaStream_t or NULL. */
+int prima_dequant_q4k(const void* dev_blocks, int64_t n_superblocks, float* dev_out, void* stream);
+
+/* y[c][r] = sum_k W[r][k] x[c][k] for c < n_cols (1..8).  dev_w: standard layout; dev_x: fp32
+ * [n_cols x cols]; dev_y: fp32 [n_cols x rows].  Allocates and frees its own temporary buffers
+ * (tiled copy of W and scratch) and waits for completion; meant for testing single projections.
+ * For timing, use prima_gemv_plan_* below. */
+int prima_gemv_q4k(const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols,
+                   float* dev_y, void* stream);
+
+/* A resident, tiled copy of one matrix for repeated products (what a loaded layer tensor is
+ * inside a context).  create copies and re-tiles dev_w (synchronises); run queues one product on
+ * `stream` with no allocation and no synchronisation; destroy frees. */
+typedef struct prima_gemv_plan prima_gemv_plan;
+int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int max_n_cols, prima_gemv_plan** out);
+int prima_gemv_plan_run(prima_gemv_plan* plan, const float* dev_x, int n_cols, float* dev_y, void* stream);
+int prima_gemv_plan_destroy(prima_gemv_plan* plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRIMA_H */

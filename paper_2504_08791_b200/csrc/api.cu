@@ -1,0 +1,561 @@
+// C ABI of the layer-window decoder: context, weight loading, window execution, output layer.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/prima.h"
+#include "common.cuh"
+
+using namespace prima;
+
+namespace {
+
+thread_local std::string g_tls_error;
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    ok = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+struct Layer {
+  TiledMat qkv, o, gu, down;
+  float* g_attn = nullptr;
+  float* g_ffn = nullptr;
+  float gmax_attn = 1.f, gmax_ffn = 1.f;
+  uint32_t have = 0;   // bit per tensor id
+  __half* k = nullptr;
+  __half* v = nullptr;
+};
+
+constexpr uint32_t kLayerMask = (1u << 9) - 1;
+
+}  // namespace
+
+struct prima_ctx {
+  prima_model_config cfg{};
+  cudaStream_t stream = nullptr;
+  int sm_count = 0;
+  std::vector<Layer> layers;
+  float* g_out = nullptr;
+  float gmax_out = 1.f;
+  TiledMat head;
+  uint8_t* embd = nullptr;
+  bool have_out_norm = false, have_head = false, have_embd = false;
+
+  float* part = nullptr;
+  size_t part_floats = 0;
+  float* h = nullptr;
+  float* qbuf = nullptr;
+  float* obuf = nullptr;
+  float* act = nullptr;
+  VecStats st_h, st_o, st_act;
+  float2* rope_tab = nullptr;
+  AttnScratch attn{};
+  uint8_t* staging = nullptr;
+  size_t staging_bytes = 0;
+  int32_t* d_tokens = nullptr;
+  float* am_val = nullptr;
+  int32_t* am_idx = nullptr;
+  int32_t* am_out = nullptr;
+  int* status = nullptr;
+
+  std::vector<void*> allocs;
+  std::string err;
+  int64_t launches = 0;
+};
+
+struct prima_gemv_plan {
+  int device = 0;
+  int sm_count = 0;
+  int max_n_cols = 1;
+  TiledMat w;
+  float* part = nullptr;
+  VecStats stats;
+};
+
+namespace {
+
+int fail(prima_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  else g_tls_error = msg;
+  return code;
+}
+
+int cuda_fail(prima_ctx* c, cudaError_t e, const char* what) {
+  std::string msg = std::string(what) + ": " + cudaGetErrorString(e);
+  return fail(c, e == cudaErrorMemoryAllocation ? PRIMA_ERR_NOMEM : PRIMA_ERR_CUDA, msg);
+}
+
+template <typename T>
+int dev_alloc(prima_ctx* c, T** p, size_t count, bool zero = false) {
+  void* raw = nullptr;
+  cudaError_t e = cudaMalloc(&raw, std::max<size_t>(count * sizeof(T), 16));
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMalloc");
+  if (zero) {
+    e = cudaMemsetAsync(raw, 0, std::max<size_t>(count * sizeof(T), 16), c->stream);
+    if (e != cudaSuccess) {
+      cudaFree(raw);
+      return cuda_fail(c, e, "cudaMemsetAsync");
+    }
+  }
+  c->allocs.push_back(raw);
+  *p = static_cast<T*>(raw);
+  return PRIMA_OK;
+}
+
+TiledMat shape_tiled(int64_t rows, int64_t cols) {
+  TiledMat t;
+  t.rows = rows;
+  t.cols = cols;
+  t.n_rt = (rows + kRowsPerTile - 1) / kRowsPerTile;
+  t.n_sb = cols / 256;
+  return t;
+}
+
+int ensure_tiled(prima_ctx* c, TiledMat* t, int64_t rows, int64_t cols) {
+  if (t->data) return PRIMA_OK;
+  TiledMat s = shape_tiled(rows, cols);
+  int rc = dev_alloc(c, &s.data, s.bytes(), true);
+  if (rc != PRIMA_OK) return rc;
+  *t = s;
+  return PRIMA_OK;
+}
+
+int ensure_kv(prima_ctx* c, int layer) {
+  Layer& L = c->layers[layer];
+  if (L.k) return PRIMA_OK;
+  const size_t n = static_cast<size_t>(c->cfg.n_kv_heads) * c->cfg.kv_capacity * kHeadDim;
+  int rc = dev_alloc(c, &L.k, n, true);
+  if (rc != PRIMA_OK) return rc;
+  return dev_alloc(c, &L.v, n, true);
+}
+
+// Copy a standard-layout matrix (host or device) through the staging buffer and re-tile it.
+int load_tiled(prima_ctx* c, TiledMat& dst, const uint8_t* data, int64_t rows, int64_t n_sb, int64_t row0, int64_t stride) {
+  const int64_t row_bytes = n_sb * kBlockBytes;
+  int64_t rows_per_chunk = std::max<int64_t>(1, static_cast<int64_t>(c->staging_bytes) / row_bytes);
+  for (int64_t r = 0; r < rows; r += rows_per_chunk) {
+    const int64_t n = std::min(rows_per_chunk, rows - r);
+    cudaError_t e = cudaMemcpyAsync(c->staging, data + r * row_bytes, static_cast<size_t>(n * row_bytes), cudaMemcpyDefault, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(weights)");
+    int k = launch_retile(c->staging, n, n_sb, dst, row0 + r * stride, stride, c->stream);
+    if (k < 0) return cuda_fail(c, static_cast<cudaError_t>(-k), "retile kernel");
+  }
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize(load)");
+  return PRIMA_OK;
+}
+
+int load_norm(prima_ctx* c, float** dst, float* gmax, const void* data, int64_t cols) {
+  std::vector<float> host(static_cast<size_t>(cols));
+  cudaError_t e = cudaMemcpy(host.data(), data, static_cast<size_t>(cols) * 4, cudaMemcpyDefault);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpy(norm)");
+  float m = 0.f;
+  for (float v : host) m = std::max(m, std::fabs(v));
+  if (!*dst) {
+    int rc = dev_alloc(c, dst, static_cast<size_t>(cols));
+    if (rc != PRIMA_OK) return rc;
+  }
+  e = cudaMemcpy(*dst, host.data(), static_cast<size_t>(cols) * 4, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpy(norm upload)");
+  *gmax = m;
+  return PRIMA_OK;
+}
+
+#define LAUNCH(c, expr, what)                                                       \
+  do {                                                                              \
+    int k_ = (expr);                                                                \
+    if (k_ < 0) return cuda_fail((c), static_cast<cudaError_t>(-k_), what);         \
+    (c)->launches += k_;                                                            \
+  } while (0)
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !out) return fail(nullptr, PRIMA_ERR_ARG, "prima_ctx_create: null argument");
+  const prima_model_config& g = *cfg;
+  if (g.n_layers < 1 || g.hidden < 256 || g.hidden % 256 || g.ffn < 256 || g.ffn % 256 || g.head_dim != kHeadDim ||
+      g.n_q_heads < 1 || g.n_kv_heads < 1 || g.n_q_heads % g.n_kv_heads || g.n_q_heads / g.n_kv_heads > 8 ||
+      g.n_q_heads > kMaxStatBlocks || g.vocab < 1 || g.kv_capacity < 1 || g.max_n_tok < 1 || g.max_n_tok > PRIMA_MAX_N_TOK ||
+      !(g.rms_eps >= 0.f) || !(g.rope_theta > 0.f) || (g.rope_mode != 0 && g.rope_mode != 1) || g.device < 0)
+    return fail(nullptr, PRIMA_ERR_ARG, "prima_ctx_create: inconsistent model shape");
+  int n_dev = 0;
+  cudaError_t e = cudaGetDeviceCount(&n_dev);
+  if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetDeviceCount");
+  if (g.device >= n_dev) return fail(nullptr, PRIMA_ERR_ARG, "prima_ctx_create: no such device");
+  DeviceGuard guard(g.device);
+  if (!guard.ok) return fail(nullptr, PRIMA_ERR_CUDA, "cudaSetDevice failed");
+
+  prima_ctx* c = new (std::nothrow) prima_ctx();
+  if (!c) return fail(nullptr, PRIMA_ERR_NOMEM, "out of host memory");
+  c->cfg = g;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->layers.resize(g.n_layers);
+  cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, g.device);
+
+  const int64_t n = g.max_n_tok;
+  const int64_t e_ = g.hidden, H = g.n_q_heads, G = g.n_kv_heads, F = g.ffn;
+  auto pad8 = [](int64_t r) { return (r + 7) / 8 * 8; };
+  int64_t part = 0;
+  part = std::max(part, (e_ / 256) * n * pad8((H + 2 * G) * kHeadDim));
+  part = std::max(part, (H * kHeadDim / 256) * n * pad8(e_));
+  part = std::max(part, (e_ / 256) * n * pad8(2 * F));
+  part = std::max(part, (F / 256) * n * pad8(e_));
+  part = std::max(part, (e_ / 256) * n * pad8(g.vocab));
+  c->part_floats = static_cast<size_t>(part);
+  c->attn.max_chunks = (g.kv_capacity + attention_chunk_len() - 1) / attention_chunk_len();
+  c->staging_bytes = 256u << 20;
+
+  int rc = PRIMA_OK;
+  auto A = [&](int r) { if (rc == PRIMA_OK) rc = r; };
+  A(dev_alloc(c, &c->part, c->part_floats));
+  A(dev_alloc(c, &c->h, static_cast<size_t>(n * e_)));
+  A(dev_alloc(c, &c->qbuf, static_cast<size_t>(n * H * kHeadDim)));
+  A(dev_alloc(c, &c->obuf, static_cast<size_t>(n * H * kHeadDim)));
+  A(dev_alloc(c, &c->act, static_cast<size_t>(n * F)));
+  A(dev_alloc(c, &c->st_h.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
+  A(dev_alloc(c, &c->st_o.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
+  A(dev_alloc(c, &c->st_act.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
+  A(dev_alloc(c, &c->rope_tab, static_cast<size_t>(kMaxTok) * (kHeadDim / 2)));
+  A(dev_alloc(c, &c->attn.o_part, static_cast<size_t>(n * H) * c->attn.max_chunks * kHeadDim));
+  A(dev_alloc(c, &c->attn.ml_part, static_cast<size_t>(n * H) * c->attn.max_chunks));
+  A(dev_alloc(c, &c->staging, c->staging_bytes));
+  A(dev_alloc(c, &c->d_tokens, static_cast<size_t>(kMaxTok)));
+  A(dev_alloc(c, &c->am_val, static_cast<size_t>(kMaxTok) * kArgmaxBlocks));
+  A(dev_alloc(c, &c->am_idx, static_cast<size_t>(kMaxTok) * kArgmaxBlocks));
+  A(dev_alloc(c, &c->am_out, static_cast<size_t>(kMaxTok)));
+  A(dev_alloc(c, &c->status, 1, true));
+  if (rc != PRIMA_OK) {
+    g_tls_error = c->err;
+    for (void* p : c->allocs) cudaFree(p);
+    delete c;
+    return rc;
+  }
+  *out = c;
+  return PRIMA_OK;
+}
+
+int prima_ctx_destroy(prima_ctx* c) {
+  if (!c) return PRIMA_OK;
+  DeviceGuard guard(c->cfg.device);
+  cudaStreamSynchronize(c->stream);
+  for (void* p : c->allocs) cudaFree(p);
+  delete c;
+  return PRIMA_OK;
+}
+
+int prima_load_q4k_weights(prima_ctx* c, int layer, int tensor_id, const void* data, int64_t rows, int64_t cols,
+                           int64_t nbytes) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_load_q4k_weights: null context");
+  if (!data) return fail(c, PRIMA_ERR_ARG, "prima_load_q4k_weights: null data");
+  if (tensor_id < PRIMA_ATTN_NORM || tensor_id > PRIMA_TOK_EMBD) return fail(c, PRIMA_ERR_ARG, "unknown tensor id");
+  const prima_model_config& g = c->cfg;
+  const bool global = tensor_id >= PRIMA_OUT_NORM;
+  if (global ? layer != -1 : (layer < 0 || layer >= g.n_layers)) return fail(c, PRIMA_ERR_ARG, "layer out of range");
+  const int64_t e_ = g.hidden, H = g.n_q_heads, G = g.n_kv_heads, F = g.ffn, V = g.vocab;
+  int64_t want_rows = 1, want_cols = e_;
+  bool is_norm = false;
+  switch (tensor_id) {
+    case PRIMA_ATTN_NORM: case PRIMA_FFN_NORM: case PRIMA_OUT_NORM: is_norm = true; break;
+    case PRIMA_WQ: want_rows = H * kHeadDim; break;
+    case PRIMA_WK: case PRIMA_WV: want_rows = G * kHeadDim; break;
+    case PRIMA_WO: want_rows = e_; want_cols = H * kHeadDim; break;
+    case PRIMA_W_GATE: case PRIMA_W_UP: want_rows = F; break;
+    case PRIMA_W_DOWN: want_rows = e_; want_cols = F; break;
+    case PRIMA_W_HEAD: case PRIMA_TOK_EMBD: want_rows = V; break;
+  }
+  if (cols % 256 != 0 && !is_norm) return fail(c, PRIMA_ERR_ARG, "cols must be a multiple of 256");
+  if (rows != want_rows || cols != want_cols) return fail(c, PRIMA_ERR_ARG, "tensor shape disagrees with the model config");
+  const int64_t want_bytes = is_norm ? cols * 4 : rows * (cols / 256) * kBlockBytes;
+  if (nbytes != want_bytes) return fail(c, PRIMA_ERR_ARG, "nbytes disagrees with rows and cols");
+  DeviceGuard guard(g.device);
+
+  const uint8_t* bytes = static_cast<const uint8_t*>(data);
+  const int64_t n_sb = cols / 256;
+  int rc = PRIMA_OK;
+  if (global) {
+    if (tensor_id == PRIMA_OUT_NORM) {
+      rc = load_norm(c, &c->g_out, &c->gmax_out, data, cols);
+      if (rc == PRIMA_OK) c->have_out_norm = true;
+    } else if (tensor_id == PRIMA_W_HEAD) {
+      rc = ensure_tiled(c, &c->head, V, e_);
+      if (rc == PRIMA_OK) rc = load_tiled(c, c->head, bytes, rows, n_sb, 0, 1);
+      if (rc == PRIMA_OK) c->have_head = true;
+    } else {
+      if (!c->embd) rc = dev_alloc(c, &c->embd, static_cast<size_t>(nbytes));
+      if (rc == PRIMA_OK) {
+        cudaError_t e = cudaMemcpy(c->embd, data, static_cast<size_t>(nbytes), cudaMemcpyDefault);
+        if (e != cudaSuccess) rc = cuda_fail(c, e, "cudaMemcpy(embedding)");
+      }
+      if (rc == PRIMA_OK) c->have_embd = true;
+    }
+    return rc;
+  }
+  Layer& L = c->layers[layer];
+  rc = ensure_kv(c, layer);
+  if (rc != PRIMA_OK) return rc;
+  switch (tensor_id) {
+    case PRIMA_ATTN_NORM: rc = load_norm(c, &L.g_attn, &L.gmax_attn, data, cols); break;
+    case PRIMA_FFN_NORM: rc = load_norm(c, &L.g_ffn, &L.gmax_ffn, data, cols); break;
+    case PRIMA_WQ: case PRIMA_WK: case PRIMA_WV: {
+      rc = ensure_tiled(c, &L.qkv, (H + 2 * G) * kHeadDim, e_);
+      const int64_t row0 = tensor_id == PRIMA_WQ ? 0 : tensor_id == PRIMA_WK ? H * kHeadDim : (H + G) * kHeadDim;
+      if (rc == PRIMA_OK) rc = load_tiled(c, L.qkv, bytes, rows, n_sb, row0, 1);
+      break;
+    }
+    case PRIMA_WO:
+      rc = ensure_tiled(c, &L.o, e_, H * kHeadDim);
+      if (rc == PRIMA_OK) rc = load_tiled(c, L.o, bytes, rows, n_sb, 0, 1);
+      break;
+    case PRIMA_W_GATE: case PRIMA_W_UP:
+      rc = ensure_tiled(c, &L.gu, 2 * F, e_);
+      if (rc == PRIMA_OK) rc = load_tiled(c, L.gu, bytes, rows, n_sb, tensor_id == PRIMA_W_GATE ? 0 : 1, 2);
+      break;
+    case PRIMA_W_DOWN:
+      rc = ensure_tiled(c, &L.down, e_, F);
+      if (rc == PRIMA_OK) rc = load_tiled(c, L.down, bytes, rows, n_sb, 0, 1);
+      break;
+  }
+  if (rc == PRIMA_OK) L.have |= 1u << tensor_id;
+  return rc;
+}
+
+int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos,
+                         int n_tok) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_forward_window: null context");
+  const prima_model_config& g = c->cfg;
+  if (!hidden_in || !hidden_out) return fail(c, PRIMA_ERR_ARG, "prima_forward_window: null hidden pointer");
+  if (layer_begin < 0 || layer_end > g.n_layers || layer_begin > layer_end) return fail(c, PRIMA_ERR_ARG, "bad layer range");
+  if (n_tok < 1 || n_tok > g.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
+  if (pos < 0 || static_cast<int64_t>(pos) + n_tok > g.kv_capacity) return fail(c, PRIMA_ERR_ARG, "pos + n_tok exceeds kv_capacity");
+  for (int l = layer_begin; l < layer_end; ++l)
+    if ((c->layers[l].have & kLayerMask) != kLayerMask) return fail(c, PRIMA_ERR_STATE, "a layer of the window is not fully loaded");
+  DeviceGuard guard(g.device);
+  cudaStream_t st = c->stream;
+  const int64_t e_ = g.hidden;
+  const int H = g.n_q_heads, G = g.n_kv_heads;
+
+  LAUNCH(c, launch_copy_stats(hidden_in, c->h, e_, n_tok, &c->st_h, st), "copy_stats");
+  if (layer_begin < layer_end) LAUNCH(c, launch_rope_table(c->rope_tab, pos, n_tok, g.rope_theta, st), "rope_table");
+  for (int l = layer_begin; l < layer_end; ++l) {
+    Layer& L = c->layers[l];
+    GemvIn in{c->h, L.g_attn, L.gmax_attn, g.rms_eps, c->st_h};
+    LAUNCH(c, launch_gemv_partials(L.qkv, in, n_tok, c->part, c->sm_count, st), "gemv(qkv)");
+    LAUNCH(c, launch_finish_qkv(c->part, L.qkv.n_sb, L.qkv.mpad(), H, G, n_tok, c->rope_tab, g.rope_mode, c->qbuf, L.k, L.v,
+                                g.kv_capacity, pos, st), "finish_qkv");
+    LAUNCH(c, launch_attention(c->qbuf, L.k, L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, &c->st_o, st), "attention");
+    GemvIn in_o{c->obuf, nullptr, 1.f, 0.f, c->st_o};
+    LAUNCH(c, launch_gemv_partials(L.o, in_o, n_tok, c->part, c->sm_count, st), "gemv(o)");
+    LAUNCH(c, launch_finish_residual(c->part, L.o.n_sb, L.o.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(o)");
+    GemvIn in_f{c->h, L.g_ffn, L.gmax_ffn, g.rms_eps, c->st_h};
+    LAUNCH(c, launch_gemv_partials(L.gu, in_f, n_tok, c->part, c->sm_count, st), "gemv(gate/up)");
+    LAUNCH(c, launch_finish_swiglu(c->part, L.gu.n_sb, L.gu.mpad(), g.ffn, n_tok, c->act, &c->st_act, st), "finish_swiglu");
+    GemvIn in_d{c->act, nullptr, 1.f, 0.f, c->st_act};
+    LAUNCH(c, launch_gemv_partials(L.down, in_d, n_tok, c->part, c->sm_count, st), "gemv(down)");
+    LAUNCH(c, launch_finish_residual(c->part, L.down.n_sb, L.down.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(down)");
+  }
+  cudaError_t e = cudaMemcpyAsync(hidden_out, c->h, static_cast<size_t>(n_tok) * e_ * 4, cudaMemcpyDeviceToDevice, st);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(hidden_out)");
+  return PRIMA_OK;
+}
+
+int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_logits: null context");
+  if (!hidden || !logits) return fail(c, PRIMA_ERR_ARG, "prima_logits: null pointer");
+  if (n_tok < 1 || n_tok > c->cfg.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
+  if (!c->have_out_norm || !c->have_head) return fail(c, PRIMA_ERR_STATE, "output norm or head not loaded");
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = c->stream;
+  LAUNCH(c, launch_copy_stats(hidden, nullptr, c->cfg.hidden, n_tok, &c->st_h, st), "copy_stats");
+  GemvIn in{hidden, c->g_out, c->gmax_out, c->cfg.rms_eps, c->st_h};
+  LAUNCH(c, launch_gemv_partials(c->head, in, n_tok, c->part, c->sm_count, st), "gemv(head)");
+  LAUNCH(c, launch_finish_plain(c->part, c->head.n_sb, c->head.mpad(), c->cfg.vocab, n_tok, logits, st), "finish_plain");
+  return PRIMA_OK;
+}
+
+int prima_embed(prima_ctx* c, const int32_t* tokens, int n_tok, float* hidden_out) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_embed: null context");
+  if (!tokens || !hidden_out) return fail(c, PRIMA_ERR_ARG, "prima_embed: null pointer");
+  if (n_tok < 1 || n_tok > c->cfg.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
+  if (!c->have_embd) return fail(c, PRIMA_ERR_STATE, "embedding table not loaded");
+  for (int t = 0; t < n_tok; ++t)
+    if (tokens[t] < 0 || tokens[t] >= c->cfg.vocab) return fail(c, PRIMA_ERR_ARG, "token id out of range");
+  DeviceGuard guard(c->cfg.device);
+  cudaError_t e = cudaMemcpyAsync(c->d_tokens, tokens, static_cast<size_t>(n_tok) * 4, cudaMemcpyHostToDevice, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(tokens)");
+  LAUNCH(c, launch_embed(c->embd, c->cfg.hidden / 256, c->d_tokens, n_tok, hidden_out, c->stream), "embed");
+  return PRIMA_OK;
+}
+
+int prima_argmax(prima_ctx* c, const float* logits, int n_tok, int32_t* tokens_out) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_argmax: null context");
+  if (!logits || !tokens_out) return fail(c, PRIMA_ERR_ARG, "prima_argmax: null pointer");
+  if (n_tok < 1 || n_tok > c->cfg.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
+  DeviceGuard guard(c->cfg.device);
+  LAUNCH(c, launch_argmax(logits, c->cfg.vocab, n_tok, c->am_val, c->am_idx, c->am_out, c->stream), "argmax");
+  cudaError_t e = cudaMemcpyAsync(tokens_out, c->am_out, static_cast<size_t>(n_tok) * 4, cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "argmax readback");
+  return PRIMA_OK;
+}
+
+static int kv_args_ok(prima_ctx* c, int layer, int pos_begin, int n_pos, const void* k, const void* v) {
+  if (!k || !v) return fail(c, PRIMA_ERR_ARG, "null k or v");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PRIMA_ERR_ARG, "layer out of range");
+  if (pos_begin < 0 || n_pos < 0 || static_cast<int64_t>(pos_begin) + n_pos > c->cfg.kv_capacity)
+    return fail(c, PRIMA_ERR_ARG, "position range outside the cache");
+  return PRIMA_OK;
+}
+
+// Host layout [n_pos][G][128]; device layout [G][capacity][128]: one strided 2-D copy per KV head.
+int prima_kv_load(prima_ctx* c, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_kv_load: null context");
+  int rc = kv_args_ok(c, layer, pos_begin, n_pos, k, v);
+  if (rc != PRIMA_OK) return rc;
+  DeviceGuard guard(c->cfg.device);
+  rc = ensure_kv(c, layer);
+  if (rc != PRIMA_OK) return rc;
+  if (n_pos == 0) return PRIMA_OK;
+  Layer& L = c->layers[layer];
+  const int G = c->cfg.n_kv_heads;
+  const size_t row = kHeadDim * 2;
+  for (int gk = 0; gk < G; ++gk) {
+    cudaError_t e = cudaMemcpy2DAsync(L.k + (static_cast<size_t>(gk) * c->cfg.kv_capacity + pos_begin) * kHeadDim, row,
+                                      k + static_cast<size_t>(gk) * kHeadDim, row * G, row, n_pos, cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess)
+      e = cudaMemcpy2DAsync(L.v + (static_cast<size_t>(gk) * c->cfg.kv_capacity + pos_begin) * kHeadDim, row,
+                            v + static_cast<size_t>(gk) * kHeadDim, row * G, row, n_pos, cudaMemcpyHostToDevice, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpy2DAsync(kv_load)");
+  }
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "kv_load sync");
+  return PRIMA_OK;
+}
+
+int prima_kv_read(prima_ctx* c, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_kv_read: null context");
+  int rc = kv_args_ok(c, layer, pos_begin, n_pos, k, v);
+  if (rc != PRIMA_OK) return rc;
+  DeviceGuard guard(c->cfg.device);
+  rc = ensure_kv(c, layer);
+  if (rc != PRIMA_OK) return rc;
+  if (n_pos == 0) return PRIMA_OK;
+  Layer& L = c->layers[layer];
+  const int G = c->cfg.n_kv_heads;
+  const size_t row = kHeadDim * 2;
+  for (int gk = 0; gk < G; ++gk) {
+    cudaError_t e = cudaMemcpy2DAsync(k + static_cast<size_t>(gk) * kHeadDim, row * G,
+                                      L.k + (static_cast<size_t>(gk) * c->cfg.kv_capacity + pos_begin) * kHeadDim, row, row, n_pos,
+                                      cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess)
+      e = cudaMemcpy2DAsync(v + static_cast<size_t>(gk) * kHeadDim, row * G,
+                            L.v + (static_cast<size_t>(gk) * c->cfg.kv_capacity + pos_begin) * kHeadDim, row, row, n_pos,
+                            cudaMemcpyDeviceToHost, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpy2DAsync(kv_read)");
+  }
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "kv_read sync");
+  return PRIMA_OK;
+}
+
+int prima_sync(prima_ctx* c) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_sync: null context");
+  DeviceGuard guard(c->cfg.device);
+  int status = 0;
+  cudaError_t e = cudaMemcpyAsync(&status, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync");
+  if (status != 0) return fail(c, PRIMA_ERR_DEVICE, "a kernel raised the device status word: " + std::to_string(status));
+  return PRIMA_OK;
+}
+
+const char* prima_last_error(prima_ctx* c) { return c ? c->err.c_str() : g_tls_error.c_str(); }
+
+int64_t prima_launch_count(prima_ctx* c) { return c ? c->launches : 0; }
+
+// ---- context-free primitives ------------------------------------------------------------------
+int prima_dequant_q4k(const void* dev_blocks, int64_t n_superblocks, float* dev_out, void* stream) {
+  if (!dev_blocks || !dev_out || n_superblocks < 0) return fail(nullptr, PRIMA_ERR_ARG, "prima_dequant_q4k: bad argument");
+  int k = launch_dequant_std(static_cast<const uint8_t*>(dev_blocks), n_superblocks, dev_out, static_cast<cudaStream_t>(stream));
+  if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "dequant kernel");
+  return PRIMA_OK;
+}
+
+int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int max_n_cols, prima_gemv_plan** out) {
+  if (out) *out = nullptr;
+  if (!dev_w || !out || rows < 1 || cols < 256 || cols % 256 || max_n_cols < 1 || max_n_cols > PRIMA_MAX_N_TOK)
+    return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_plan_create: bad argument");
+  prima_gemv_plan* p = new (std::nothrow) prima_gemv_plan();
+  if (!p) return fail(nullptr, PRIMA_ERR_NOMEM, "out of host memory");
+  cudaGetDevice(&p->device);
+  cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+  p->max_n_cols = max_n_cols;
+  p->w = shape_tiled(rows, cols);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&p->w.data), p->w.bytes());
+  if (e == cudaSuccess) e = cudaMemset(p->w.data, 0, p->w.bytes());
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->part), static_cast<size_t>(p->w.n_sb) * max_n_cols * p->w.mpad() * 4);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->stats.data), sizeof(float2) * kMaxTok * kMaxStatBlocks);
+  if (e == cudaSuccess) {
+    int k = launch_retile(static_cast<const uint8_t*>(dev_w), rows, p->w.n_sb, p->w, 0, 1, nullptr);
+    if (k < 0) e = static_cast<cudaError_t>(-k);
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    prima_gemv_plan_destroy(p);
+    return cuda_fail(nullptr, e, "prima_gemv_plan_create");
+  }
+  *out = p;
+  return PRIMA_OK;
+}
+
+int prima_gemv_plan_run(prima_gemv_plan* p, const float* dev_x, int n_cols, float* dev_y, void* stream) {
+  if (!p || !dev_x || !dev_y || n_cols < 1 || n_cols > p->max_n_cols) return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_plan_run: bad argument");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int k = launch_copy_stats(dev_x, nullptr, p->w.cols, n_cols, &p->stats, st);
+  if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "copy_stats");
+  GemvIn in{dev_x, nullptr, 1.f, 0.f, p->stats};
+  k = launch_gemv_partials(p->w, in, n_cols, p->part, p->sm_count, st);
+  if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "gemv kernel");
+  k = launch_finish_plain(p->part, p->w.n_sb, p->w.mpad(), p->w.rows, n_cols, dev_y, st);
+  if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "finish kernel");
+  return PRIMA_OK;
+}
+
+int prima_gemv_plan_destroy(prima_gemv_plan* p) {
+  if (!p) return PRIMA_OK;
+  cudaFree(p->w.data);
+  cudaFree(p->part);
+  cudaFree(p->stats.data);
+  delete p;
+  return PRIMA_OK;
+}
+
+int prima_gemv_q4k(const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols, float* dev_y, void* stream) {
+  if (!dev_x || !dev_y || n_cols < 1 || n_cols > PRIMA_MAX_N_TOK) return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_q4k: bad argument");
+  prima_gemv_plan* p = nullptr;
+  int rc = prima_gemv_plan_create(dev_w, rows, cols, n_cols, &p);
+  if (rc != PRIMA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = prima_gemv_plan_run(p, dev_x, n_cols, dev_y, st);
+  cudaError_t e = cudaStreamSynchronize(st);
+  prima_gemv_plan_destroy(p);
+  if (rc != PRIMA_OK) return rc;
+  if (e != cudaSuccess) return cuda_fail(nullptr, e, "prima_gemv_q4k");
+  return PRIMA_OK;
+}
+
+}  // extern "C"

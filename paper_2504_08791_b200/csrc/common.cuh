@@ -1,0 +1,133 @@
+// Shared declarations of the CUDA sources: tiled weight layout, launch interfaces, small helpers.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace prima {
+
+// ---------------------------------------------------------------------------------------------
+// Tiled weight layout (what a Q4_K matrix looks like in HBM after loading)
+//
+// A "unit" is the 8 super-blocks found at the crossing of one row tile (8 consecutive rows) and one
+// super-block column s (256 consecutive weights): 8 * 144 = 1152 bytes, the same bytes as the
+// source blocks, rearranged so that one warp reads it with three 16-byte loads per lane:
+//
+//   bytes    0..127   headers: row g (0..7) at g*16: word0 = d | dmin << 16 (binary16 bits),
+//                     words 1..3 = the sixteen 6-bit fields regrouped per lane quad position t:
+//                     f_t = sc_t | sc_{t+4} << 6 | m_t << 12 | m_{t+4} << 18  (24 bits, t = 0..3)
+//                     word1 = f_0 | (f_3 & 0xff) << 24, word2 = f_1 | (f_3 >> 8 & 0xff) << 24,
+//                     word3 = f_2 | (f_3 >> 16) << 24
+//   bytes  128..639   nibbles of sub-blocks 0..3: lane (g, t) = g*4 + t owns 16 bytes at lane*16,
+//                     the 32 weights of row g, sub-block t
+//   bytes  640..1151  the same for sub-blocks 4..7 (lane (g, t) owns sub-block 4 + t)
+//
+// Inside a 16-byte sub-block chunk, word w (0..3) holds weights 8w..8w+7 with nibble positions
+//   bits 0-3: 8w+0   bits 16-19: 8w+1   bits 4-7: 8w+2   bits 20-23: 8w+3
+//   bits 8-11: 8w+4  bits 24-27: 8w+5   bits 12-15: 8w+6 bits 28-31: 8w+7
+// so that (word & 0x000f000f) is a pair of consecutive weights sitting in the low mantissa bits of
+// two binary16 lanes (value q * 2^-24, a subnormal, exact), (word & 0x00f000f0) the next pair
+// scaled by 16, and the same two masks applied to word >> 8 give the remaining two pairs.
+//
+// Units are stored column-major over the (row tile, super-block column) grid:
+//   offset(s, rt) = (s * n_rt + rt) * 1152
+// so that a warp that walks down the rows at a fixed column s -- which lets it keep its 256
+// activations in registers -- streams one contiguous byte range.
+// Rows are padded with zero blocks up to a multiple of 8.
+// ---------------------------------------------------------------------------------------------
+constexpr int kUnitBytes = 1152;
+constexpr int kUnitHdrBytes = 128;
+constexpr int kRowsPerTile = 8;
+constexpr int kBlockBytes = 144;
+constexpr int kMaxTok = 8;
+constexpr int kMaxStatBlocks = 256;
+constexpr int kHeadDim = 128;
+
+struct TiledMat {
+  uint8_t* data = nullptr;   // device, n_sb * n_rt * 1152 bytes
+  int64_t rows = 0;          // logical rows (of the fused matrix)
+  int64_t cols = 0;
+  int64_t n_rt = 0;          // row tiles = ceil(rows / 8)
+  int64_t n_sb = 0;          // cols / 256
+  size_t bytes() const { return static_cast<size_t>(n_sb) * n_rt * kUnitBytes; }
+  int64_t mpad() const { return n_rt * kRowsPerTile; }
+};
+
+// Per-token activation statistics written by whichever kernel produced a vector and read by the
+// GEMV that consumes it: stats[tok][block] = (sum of squares, max |x|) over the block's slice.
+struct VecStats {
+  float2* data = nullptr;    // device, [kMaxTok][kMaxStatBlocks]
+  int n_blocks = 0;
+};
+
+// ---- launch interfaces (definitions in the .cu files) ----------------------------------------
+// Each returns the number of kernels it launched (for accounting) or a negative cudaError_t.
+
+// Standard-layout dequantisation (bit-exact definition of the format).
+int launch_dequant_std(const uint8_t* blocks, int64_t n_sb, float* out, cudaStream_t st);
+
+// Re-tile `rows_src` rows of a standard-layout matrix into dst; source row r lands at fused row
+// dst_row0 + r * dst_row_stride.
+int launch_retile(const uint8_t* src, int64_t rows_src, int64_t n_sb, TiledMat dst, int64_t dst_row0,
+                  int64_t dst_row_stride, cudaStream_t st);
+
+// Partial products of every (row, super-block column):
+//   part[(s * n_tok + t) * mpad + r] = sum over the 256 weights of column s of W[r][k] * xhat[t][k]
+// where xhat = x * gain * rsqrt(mean(x^2) + eps) if gain != nullptr, else x.  x: [n_tok][cols].
+struct GemvIn {
+  const float* x;        // [n_tok][cols] fp32
+  const float* gain;     // [cols] or nullptr (no normalisation)
+  float gain_max;        // max |gain| (1 if gain == nullptr)
+  float eps;
+  VecStats stats;        // statistics of x
+};
+int launch_gemv_partials(const TiledMat& w, const GemvIn& in, int n_tok, float* part, int sm_count,
+                         cudaStream_t st);
+
+// Finishers: sum the partials of a row over the super-block columns in ascending order, then
+//   plain:    y[t][r] = sum
+//   residual: h[t][r] = h[t][r] + sum, and statistics of the new h
+//   swiglu:   act[t][r] = silu(sum of fused row 2r) * (sum of fused row 2r+1), statistics of act
+//   qkv:      rows are [q heads | k heads | v heads] x 128; rotate q and k with the cos/sin table,
+//             write q (fp32, [n_tok][H*128]) and append k, v as binary16 to the cache at pos + t
+int launch_finish_plain(const float* part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok, float* y,
+                        cudaStream_t st);
+int launch_finish_residual(const float* part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok, float* h,
+                           VecStats* stats, cudaStream_t st);
+int launch_finish_swiglu(const float* part, int64_t n_sb, int64_t mpad, int64_t ffn, int n_tok, float* act,
+                         VecStats* stats, cudaStream_t st);
+int launch_finish_qkv(const float* part, int64_t n_sb, int64_t mpad, int n_q_heads, int n_kv_heads, int n_tok,
+                      const float2* rope_tab, int rope_mode, float* q_out, __half* k_cache, __half* v_cache,
+                      int kv_capacity, int pos, cudaStream_t st);
+
+// Statistics of an arbitrary vector (used for the hidden state entering a window) and copy.
+int launch_copy_stats(const float* src, float* dst, int64_t width, int n_tok, VecStats* stats, cudaStream_t st);
+
+// cos/sin table for positions pos..pos+n_tok-1: tab[t][i] = (cos, sin)(pos_t * theta^(-2i/128)),
+// evaluated in double precision.
+int launch_rope_table(float2* tab, int pos, int n_tok, float theta, cudaStream_t st);
+
+// Grouped-query decode attention over the fp16 cache, split along the context, merged by
+// log-sum-exp.  q: [n_tok][H*128] fp32 (rotated).  Cache layout [G][capacity][128] binary16.
+// o: [n_tok][H*128] fp32 with statistics (max |o| per head).
+struct AttnScratch {
+  float* o_part;    // [n_tok*H][n_chunks][128]
+  float2* ml_part;  // [n_tok*H][n_chunks]  (running max, running sum)
+  int max_chunks;
+};
+int launch_attention(const float* q, const __half* k_cache, const __half* v_cache, int kv_capacity, int n_q_heads,
+                     int n_kv_heads, int pos, int n_tok, const AttnScratch& scr, float* o, VecStats* stats,
+                     cudaStream_t st);
+int attention_chunk_len();
+
+// Embedding lookup from a standard-layout table, and greedy argmax.
+int launch_embed(const uint8_t* table_std, int64_t n_sb_per_row, const int32_t* dev_tokens, int n_tok, float* out,
+                 cudaStream_t st);
+int launch_argmax(const float* logits, int64_t vocab, int n_tok, float* scratch_val, int32_t* scratch_idx,
+                  int32_t* dev_out, cudaStream_t st);
+constexpr int kArgmaxBlocks = 128;
+
+inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? 0 : -static_cast<int>(e); }
+
+}  // namespace prima

@@ -1,0 +1,195 @@
+"""GPU parity of layer windows, logits and greedy decoding against the CPU checker, through the C ABI."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2504_08791_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = 2e-2          # absolute, on the final logits
+HIDDEN_TOL = 2e-3         # of the vector's RMS, per element, after a window
+MARGIN = 2 * LOGIT_TOL    # greedy tokens must agree wherever the checker's top-2 gap exceeds this
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    from paper_2504_08791_b200 import binding
+    assert torch.cuda.is_available()
+    binding.lib()
+    return torch, binding
+
+
+class Pair:
+    """The same synthetic model loaded into the checker and into a GPU context."""
+
+    def __init__(self, gpu, cfg, seed, n_prefill, layers=None, with_globals=True):
+        self.torch, self.binding = gpu
+        self.cfg, self.seed = cfg, seed
+        self.ref = oracle.Model(cfg)
+        self.ctx = self.binding.Context(cfg)
+        for layer, tid, rows, cols, data in synth.iter_model_tensors(seed, cfg, layers=layers, with_globals=with_globals):
+            self.ref.load(layer, tid, data, rows, cols)
+            self.ctx.load(layer, tid, data, rows, cols)
+        for l in (range(cfg["n_layers"]) if layers is None else layers):
+            if n_prefill:
+                k, v = synth.kv_prefill(seed, l, n_prefill, cfg["n_kv_heads"], cfg["head_dim"])
+                self.ref.kv_load(l, 0, k, v)
+                self.ctx.kv_load(l, 0, k, v)
+
+    def gpu_window(self, lb, le, h, pos):
+        t = self.torch
+        n_tok = h.shape[0]
+        hin = t.from_numpy(np.ascontiguousarray(h, np.float32)).cuda()
+        hout = t.empty_like(hin)
+        self.ctx.forward_window(lb, le, hin, hout, pos, n_tok)
+        self.ctx.sync()
+        return hout.cpu().numpy()
+
+    def gpu_logits(self, h):
+        t = self.torch
+        hin = t.from_numpy(np.ascontiguousarray(h, np.float32)).cuda()
+        out = t.empty((h.shape[0], self.cfg["vocab"]), dtype=t.float32, device="cuda")
+        self.ctx.logits(hin, h.shape[0], out)
+        self.ctx.sync()
+        return out.cpu().numpy()
+
+    def close(self):
+        self.ctx.close()
+        self.ref.close()
+
+
+def _hidden_close(got, want, tol=HIDDEN_TOL):
+    rms = np.sqrt(np.mean(want.astype(np.float64) ** 2, axis=-1, keepdims=True))
+    err = np.abs(got.astype(np.float64) - want) / rms
+    assert err.max() <= tol, f"hidden differs by {err.max():.2e} of its RMS (allowed {tol:.0e})"
+    return float(err.max())
+
+
+@pytest.mark.parametrize("name,pos,n_tok", [("tiny", 0, 1), ("tiny", 37, 1), ("tiny", 63, 2), ("small", 130, 1), ("small", 255, 5),
+                                            ("small", 64, 8), ("small", 0, 3)])
+def test_full_depth_window_matches_checker(gpu, name, pos, n_tok):
+    cfg = synth.model_config(name)
+    p = Pair(gpu, cfg, seed=11, n_prefill=pos)
+    h0 = synth.activations(11, n_tok, cfg["hidden"])
+    want = p.ref.forward_window(0, cfg["n_layers"], h0, pos)
+    got = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    _hidden_close(got, want)
+    # appended cache entries: binary16 roundings of nearly equal numbers, at most a few ulps apart
+    for l in range(cfg["n_layers"]):
+        kr, vr = p.ref.kv_read(l, pos, n_tok)
+        kg, vg = p.ctx.kv_read(l, pos, n_tok)
+        for a, b in ((kr, kg), (vr, vg)):
+            fa, fb = a.view(np.float16).astype(np.float64), b.view(np.float16).astype(np.float64)
+            assert np.abs(fa - fb).max() <= 4e-3 * max(1.0, np.abs(fa).max())
+        if pos:
+            # prefilled entries are untouched
+            k0, v0 = synth.kv_prefill(11, l, pos, cfg["n_kv_heads"], cfg["head_dim"])
+            kg, vg = p.ctx.kv_read(l, 0, pos)
+            assert np.array_equal(kg, k0) and np.array_equal(vg, v0)
+    logits_ref = p.ref.logits(want)
+    logits_gpu = p.gpu_logits(got)
+    assert np.abs(logits_gpu.astype(np.float64) - logits_ref).max() <= LOGIT_TOL
+    p.close()
+
+
+@pytest.mark.parametrize("splits", [[(0, 1), (1, 2), (2, 3), (3, 4)], [(0, 2), (2, 4)], [(0, 1), (1, 4)], [(0, 3), (3, 4)]])
+@pytest.mark.parametrize("n_tok", [1, 5])
+def test_window_splits_are_bit_identical_on_the_gpu(gpu, splits, n_tok):
+    cfg = synth.model_config("small")
+    pos = 100
+    h0 = synth.activations(13, n_tok, cfg["hidden"])
+    full = Pair(gpu, cfg, seed=13, n_prefill=pos, with_globals=False)
+    want = full.gpu_window(0, cfg["n_layers"], h0, pos)
+    part = Pair(gpu, cfg, seed=13, n_prefill=pos, with_globals=False)
+    h = h0
+    for lb, le in splits:
+        h = part.gpu_window(lb, le, h, pos)
+    assert np.array_equal(h.view(np.uint32), want.view(np.uint32))
+    for l in range(cfg["n_layers"]):
+        for a, b in zip(full.ctx.kv_read(l, 0, pos + n_tok), part.ctx.kv_read(l, 0, pos + n_tok)):
+            assert np.array_equal(a, b)
+    full.close()
+    part.close()
+
+
+def test_five_token_step_agrees_with_five_single_steps_on_the_gpu(gpu):
+    cfg = synth.model_config("small")
+    pos = 77
+    h0 = synth.activations(17, 5, cfg["hidden"])
+    a = Pair(gpu, cfg, seed=17, n_prefill=pos, with_globals=False)
+    batch = a.gpu_window(0, cfg["n_layers"], h0, pos)
+    single = np.concatenate([a.gpu_window(0, cfg["n_layers"], h0[t:t + 1], pos + t) for t in range(5)])
+    _hidden_close(batch, single)
+    a.close()
+
+
+def test_llama8b_shaped_layer_with_1024_cached_positions(gpu):
+    cfg = synth.model_config("8b", n_layers=1, vocab=1024)
+    pos = 1024
+    p = Pair(gpu, cfg, seed=1, n_prefill=pos, with_globals=False)
+    h0 = synth.activations(1, 1, cfg["hidden"])
+    want = p.ref.forward_window(0, 1, h0, pos)
+    got = p.gpu_window(0, 1, h0, pos)
+    _hidden_close(got, want)
+    p.close()
+
+
+def test_greedy_decode_64_tokens_matches_checker(gpu):
+    torch, binding = gpu
+    cfg = synth.model_config("small")
+    n_prefill, steps = 40, 64
+    p = Pair(gpu, cfg, seed=19, n_prefill=n_prefill)
+    hid = torch.empty((1, cfg["hidden"]), dtype=torch.float32, device="cuda")
+    logits = torch.empty((1, cfg["vocab"]), dtype=torch.float32, device="cuda")
+    tok = 0
+    low_margin = 0
+    for step in range(steps):
+        pos = n_prefill + step
+        # checker
+        h_ref = p.ref.forward_window(0, cfg["n_layers"], p.ref.embed([tok]), pos)
+        l_ref = p.ref.logits(h_ref)[0]
+        want_tok, margin = oracle.argmax(l_ref)
+        # GPU, all through the ABI
+        p.ctx.embed([tok], hid)
+        p.ctx.forward_window(0, cfg["n_layers"], hid, hid, pos, 1)
+        p.ctx.logits(hid, 1, logits)
+        got_tok = int(p.ctx.argmax(logits, 1)[0])
+        l_gpu = logits.cpu().numpy()[0]
+        assert np.abs(l_gpu.astype(np.float64) - l_ref).max() <= LOGIT_TOL, f"step {step}"
+        assert got_tok == int(np.argmax(l_gpu))           # the device argmax is the argmax of the device logits
+        if margin > MARGIN:
+            assert got_tok == want_tok, f"step {step}: margin {margin}"
+        else:
+            low_margin += 1
+        tok = want_tok                                    # both sides continue from the checker's token
+    assert low_margin <= 8, f"{low_margin} of {steps} steps had a top-2 gap below {MARGIN}"
+    p.close()
+
+
+def test_errors_leave_the_context_usable(gpu):
+    torch, binding = gpu
+    cfg = synth.model_config("tiny")
+    ctx = binding.Context(cfg)
+    h = torch.zeros((1, cfg["hidden"]), dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.PrimaError) as e:
+        ctx.forward_window(0, 1, h, h, 0, 1)              # nothing loaded yet
+    assert e.value.code == binding.ERR_STATE
+    for layer, tid, rows, cols, data in synth.iter_model_tensors(3, cfg, layers=[0], with_globals=False):
+        ctx.load(layer, tid, data, rows, cols)
+    for bad in [dict(lb=0, le=2, pos=0, n=1), dict(lb=0, le=1, pos=cfg["kv_capacity"], n=1), dict(lb=0, le=1, pos=0, n=9),
+                dict(lb=1, le=0, pos=0, n=1), dict(lb=0, le=1, pos=-1, n=1)]:
+        with pytest.raises(binding.PrimaError):
+            ctx.forward_window(bad["lb"], bad["le"], h, h, bad["pos"], bad["n"])
+    w = synth.model_tensor(3, 0, synth.WQ, 512, 512)
+    with pytest.raises(binding.PrimaError):
+        ctx.load(0, synth.WQ, w, 512, 256)                # wrong shape
+    with pytest.raises(binding.PrimaError):
+        ctx.load(5, synth.WQ, w, 512, 512)                # layer out of range
+    with pytest.raises(binding.PrimaError):
+        ctx.load(0, 99, w, 512, 512)
+    ctx.forward_window(0, 1, h, h, 0, 1)                  # still works
+    ctx.sync()
+    assert ctx.launch_count() > 0
+    ctx.close()
