@@ -489,6 +489,7 @@ int64_t prima_launch_count(prima_ctx* c) { return c ? c->launches : 0; }
 
 // ---- context-free primitives ------------------------------------------------------------------
 int prima_dequant_q4k(const void* dev_blocks, int64_t n_superblocks, float* dev_out, void* stream) {
+  if (n_superblocks == 0) return PRIMA_OK;
   if (!dev_blocks || !dev_out || n_superblocks < 0) return fail(nullptr, PRIMA_ERR_ARG, "prima_dequant_q4k: bad argument");
   int k = launch_dequant_std(static_cast<const uint8_t*>(dev_blocks), n_superblocks, dev_out, static_cast<cudaStream_t>(stream));
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "dequant kernel");

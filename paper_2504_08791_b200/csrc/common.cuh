@@ -23,12 +23,9 @@ namespace prima {
 //                     the 32 weights of row g, sub-block t
 //   bytes  640..1151  the same for sub-blocks 4..7 (lane (g, t) owns sub-block 4 + t)
 //
-// Inside a 16-byte sub-block chunk, word w (0..3) holds weights 8w..8w+7 with nibble positions
-//   bits 0-3: 8w+0   bits 16-19: 8w+1   bits 4-7: 8w+2   bits 20-23: 8w+3
-//   bits 8-11: 8w+4  bits 24-27: 8w+5   bits 12-15: 8w+6 bits 28-31: 8w+7
-// so that (word & 0x000f000f) is a pair of consecutive weights sitting in the low mantissa bits of
-// two binary16 lanes (value q * 2^-24, a subnormal, exact), (word & 0x00f000f0) the next pair
-// scaled by 16, and the same two masks applied to word >> 8 give the remaining two pairs.
+// Inside a 16-byte sub-block chunk, word w (0..3) holds weights 8w..8w+7, weight 8w+i in bits
+// 4i..4i+3, so that (word & 0x0f0f0f0f) is four weights (8w, 8w+2, 8w+4, 8w+6) as unsigned bytes and
+// ((word >> 4) & 0x0f0f0f0f) the other four: ready-made operands of the 4-way byte dot product.
 //
 // Units are stored column-major over the (row tile, super-block column) grid:
 //   offset(s, rt) = (s * n_rt + rt) * 1152

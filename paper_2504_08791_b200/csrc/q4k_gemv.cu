@@ -5,18 +5,18 @@
 // is also its position in memory.  The grid is persistent (a fixed number of CTAs per SM); the
 // U units are cut into one contiguous range per warp, so every warp streams one contiguous slice
 // of HBM, and all warps get the same number of units to within one.  A warp therefore stays at
-// one column s for (almost) its whole range and keeps that column's 256 activations in registers
-// as binary16 pairs.
+// one column s for (almost) its whole range and keeps that column's 256 activations in registers.
 //
 // Arithmetic.  Lane (g, t) = (lane / 4, lane % 4) owns row g of the tile and sub-blocks t and
 // 4 + t of the super-block: two 16-byte nibble chunks plus the 16-byte header of its row.
-// Nibbles are never converted: masked in place they are binary16 subnormals q * 2^-24 (or
-// q * 2^-20 for the odd pairs), which HFMA2 multiplies exactly by the binary16 activations.
-// Each sub-block is accumulated in two binary16x2 chains of 8 products, promoted to fp32, scaled
-// by d*sc, and the -dmin*m term uses the per-sub-block activation sums held in fp32.  Activations
-// are pre-scaled by a power of two chosen from the vector's max |x| so that the largest lies in
-// [2^14, 2^15): products and chain sums stay well inside binary16's range and the scale is undone
-// exactly on the fp32 result.
+// The activations of a sub-block are held as 16-bit integers x_q = round(x / s_j), with one fp32
+// step s_j = max|x| / 32767 per sub-block, split into a signed high byte and an unsigned low byte.
+// Nibbles are masked in place into unsigned bytes and multiplied with the 4-way byte dot product
+// (dp4a): I_j = sum q * x_q is an exact integer below 2^24, so the only rounding errors are the
+// 16-bit step of x (about 2e-5 of a typical activation) and a handful of fp32 operations per
+// sub-block:  partial = d * sum_j sc_j * s_j * I_j  -  dmin * sum_j m_j * s_j * sum(x_q).
+// With RMSNorm fused, x is multiplied by the gain before quantisation and the scalar
+// rsqrt(mean(x^2) + eps) is applied to the fp32 partial.
 //
 // Output.  Each unit yields 8 row partials per token; they are written to
 //   part[(s * n_tok + t) * mpad + row]
@@ -40,62 +40,95 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   return v;
 }
 
-__device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<__half2*>(&v); }
-
-// Eight weights of one 32-bit word against four activation pairs; lo collects the pairs whose
-// nibbles sit at mantissa bits 0..3 (q * 2^-24), hi those at bits 4..7 (q * 2^-20).
-__device__ __forceinline__ void word_fma(uint32_t w, const __half2* x, __half2& lo, __half2& hi) {
-  const uint32_t w8 = w >> 8;
-  lo = __hfma2(as_h2(w & 0x000f000fu), x[0], lo);
-  hi = __hfma2(as_h2(w & 0x00f000f0u), x[1], hi);
-  lo = __hfma2(as_h2(w8 & 0x000f000fu), x[2], lo);
-  hi = __hfma2(as_h2(w8 & 0x00f000f0u), x[3], hi);
+// 4-way byte dot products: unsigned nibble bytes times signed / unsigned activation bytes.
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
+  int d;
+  asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t dp4a_uu(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
 }
 
-// sum over 32 weights of q * xs, in units of 2^-24
-__device__ __forceinline__ float chunk_dot(const uint4& q, const __half2* x) {
-  __half2 lo = __float2half2_rn(0.f), hi = __float2half2_rn(0.f);
-  word_fma(q.x, x + 0, lo, hi);
-  word_fma(q.y, x + 4, lo, hi);
-  word_fma(q.z, x + 8, lo, hi);
-  word_fma(q.w, x + 12, lo, hi);
-  const float2 l = __half22float2(lo), h = __half22float2(hi);
-  return (l.x + l.y) + (h.x + h.y) * 0.0625f;
-}
+// The 32 activations of one sub-block as bytes: hi[2w + p] / lo[2w + p] hold the high / low bytes of
+// x_q for weights 8w + p, 8w + p + 2, 8w + p + 4, 8w + p + 6 (p = 0 even nibbles, 1 odd nibbles).
+struct SubX {
+  uint32_t hi[8], lo[8];
+  float step;       // s_j
+  float step_sum;   // s_j * sum(x_q)
+};
 
-// Reduce the statistics blocks of one token the same way in every warp.
-__device__ __forceinline__ void token_scale(const float2* __restrict__ stats, int n_blocks, int tok, int64_t cols,
-                                            bool has_norm, float eps, float gain_max, float& mul, float& post) {
-  const int lane = threadIdx.x & 31;
-  float ss = 0.f, am = 0.f;
-  for (int b = lane; b < n_blocks; b += 32) {
-    const float2 v = stats[tok * kMaxStatBlocks + b];
-    ss += v.x;
-    am = fmaxf(am, v.y);
-  }
+// sum over the 32 weights of q * x_q (exact)
+__device__ __forceinline__ int chunk_dot(const uint4& q, const SubX& x) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  int he = 0, ho = 0;
+  uint32_t le = 0, lo = 0;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t e = w[i] & 0x0f0f0f0fu, o = (w[i] >> 4) & 0x0f0f0f0fu;
+    he = dp4a_us(e, x.hi[2 * i], he);
+    ho = dp4a_us(o, x.hi[2 * i + 1], ho);
+    le = dp4a_uu(e, x.lo[2 * i], le);
+    lo = dp4a_uu(o, x.lo[2 * i + 1], lo);
   }
-  const float inv = has_norm ? 1.0f / sqrtf(ss / static_cast<float>(cols) + eps) : 1.0f;
-  const float amax = am * gain_max * inv;
-  int k = 0;
-  if (amax > 0.f && amax < 3.0e38f) {
-    int e;
-    frexpf(amax, &e);        // amax < 2^e
-    k = 15 - e;              // largest scaled activation < 2^15
-    k = max(-100, min(100, k));
+  return (he + ho) * 256 + static_cast<int>(le + lo);
+}
+
+// Quantise 32 consecutive activations (times gain, if any) into a SubX.
+__device__ __forceinline__ void load_sub(const float* __restrict__ xp, const float* __restrict__ gp, SubX& out) {
+  float v[32];
+  float amax = 0.f;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    float4 a = *reinterpret_cast<const float4*>(xp + 4 * c);
+    if (gp) {
+      const float4 gv = *reinterpret_cast<const float4*>(gp + 4 * c);
+      a.x *= gv.x; a.y *= gv.y; a.z *= gv.z; a.w *= gv.w;
+    }
+    v[4 * c] = a.x; v[4 * c + 1] = a.y; v[4 * c + 2] = a.z; v[4 * c + 3] = a.w;
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
   }
-  mul = ldexpf(inv, k);
-  post = ldexpf(1.0f, -k);
+  const bool ok = amax > 0.f && amax < 3.0e38f;
+  const float inv_step = ok ? 32767.0f / amax : 0.f;
+  int sum = 0;
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      uint32_t hi = 0, lo = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        int xq = __float2int_rn(v[8 * w + 2 * b + p] * inv_step);
+        xq = max(-32767, min(32767, xq));
+        sum += xq;
+        hi |= (static_cast<uint32_t>(xq >> 8) & 0xffu) << (8 * b);
+        lo |= (static_cast<uint32_t>(xq) & 0xffu) << (8 * b);
+      }
+      out.hi[2 * w + p] = hi;
+      out.lo[2 * w + p] = lo;
+    }
+  }
+  out.step = ok ? amax / 32767.0f : 0.f;
+  out.step_sum = out.step * static_cast<float>(sum);
+}
+
+// rsqrt(mean(x^2) + eps) of one token from the statistics blocks, reduced the same way in every warp.
+__device__ __forceinline__ float token_inv_rms(const float2* __restrict__ stats, int n_blocks, int tok, int64_t cols, float eps) {
+  const int lane = threadIdx.x & 31;
+  float ss = 0.f;
+  for (int b = lane; b < n_blocks; b += 32) ss += stats[tok * kMaxStatBlocks + b].x;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  return 1.0f / sqrtf(ss / static_cast<float>(cols) + eps);
 }
 
 template <int NTOK>
 __global__ void __launch_bounds__(kWarpsPerCta * 32, (NTOK == 1 ? 2 : 1))
 gemv_partials_kernel(const uint8_t* __restrict__ w, int64_t n_rt, int64_t n_sb, int64_t cols, const float* __restrict__ x,
-                     const float* __restrict__ gain, float gain_max, float eps, const float2* __restrict__ stats,
-                     int n_stat_blocks, int tok0, int n_tok_total, float* __restrict__ part, int64_t mpad) {
+                     const float* __restrict__ gain, float eps, const float2* __restrict__ stats, int n_stat_blocks, int tok0,
+                     int n_tok_total, float* __restrict__ part, int64_t mpad) {
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -119,17 +152,15 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int64_t n_rt, int64_t n_sb, 
     }
   }
 
-  float mul[NTOK], post[NTOK];
+  float post[NTOK];
 #pragma unroll
-  for (int k = 0; k < NTOK; ++k)
-    token_scale(stats, n_stat_blocks, tok0 + k, cols, gain != nullptr, eps, gain_max, mul[k], post[k]);
+  for (int k = 0; k < NTOK; ++k) post[k] = gain ? token_inv_rms(stats, n_stat_blocks, tok0 + k, cols, eps) : 1.0f;
 
   // lane-constant byte selectors that pull this lane's 24-bit field group out of header words 1..3
   const uint32_t sel_a = t == 1 ? 0x7654u : (t == 3 ? 0x0073u : 0x3210u);
   const uint32_t sel_b = t == 2 ? 0x7654u : (t == 3 ? 0x0710u : 0x3210u);
 
-  __half2 xr[NTOK][32];
-  float x_lo[NTOK], x_hi[NTOK];
+  SubX xa[NTOK], xb[NTOK];   // sub-blocks t and 4 + t of the current column
   int64_t cur_s = -1;
 
   for (int64_t ub = u0; ub < u1; ub += kPipe) {
@@ -151,27 +182,8 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int64_t n_rt, int64_t n_sb, 
           for (int k = 0; k < NTOK; ++k) {
             const float* xp = x + static_cast<int64_t>(tok0 + k) * cols + s * 256 + 32 * t;
             const float* gp = gain ? gain + s * 256 + 32 * t : nullptr;
-            float sum_lo = 0.f, sum_hi = 0.f;
-#pragma unroll
-            for (int hlf = 0; hlf < 2; ++hlf) {
-#pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                float4 v = *reinterpret_cast<const float4*>(xp + 128 * hlf + 4 * c);
-                if (gp) {
-                  const float4 gv = *reinterpret_cast<const float4*>(gp + 128 * hlf + 4 * c);
-                  v.x *= gv.x; v.y *= gv.y; v.z *= gv.z; v.w *= gv.w;
-                }
-                const __half2 a = __floats2half2_rn(v.x * mul[k], v.y * mul[k]);
-                const __half2 b = __floats2half2_rn(v.z * mul[k], v.w * mul[k]);
-                xr[k][16 * hlf + 2 * c] = a;
-                xr[k][16 * hlf + 2 * c + 1] = b;
-                const float2 af = __half22float2(a), bf = __half22float2(b);
-                if (hlf == 0) sum_lo += (af.x + af.y) + (bf.x + bf.y);
-                else sum_hi += (af.x + af.y) + (bf.x + bf.y);
-              }
-            }
-            x_lo[k] = sum_lo;
-            x_hi[k] = sum_hi;
+            load_sub(xp, gp, xa[k]);
+            load_sub(xp + 128, gp ? gp + 128 : nullptr, xb[k]);
           }
         }
         const float d = __half2float(__ushort_as_half(static_cast<unsigned short>(r.h.x & 0xffffu)));
@@ -179,14 +191,13 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int64_t n_rt, int64_t n_sb, 
         const uint32_t f = __byte_perm(__byte_perm(r.h.y, r.h.z, sel_a), r.h.w, sel_b);
         const float sc_lo = static_cast<float>(f & 63u), sc_hi = static_cast<float>((f >> 6) & 63u);
         const float m_lo = static_cast<float>((f >> 12) & 63u), m_hi = static_cast<float>((f >> 18) & 63u);
-        const float d24 = d * 16777216.0f;
 #pragma unroll
         for (int k = 0; k < NTOK; ++k) {
-          const float a0 = chunk_dot(r.q0, &xr[k][0]);
-          const float a1 = chunk_dot(r.q1, &xr[k][16]);
-          const float t1 = sc_lo * a0 + sc_hi * a1;
-          const float t2 = m_lo * x_lo[k] + m_hi * x_hi[k];
-          float acc = d24 * t1 - dmin * t2;
+          const float i0 = static_cast<float>(chunk_dot(r.q0, xa[k]));
+          const float i1 = static_cast<float>(chunk_dot(r.q1, xb[k]));
+          const float t1 = sc_lo * (xa[k].step * i0) + sc_hi * (xb[k].step * i1);
+          const float t2 = m_lo * xa[k].step_sum + m_hi * xb[k].step_sum;
+          float acc = d * t1 - dmin * t2;
           acc += __shfl_xor_sync(0xffffffffu, acc, 1);
           acc += __shfl_xor_sync(0xffffffffu, acc, 2);
           if (t == 0) part[(s * n_tok_total + tok0 + k) * mpad + rt * kRowsPerTile + g] = acc * post[k];
@@ -212,12 +223,10 @@ int launch_gemv_partials(const TiledMat& w, const GemvIn& in, int n_tok, float* 
     if (grid > max_useful) grid = max_useful;
     if (chunk == 1)
       gemv_partials_kernel<1><<<static_cast<unsigned>(grid), block, 0, st>>>(
-          w.data, w.n_rt, w.n_sb, w.cols, in.x, in.gain, in.gain_max, in.eps, in.stats.data, in.stats.n_blocks, tok,
-          n_tok, part, w.mpad());
+          w.data, w.n_rt, w.n_sb, w.cols, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok, n_tok, part, w.mpad());
     else
       gemv_partials_kernel<2><<<static_cast<unsigned>(grid), block, 0, st>>>(
-          w.data, w.n_rt, w.n_sb, w.cols, in.x, in.gain, in.gain_max, in.eps, in.stats.data, in.stats.n_blocks, tok,
-          n_tok, part, w.mpad());
+          w.data, w.n_rt, w.n_sb, w.cols, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok, n_tok, part, w.mpad());
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_rc(e);
     ++launches;

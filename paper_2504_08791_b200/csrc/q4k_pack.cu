@@ -93,13 +93,13 @@ __global__ void retile_kernel(const uint8_t* __restrict__ src, int64_t rows_src,
     uint32_t words[4];
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-      uint32_t q[8];
+      uint32_t word = 0;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const uint32_t byte = qs[32 * p + 8 * w + i];
-        q[i] = hi ? (byte >> 4) : (byte & 15u);
+        word |= (hi ? (byte >> 4) : (byte & 15u)) << (4 * i);
       }
-      words[w] = q[0] | (q[2] << 4) | (q[4] << 8) | (q[6] << 12) | (q[1] << 16) | (q[3] << 20) | (q[5] << 24) | (q[7] << 28);
+      words[w] = word;
     }
     const int half_idx = j >> 2, t = j & 3;
     uint8_t* chunk = unit + kUnitHdrBytes + half_idx * 512 + (g * 4 + t) * 16;
