@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Decode benchmark of the Q4_K layer-window hot path.
+
+One "step" is one decoded token: the hidden state of the newest token goes through every layer of
+the model, issued as contiguous layer windows (4 windows of 20 layers for the 70B shape, the
+paper's ring schedule with window 20), then through the output layer.  Weights are synthetic
+random-init Q4_K tensors of the named shape; the KV cache is prefilled with N(0,1) fp16 entries.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 70b|32b|8b] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank decodes its own request on its own
+GPU: the path does not shard, ranks are independent replicas and no collective is on the data
+path; the barrier and the max-over-ranks reduction only bracket the timing.
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2504_08791_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (shape, context length, number of windows, description)
+    "70b": ("70b", 4096, 4, "Llama-3-70B-shaped random-init Q4_K, 80 layers as 4 windows x 20, fp16 KV context 4096, batch 1"),
+    "32b": ("32b", 4096, 1, "Qwen2.5-32B-shaped random-init Q4_K, 64 layers, fp16 KV context 4096, batch 1"),
+    "8b": ("8b", 1024, 1, "Llama-3-8B-shaped random-init Q4_K, 32 layers, fp16 KV context 1024, batch 1"),
+}
+SEEDS = {"70b": 3, "32b": 2, "8b": 1}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def bytes_per_token(cfg: dict, n_ctx: int, n_layers: int | None = None, with_head: bool = True) -> dict:
+    """Algorithmic bytes one decoded token must move: Q4_K weight bytes touched + K and V bytes of
+    the attended positions (the paper's device-loading model: b + 2(h_k e_k + h_v e_v) n_kv per
+    layer, b_o for the output layer)."""
+    L = cfg["n_layers"] if n_layers is None else n_layers
+    layer_w = synth.weight_bytes(cfg, (synth.WQ, synth.WK, synth.WV, synth.WO, synth.W_GATE, synth.W_UP, synth.W_DOWN))
+    kv = 2 * (cfg["n_kv_heads"] * cfg["head_dim"] * 2) * n_ctx
+    head = synth.weight_bytes(cfg, (synth.W_HEAD,)) if with_head else 0
+    return dict(layer_weights=layer_w, layer_kv=kv, head=head, total=L * (layer_w + kv) + head)
+
+
+# ------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """nvidia-smi sampled every 200 ms while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.device = device
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "200",
+                                          "-i", str(self.device)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) >= 9:
+                    rows.append(f)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not rows:
+            return out
+        sm = [float(r[1]) for r in rows if r[1].replace(".", "").isdigit()]
+        mx = [float(r[2]) for r in rows if r[2].replace(".", "").isdigit()]
+        reasons = set()
+        for r in rows:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        out.update(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None, reasons=sorted(reasons),
+                   samples=len(rows))
+        return out
+
+
+# ------------------------------------------------------------------------------------ the GPU arm
+def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None):
+    import torch
+    t0 = time.time()
+    ctx = binding.Context(cfg, device=device)
+    layers = range(cfg["n_layers"]) if n_layers is None else range(n_layers)
+    for layer, tid, rows, cols, data in synth.iter_model_tensors(seed, cfg, layers=layers):
+        ctx.load(layer, tid, data, rows, cols)
+    t1 = time.time()
+    for l in layers:
+        k, v = synth.kv_prefill(seed, l, n_ctx, cfg["n_kv_heads"], cfg["head_dim"])
+        ctx.kv_load(l, 0, k, v)
+    torch.cuda.synchronize()
+    log(f"[bench] model resident: weights {t1 - t0:.1f}s, kv prefill {time.time() - t1:.1f}s")
+    return ctx
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_2504_08791_b200 import binding
+
+    binding.lib()
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    shape, n_ctx, n_windows, desc = WORKLOADS[args.workload]
+    cfg = synth.model_config(shape)
+    if args.layers:
+        cfg["n_layers"] = args.layers
+    L = cfg["n_layers"]
+    seed = SEEDS[args.workload] + 1000 * rank
+    ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank)
+    bpt = bytes_per_token(cfg, n_ctx)
+    bounds = [L * i // n_windows for i in range(n_windows + 1)]
+
+    h0 = torch.from_numpy(synth.activations(seed, 1, cfg["hidden"])).cuda()
+    hid = torch.empty_like(h0)
+    logits = torch.empty((1, cfg["vocab"]), dtype=torch.float32, device="cuda")
+
+    def device_step(pos):
+        hid.copy_(h0)
+        for w in range(n_windows):
+            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, 1)
+        ctx.logits(hid, 1, logits)
+
+    def e2e_step(tok, pos):
+        ctx.embed([tok], hid)                      # host token id -> device (4 bytes)
+        for w in range(n_windows):
+            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, 1)
+        ctx.logits(hid, 1, logits)
+        return int(ctx.argmax(logits, 1)[0])       # device -> host (4 bytes), waits
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(args.warmup):
+        device_step(n_ctx)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        device_step(n_ctx)
+    ev1.record()
+    barrier()
+    launches = ctx.launch_count() - launches0
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    ms_step = ms_total / args.steps
+
+    # end to end through the ABI: host token in, host token out, every step
+    tok = 0
+    for i in range(min(args.warmup, 3)):
+        tok = e2e_step(tok, n_ctx + i)
+    barrier()
+    e2e_steps = min(args.steps, cfg["kv_capacity"] - n_ctx - 3)
+    ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.perf_counter()
+    ev2.record()
+    for i in range(e2e_steps):
+        tok = e2e_step(tok, n_ctx + 3 + i)
+    ev3.record()
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - wall0) * 1e3
+    e2e_ms = max_over_ranks(max(ev2.elapsed_time(ev3), wall_ms)) / e2e_steps
+    clocks = sampler.stop()
+
+    # dominant kernel: event-bracketed GEMV launches in a separate pass (bracketing perturbs whole-step time)
+    ctx.profile_enable(True)
+    prof_steps = max(1, min(args.steps, 5))
+    for _ in range(prof_steps):
+        device_step(n_ctx)
+    g_ms, g_n, g_bytes = ctx.profile_read(binding.PROF_GEMV)
+    a_ms, a_n, a_bytes = ctx.profile_read(binding.PROF_ATTENTION)
+    ctx.profile_enable(False)
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    gemv_gbs = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
+    attn_gbs = a_bytes / (a_ms * 1e-3) / 1e9 if a_ms > 0 else 0.0
+    step_gbs = bpt["total"] / (ms_step * 1e-3) / 1e9
+
+    result = {
+        "metric": "decode_ms_per_token",
+        "value": ms_step / world,
+        "unit": "ms/token",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step,
+        "higher_is_better": False,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "q4_k weights x int16 activations, int32/fp32 accumulate",
+        "data": "synthetic",
+        "tokens_per_s": world * 1e3 / ms_step,
+        "config": {"workload": desc, "layers": L, "windows": n_windows, "n_ctx": n_ctx, "n_tok": 1,
+                   "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs larger than L2 (>= 4.9 GB per step)",
+                   "bytes_per_token": bpt["total"]},
+        "step_roofline": {"bound": "hbm", "achieved": step_gbs, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                          "frac": step_gbs / peak, "frac_of_nominal_8000": step_gbs / 8000.0},
+        "roofline": {"kernel": "gemv_partials_kernel<1>", "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
+                     "unit": "GB/s", "frac": gemv_gbs / peak, "traffic": None,
+                     "launches": g_n // prof_steps, "avg_launch_us": (g_ms * 1e3 / g_n) if g_n else None,
+                     "timing": f"cuda events around each launch, separate pass of {prof_steps} steps"},
+        "attention_kernel": {"achieved": attn_gbs, "unit": "GB/s", "frac": attn_gbs / peak, "launches": a_n // prof_steps},
+        "e2e": {"value": e2e_ms / world, "unit": "ms/token", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    ctx.close()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return result
+
+
+# ------------------------------------------------------------------------------- the CPU checker arm
+def cpu_baseline(workload: str, budget_s: float = 20.0, repeat: int = 1) -> dict:
+    """The CPU checker as it stands, timed on a bounded sample: one full-width layer at full context."""
+    import oracle
+    shape, n_ctx, _, _ = WORKLOADS[workload]
+    cfg = synth.model_config(shape)
+    seed = SEEDS[workload]
+    cores = oracle.default_threads()
+    one = dict(cfg, n_layers=1)
+    mdl = oracle.Model(one, n_threads=cores)
+    for layer, tid, rows, cols, data in synth.iter_model_tensors(seed, one, with_globals=False):
+        mdl.load(layer, tid, data, rows, cols)
+    k, v = synth.kv_prefill(seed, 0, n_ctx, cfg["n_kv_heads"], cfg["head_dim"])
+    mdl.kv_load(0, 0, k, v)
+    h0 = synth.activations(seed, 1, cfg["hidden"])
+    times = []
+    t_start = time.perf_counter()
+    while len(times) < max(1, repeat) or (time.perf_counter() - t_start < budget_s * 0.5 and len(times) < 8):
+        t0 = time.perf_counter()
+        mdl.forward_window(0, 1, h0, n_ctx)
+        times.append(time.perf_counter() - t0)
+    mdl.close()
+    bpt_layer = bytes_per_token(one, n_ctx, with_head=False)["total"]
+    bpt_all = bytes_per_token(cfg, n_ctx)["total"]
+    per_layer = float(np.median(times))
+    return {"value": per_layer * 1e3 * bpt_all / bpt_layer, "unit": "ms/token", "cores": cores, "kind": "oracle",
+            "sample": f"1 of {cfg['n_layers']} layers at full width and {n_ctx} cached positions, {len(times)} runs, median "
+                      f"{per_layer * 1e3:.0f} ms per layer, scaled to the whole token by algorithmic bytes"}
+
+
+def run_reference(args):
+    shape, n_ctx, n_windows, desc = WORKLOADS[args.workload]
+    vals = []
+    base = None
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        cpu_baseline(args.workload, budget_s=1.0)
+    for _ in range(max(1, min(args.steps, 5))):
+        base = cpu_baseline(args.workload, budget_s=1.0)
+        vals.append(base["value"])
+    v = float(np.median(vals))
+    base["value"] = v
+    cfg = synth.model_config(shape)
+    return {
+        "impl": "reference", "metric": "decode_ms_per_token", "value": v, "unit": "ms/token", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": v, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": desc, "layers": cfg["n_layers"], "windows": n_windows, "n_ctx": n_ctx, "n_tok": 1},
+        "cpu_baseline": base,
+        "e2e": {"value": v, "unit": "ms/token", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="70b", choices=sorted(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+    if args.warmup < 3:
+        log("[bench] fewer than 3 warm-up steps: the number is not a valid measurement")
+    res = run_ours(args, rank, world, local_rank)
+    if rank == 0:
+        print(json.dumps(res), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -149,6 +149,19 @@ const char* prima_last_error(prima_ctx* ctx);
 /* Number of kernels this context has launched since it was created (for accounting). */
 int64_t prima_launch_count(prima_ctx* ctx);
 
+/* Device-side timing by kernel class, for measurement runs (the counterpart of the paper's device
+ * profiler, which measures how fast weights and KV cache reach the cores: Appendix A.3, device
+ * loading time).  While enabled, every launch of the listed classes is bracketed by a pair of
+ * CUDA events on the context's stream; enable(…, 0 or 1) also discards what was recorded.  read
+ * waits for the stream and returns, for one class, the summed event time in milliseconds, the
+ * number of kernel launches and the algorithmic bytes they had to move (Q4_K weight bytes of the
+ * matrices, or K and V bytes of the attended positions).  Timing perturbs the run: keep it off
+ * when measuring whole steps. */
+#define PRIMA_PROF_GEMV 0
+#define PRIMA_PROF_ATTENTION 1
+int prima_profile_enable(prima_ctx* ctx, int on);
+int prima_profile_read(prima_ctx* ctx, int klass, double* ms_total, int64_t* launches, int64_t* algo_bytes);
+
 /* ---- context-free exports of the two primitives (tests and micro-benchmarks) ---------------- */
 
 /* Dequantise n_superblocks blocks (dev, standard 144-byte layout) to fp32 (dev, 256 per block).

@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libprima.so")
 OK, ERR_ARG, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_DEVICE = 0, -1, -2, -3, -4, -5
 ATTN_NORM, WQ, WK, WV, WO, FFN_NORM, W_GATE, W_UP, W_DOWN, OUT_NORM, W_HEAD, TOK_EMBD = range(12)
 MAX_N_TOK = 8
+PROF_GEMV, PROF_ATTENTION = 0, 1
 
 EXPORTS = [
     "prima_ctx_create", "prima_ctx_destroy", "prima_load_q4k_weights", "prima_forward_window", "prima_logits",
     "prima_embed", "prima_argmax", "prima_kv_load", "prima_kv_read", "prima_sync", "prima_last_error",
-    "prima_launch_count", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
+    "prima_launch_count", "prima_profile_enable", "prima_profile_read", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
     "prima_gemv_plan_destroy",
 ]
 
@@ -64,6 +65,8 @@ def lib():
         L.prima_last_error.restype = C.c_char_p
         L.prima_launch_count.argtypes = [vp]
         L.prima_launch_count.restype = i64
+        L.prima_profile_enable.argtypes = [vp, i32]
+        L.prima_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)]
         L.prima_dequant_q4k.argtypes = [vp, i64, vp, vp]
         L.prima_gemv_q4k.argtypes = [vp, i64, i64, vp, i32, vp, vp]
         L.prima_gemv_plan_create.argtypes = [vp, i64, i64, i32, C.POINTER(vp)]
@@ -192,6 +195,15 @@ class Context:
 
     def sync(self):
         _check(lib().prima_sync(self._h), self._h)
+
+    def profile_enable(self, on: bool):
+        _check(lib().prima_profile_enable(self._h, 1 if on else 0), self._h)
+
+    def profile_read(self, klass: int):
+        """(milliseconds, launches, algorithmic bytes) recorded for one kernel class."""
+        ms, n, b = C.c_double(), C.c_int64(), C.c_int64()
+        _check(lib().prima_profile_read(self._h, klass, C.byref(ms), C.byref(n), C.byref(b)), self._h)
+        return ms.value, n.value, b.value
 
     def launch_count(self) -> int:
         return int(lib().prima_launch_count(self._h))

@@ -72,6 +72,11 @@ struct prima_ctx {
   std::vector<void*> allocs;
   std::string err;
   int64_t launches = 0;
+
+  // optional per-class device timing (prima_profile_*)
+  bool profiling = false;
+  struct Span { cudaEvent_t a, b; int klass; int64_t bytes; int launches; };
+  std::vector<Span> spans;
 };
 
 struct prima_gemv_plan {
@@ -179,6 +184,27 @@ int load_norm(prima_ctx* c, float** dst, float* gmax, const void* data, int64_t 
     (c)->launches += k_;                                                            \
   } while (0)
 
+// Same, bracketed by a pair of events when profiling is on.
+#define LAUNCH_P(c, klass_, bytes_, expr, what)                                     \
+  do {                                                                              \
+    prima_ctx::Span sp_{nullptr, nullptr, (klass_), (bytes_), 0};                   \
+    if ((c)->profiling) {                                                           \
+      cudaEventCreate(&sp_.a);                                                      \
+      cudaEventCreate(&sp_.b);                                                      \
+      cudaEventRecord(sp_.a, (c)->stream);                                          \
+    }                                                                               \
+    int k_ = (expr);                                                                \
+    if (k_ < 0) return cuda_fail((c), static_cast<cudaError_t>(-k_), what);         \
+    (c)->launches += k_;                                                            \
+    if ((c)->profiling) {                                                           \
+      cudaEventRecord(sp_.b, (c)->stream);                                          \
+      sp_.launches = k_;                                                            \
+      (c)->spans.push_back(sp_);                                                    \
+    }                                                                               \
+  } while (0)
+
+int64_t q4k_bytes(const TiledMat& t) { return t.rows * t.n_sb * kBlockBytes; }
+
 }  // namespace
 
 // =============================================================================================
@@ -253,6 +279,10 @@ int prima_ctx_destroy(prima_ctx* c) {
   if (!c) return PRIMA_OK;
   DeviceGuard guard(c->cfg.device);
   cudaStreamSynchronize(c->stream);
+  for (auto& sp : c->spans) {
+    cudaEventDestroy(sp.a);
+    cudaEventDestroy(sp.b);
+  }
   for (void* p : c->allocs) cudaFree(p);
   delete c;
   return PRIMA_OK;
@@ -354,18 +384,19 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
   for (int l = layer_begin; l < layer_end; ++l) {
     Layer& L = c->layers[l];
     GemvIn in{c->h, L.g_attn, L.gmax_attn, g.rms_eps, c->st_h};
-    LAUNCH(c, launch_gemv_partials(L.qkv, in, n_tok, c->part, c->sm_count, st), "gemv(qkv)");
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->part, c->sm_count, st), "gemv(qkv)");
     LAUNCH(c, launch_finish_qkv(c->part, L.qkv.n_sb, L.qkv.mpad(), H, G, n_tok, c->rope_tab, g.rope_mode, c->qbuf, L.k, L.v,
                                 g.kv_capacity, pos, st), "finish_qkv");
-    LAUNCH(c, launch_attention(c->qbuf, L.k, L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, &c->st_o, st), "attention");
+    LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos + n_tok),
+             launch_attention(c->qbuf, L.k, L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, &c->st_o, st), "attention");
     GemvIn in_o{c->obuf, nullptr, 1.f, 0.f, c->st_o};
-    LAUNCH(c, launch_gemv_partials(L.o, in_o, n_tok, c->part, c->sm_count, st), "gemv(o)");
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->part, c->sm_count, st), "gemv(o)");
     LAUNCH(c, launch_finish_residual(c->part, L.o.n_sb, L.o.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(o)");
     GemvIn in_f{c->h, L.g_ffn, L.gmax_ffn, g.rms_eps, c->st_h};
-    LAUNCH(c, launch_gemv_partials(L.gu, in_f, n_tok, c->part, c->sm_count, st), "gemv(gate/up)");
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->part, c->sm_count, st), "gemv(gate/up)");
     LAUNCH(c, launch_finish_swiglu(c->part, L.gu.n_sb, L.gu.mpad(), g.ffn, n_tok, c->act, &c->st_act, st), "finish_swiglu");
     GemvIn in_d{c->act, nullptr, 1.f, 0.f, c->st_act};
-    LAUNCH(c, launch_gemv_partials(L.down, in_d, n_tok, c->part, c->sm_count, st), "gemv(down)");
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->part, c->sm_count, st), "gemv(down)");
     LAUNCH(c, launch_finish_residual(c->part, L.down.n_sb, L.down.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(down)");
   }
   cudaError_t e = cudaMemcpyAsync(hidden_out, c->h, static_cast<size_t>(n_tok) * e_ * 4, cudaMemcpyDeviceToDevice, st);
@@ -382,7 +413,7 @@ int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
   cudaStream_t st = c->stream;
   LAUNCH(c, launch_copy_stats(hidden, nullptr, c->cfg.hidden, n_tok, &c->st_h, st), "copy_stats");
   GemvIn in{hidden, c->g_out, c->gmax_out, c->cfg.rms_eps, c->st_h};
-  LAUNCH(c, launch_gemv_partials(c->head, in, n_tok, c->part, c->sm_count, st), "gemv(head)");
+  LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->part, c->sm_count, st), "gemv(head)");
   LAUNCH(c, launch_finish_plain(c->part, c->head.n_sb, c->head.mpad(), c->cfg.vocab, n_tok, logits, st), "finish_plain");
   return PRIMA_OK;
 }
@@ -480,6 +511,41 @@ int prima_sync(prima_ctx* c) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync");
   if (status != 0) return fail(c, PRIMA_ERR_DEVICE, "a kernel raised the device status word: " + std::to_string(status));
+  return PRIMA_OK;
+}
+
+int prima_profile_enable(prima_ctx* c, int on) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_profile_enable: null context");
+  DeviceGuard guard(c->cfg.device);
+  cudaStreamSynchronize(c->stream);
+  for (auto& sp : c->spans) {
+    cudaEventDestroy(sp.a);
+    cudaEventDestroy(sp.b);
+  }
+  c->spans.clear();
+  c->profiling = on != 0;
+  return PRIMA_OK;
+}
+
+int prima_profile_read(prima_ctx* c, int klass, double* ms_total, int64_t* launches, int64_t* algo_bytes) {
+  if (!c || !ms_total || !launches || !algo_bytes) return fail(c, PRIMA_ERR_ARG, "prima_profile_read: null argument");
+  DeviceGuard guard(c->cfg.device);
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "prima_profile_read");
+  double ms = 0;
+  int64_t n = 0, bytes = 0;
+  for (auto& sp : c->spans) {
+    if (sp.klass != klass) continue;
+    float t = 0.f;
+    e = cudaEventElapsedTime(&t, sp.a, sp.b);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaEventElapsedTime");
+    ms += t;
+    n += sp.launches;
+    bytes += sp.bytes;
+  }
+  *ms_total = ms;
+  *launches = n;
+  *algo_bytes = bytes;
   return PRIMA_OK;
 }
 
