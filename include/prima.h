@@ -184,6 +184,25 @@ int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int ma
 int prima_gemv_plan_run(prima_gemv_plan* plan, const float* dev_x, int n_cols, float* dev_y, void* stream);
 int prima_gemv_plan_destroy(prima_gemv_plan* plan);
 
+/* The same product as prima_gemv_q4k for callers that cannot allocate device memory: programs that
+ * gave all of the GPU's memory to their own arena at start-up, or latency-critical loops in which
+ * cudaMalloc / cudaFree (which may stall the device, and may fail late) are not allowed.  The paper
+ * has no counterpart of this call; it exists only for such callers.
+ *   dev_w: standard 144-byte block layout, rows*(cols/256) blocks; dev_x: fp32 [n_cols x cols];
+ *   dev_y: fp32 [n_cols x rows]; all device memory owned by the caller; stream: cudaStream_t or NULL.
+ * Nothing is allocated or freed, here or in anything it calls: the partial sums live in a 16 MiB
+ * array built into the library (each GPU that loads the library holds it until exit).  Limit:
+ * rows * (cols/256) * n_cols <= 4,194,304; larger products return PRIMA_ERR_ARG with a message
+ * that says so.  The first call on a device looks up the array's device address; make that
+ * first call before any stream capture begins.  The call queues its kernels on `stream` and
+ * returns without waiting.  All calls on a device share the array: calls whose kernels may
+ * overlap on the GPU (different streams without ordering) corrupt each other; calls ordered on a
+ * stream, or by events, are safe, and nothing has to be cleared between them.
+ * prima_gemv_q4k_noalloc_error returns this thread's last message from this call ("" if none). */
+int prima_gemv_q4k_noalloc(const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols,
+                           float* dev_y, void* stream);
+const char* prima_gemv_q4k_noalloc_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,7 @@ EXPORTS = [
     "prima_ctx_create", "prima_ctx_destroy", "prima_load_q4k_weights", "prima_forward_window", "prima_logits",
     "prima_embed", "prima_argmax", "prima_kv_load", "prima_kv_read", "prima_sync", "prima_last_error",
     "prima_launch_count", "prima_profile_enable", "prima_profile_read", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
-    "prima_gemv_plan_destroy",
+    "prima_gemv_plan_destroy", "prima_gemv_q4k_noalloc", "prima_gemv_q4k_noalloc_error",
 ]
 
 
@@ -72,8 +72,11 @@ def lib():
         L.prima_gemv_plan_create.argtypes = [vp, i64, i64, i32, C.POINTER(vp)]
         L.prima_gemv_plan_run.argtypes = [vp, vp, i32, vp, vp]
         L.prima_gemv_plan_destroy.argtypes = [vp]
+        L.prima_gemv_q4k_noalloc.argtypes = [vp, i64, i64, vp, i32, vp, vp]
+        L.prima_gemv_q4k_noalloc_error.argtypes = []
+        L.prima_gemv_q4k_noalloc_error.restype = C.c_char_p
         for name in EXPORTS:
-            if name not in ("prima_last_error", "prima_launch_count"):
+            if name not in ("prima_last_error", "prima_launch_count", "prima_gemv_q4k_noalloc_error"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -109,6 +112,16 @@ def prima_dequant_q4k(dev_blocks, n_superblocks: int, dev_out, stream=None):
 
 def prima_gemv_q4k(dev_w, rows: int, cols: int, dev_x, n_cols: int, dev_y, stream=None):
     _check(lib().prima_gemv_q4k(_dev_ptr(dev_w), rows, cols, _dev_ptr(dev_x), n_cols, _dev_ptr(dev_y), _stream_ptr(stream)))
+
+
+def prima_gemv_q4k_noalloc(dev_w, rows: int, cols: int, dev_x, n_cols: int, dev_y, stream=None):
+    """Matrix-vector product that allocates nothing (for callers that own all device memory themselves).
+
+    Same arguments as ``prima_gemv_q4k``; limited to rows*(cols/256)*n_cols <= 4,194,304; queues its
+    kernels on the stream and returns without waiting.  Calls on one device must not overlap."""
+    rc = lib().prima_gemv_q4k_noalloc(_dev_ptr(dev_w), rows, cols, _dev_ptr(dev_x), n_cols, _dev_ptr(dev_y), _stream_ptr(stream))
+    if rc != OK:
+        raise PrimaError(rc, lib().prima_gemv_q4k_noalloc_error().decode())
 
 
 class GemvPlan:
