@@ -86,6 +86,7 @@ struct prima_gemv_plan {
   TiledMat w;
   float* part = nullptr;
   VecStats stats;
+  int* status = nullptr;
 };
 
 namespace {
@@ -383,21 +384,21 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
   if (layer_begin < layer_end) LAUNCH(c, launch_rope_table(c->rope_tab, pos, n_tok, g.rope_theta, st), "rope_table");
   for (int l = layer_begin; l < layer_end; ++l) {
     Layer& L = c->layers[l];
-    GemvIn in{c->h, L.g_attn, L.gmax_attn, g.rms_eps, c->st_h};
+    GemvIn in{c->h, L.g_attn, L.gmax_attn, g.rms_eps, c->st_h, c->status};
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->part, c->sm_count, st), "gemv(qkv)");
-    LAUNCH(c, launch_finish_qkv(c->part, L.qkv.n_sb, L.qkv.mpad(), H, G, n_tok, c->rope_tab, g.rope_mode, c->qbuf, L.k, L.v,
+    LAUNCH(c, launch_finish_qkv(c->part, gemv_n_parts(L.qkv.n_sb), L.qkv.mpad(), H, G, n_tok, c->rope_tab, g.rope_mode, c->qbuf, L.k, L.v,
                                 g.kv_capacity, pos, st), "finish_qkv");
     LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos + n_tok),
              launch_attention(c->qbuf, L.k, L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, &c->st_o, st), "attention");
-    GemvIn in_o{c->obuf, nullptr, 1.f, 0.f, c->st_o};
+    GemvIn in_o{c->obuf, nullptr, 1.f, 0.f, c->st_o, c->status};
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->part, c->sm_count, st), "gemv(o)");
-    LAUNCH(c, launch_finish_residual(c->part, L.o.n_sb, L.o.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(o)");
-    GemvIn in_f{c->h, L.g_ffn, L.gmax_ffn, g.rms_eps, c->st_h};
+    LAUNCH(c, launch_finish_residual(c->part, gemv_n_parts(L.o.n_sb), L.o.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(o)");
+    GemvIn in_f{c->h, L.g_ffn, L.gmax_ffn, g.rms_eps, c->st_h, c->status};
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->part, c->sm_count, st), "gemv(gate/up)");
-    LAUNCH(c, launch_finish_swiglu(c->part, L.gu.n_sb, L.gu.mpad(), g.ffn, n_tok, c->act, &c->st_act, st), "finish_swiglu");
-    GemvIn in_d{c->act, nullptr, 1.f, 0.f, c->st_act};
+    LAUNCH(c, launch_finish_swiglu(c->part, gemv_n_parts(L.gu.n_sb), L.gu.mpad(), g.ffn, n_tok, c->act, &c->st_act, st), "finish_swiglu");
+    GemvIn in_d{c->act, nullptr, 1.f, 0.f, c->st_act, c->status};
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->part, c->sm_count, st), "gemv(down)");
-    LAUNCH(c, launch_finish_residual(c->part, L.down.n_sb, L.down.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(down)");
+    LAUNCH(c, launch_finish_residual(c->part, gemv_n_parts(L.down.n_sb), L.down.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(down)");
   }
   cudaError_t e = cudaMemcpyAsync(hidden_out, c->h, static_cast<size_t>(n_tok) * e_ * 4, cudaMemcpyDeviceToDevice, st);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(hidden_out)");
@@ -412,9 +413,9 @@ int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = c->stream;
   LAUNCH(c, launch_copy_stats(hidden, nullptr, c->cfg.hidden, n_tok, &c->st_h, st), "copy_stats");
-  GemvIn in{hidden, c->g_out, c->gmax_out, c->cfg.rms_eps, c->st_h};
+  GemvIn in{hidden, c->g_out, c->gmax_out, c->cfg.rms_eps, c->st_h, c->status};
   LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->part, c->sm_count, st), "gemv(head)");
-  LAUNCH(c, launch_finish_plain(c->part, c->head.n_sb, c->head.mpad(), c->cfg.vocab, n_tok, logits, st), "finish_plain");
+  LAUNCH(c, launch_finish_plain(c->part, gemv_n_parts(c->head.n_sb), c->head.mpad(), c->cfg.vocab, n_tok, logits, st), "finish_plain");
   return PRIMA_OK;
 }
 
@@ -576,6 +577,8 @@ int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int ma
   if (e == cudaSuccess) e = cudaMemset(p->w.data, 0, p->w.bytes());
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->part), static_cast<size_t>(p->w.n_sb) * max_n_cols * p->w.mpad() * 4);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->stats.data), sizeof(float2) * kMaxTok * kMaxStatBlocks);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->status), sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(int));
   if (e == cudaSuccess) {
     int k = launch_retile(static_cast<const uint8_t*>(dev_w), rows, p->w.n_sb, p->w, 0, 1, nullptr);
     if (k < 0) e = static_cast<cudaError_t>(-k);
@@ -594,10 +597,10 @@ int prima_gemv_plan_run(prima_gemv_plan* p, const float* dev_x, int n_cols, floa
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int k = launch_copy_stats(dev_x, nullptr, p->w.cols, n_cols, &p->stats, st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "copy_stats");
-  GemvIn in{dev_x, nullptr, 1.f, 0.f, p->stats};
+  GemvIn in{dev_x, nullptr, 1.f, 0.f, p->stats, p->status};
   k = launch_gemv_partials(p->w, in, n_cols, p->part, p->sm_count, st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "gemv kernel");
-  k = launch_finish_plain(p->part, p->w.n_sb, p->w.mpad(), p->w.rows, n_cols, dev_y, st);
+  k = launch_finish_plain(p->part, gemv_n_parts(p->w.n_sb), p->w.mpad(), p->w.rows, n_cols, dev_y, st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "finish kernel");
   return PRIMA_OK;
 }
@@ -607,6 +610,7 @@ int prima_gemv_plan_destroy(prima_gemv_plan* p) {
   cudaFree(p->w.data);
   cudaFree(p->part);
   cudaFree(p->stats.data);
+  cudaFree(p->status);
   delete p;
   return PRIMA_OK;
 }

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+
 namespace prima {
 
 // ---------------------------------------------------------------------------------------------
@@ -69,8 +71,14 @@ int launch_dequant_std(const uint8_t* blocks, int64_t n_sb, float* out, cudaStre
 int launch_retile(const uint8_t* src, int64_t rows_src, int64_t n_sb, TiledMat dst, int64_t dst_row0,
                   int64_t dst_row_stride, cudaStream_t st);
 
-// Partial products of every (row, super-block column):
-//   part[(s * n_tok + t) * mpad + r] = sum over the 256 weights of column s of W[r][k] * xhat[t][k]
+// Number of adjacent super-block columns one CTA of the GEMV works on (largest divisor of n_sb
+// that is <= 8), and the number of partial sums per row that the GEMV leaves for the finishers.
+int gemv_group_size(int64_t n_sb);
+bool gemv_uses_tensor_cores();
+inline int64_t gemv_n_parts(int64_t n_sb) { return n_sb / gemv_group_size(n_sb); }
+
+// Partial products of every (row, column group p of gemv_group_size(n_sb) super-block columns):
+//   part[(p * n_tok + t) * mpad + r] = sum over the weights of group p of W[r][k] * xhat[t][k]
 // where xhat = x * gain * rsqrt(mean(x^2) + eps) if gain != nullptr, else x.  x: [n_tok][cols].
 struct GemvIn {
   const float* x;        // [n_tok][cols] fp32
@@ -78,6 +86,7 @@ struct GemvIn {
   float gain_max;        // max |gain| (1 if gain == nullptr)
   float eps;
   VecStats stats;        // statistics of x
+  int* status;           // device word raised if a bounded wait inside the kernel gives up
 };
 int launch_gemv_partials(const TiledMat& w, const GemvIn& in, int n_tok, float* part, int sm_count,
                          cudaStream_t st);

@@ -190,9 +190,9 @@ __global__ void argmax_stage2_kernel(const float* __restrict__ val, const int32_
 }
 
 int stat_blocks_for(int64_t width) {
-  int64_t nb = (width + kBlock * 4 - 1) / (kBlock * 4);
+  int64_t nb = (width + kBlock - 1) / kBlock;
   if (nb < 1) nb = 1;
-  if (nb > 64) nb = 64;
+  if (nb > kMaxStatBlocks) nb = kMaxStatBlocks;
   return static_cast<int>(nb);
 }
 

@@ -1,117 +1,228 @@
-// Dequantise-fused Q4_K matrix-vector product, streaming formulation.
+// Dequantise-fused Q4_K matrix-vector / small-n matrix product, streaming formulation.
 //
 // Work decomposition.  The matrix is a grid of units (row tile of 8 rows  x  super-block column of
-// 256 weights, 1152 bytes each, see common.cuh) stored column-major, so unit index u = s*n_rt + rt
-// is also its position in memory.  The grid is persistent (a fixed number of CTAs per SM); the
-// U units are cut into one contiguous range per warp, so every warp streams one contiguous slice
-// of HBM, and all warps get the same number of units to within one.  A warp therefore stays at
-// one column s for (almost) its whole range and keeps that column's 256 activations in registers.
+// 256 weights, 1152 bytes each, see common.cuh) stored column-major.  The n_sb columns are taken in
+// groups of SG adjacent columns (SG = the largest divisor of n_sb that is <= 8); a CTA has SG warps,
+// warp w always works on column  group*SG + w.  The n_groups * n_rt (group, row tile) positions are
+// ordered group-major and cut into one contiguous range per CTA of a persistent grid, so all CTAs
+// get the same number of tiles to within one.  A CTA walks its range in batches of up to 4
+// consecutive row tiles of one group (a batch never crosses a group boundary), so each warp's part
+// of a batch is one contiguous piece of HBM of up to 4608 bytes, and the warp keeps its column's
+// 256 activations in registers for the whole walk.
+//
+// Data movement.  Each warp owns a ring of kRing batch slots in shared memory.  Lane 0 requests a
+// batch with one 1-D bulk asynchronous copy (TMA) that signals an mbarrier with its byte count;
+// the warp waits on the mbarrier (bounded: a wait that does not end raises the status word and the
+// kernel drains and returns), reads its three 16-byte pieces per unit with ordinary shared loads,
+// and after the batch is consumed lane 0 re-arms the slot with the next request.  Memory-level
+// parallelism is therefore set by the ring, not by registers or occupancy.
 //
 // Arithmetic.  Lane (g, t) = (lane / 4, lane % 4) owns row g of the tile and sub-blocks t and
-// 4 + t of the super-block: two 16-byte nibble chunks plus the 16-byte header of its row.
-// The activations of a sub-block are held as 16-bit integers x_q = round(x / s_j), with one fp32
-// step s_j = max|x| / 32767 per sub-block, split into a signed high byte and an unsigned low byte.
-// Nibbles are masked in place into unsigned bytes and multiplied with the 4-way byte dot product
-// (dp4a): I_j = sum q * x_q is an exact integer below 2^24, so the only rounding errors are the
-// 16-bit step of x (about 2e-5 of a typical activation) and a handful of fp32 operations per
-// sub-block:  partial = d * sum_j sc_j * s_j * I_j  -  dmin * sum_j m_j * s_j * sum(x_q).
+// 4 + t of the super-block.  The activations of a sub-block are held as 16-bit integers
+// x_q = round(x / s_j), |x_q| <= 32639, with one fp32 step s_j = max|x| / 32639 per sub-block,
+// split into two signed bytes x_q = 256 hi + lo.  Nibbles are masked in place into unsigned bytes
+// (even nibbles as q, odd nibbles as 16 q, shifted back after the sums).  I_j = sum q * x_q is an
+// exact integer below 2^24, and so are sc_j * I_j and m_j * sum(x_q) in 32 bits; the only rounding
+// errors are the 16-bit step of x (about 2e-5 of a typical activation) and a few fp32 operations
+// per sub-block:  partial = sum_j s_j * (d * sc_j * I_j  -  dmin * m_j * sum(x_q)).
+// Two interchangeable inner products compute I_j:
+//   * dp4a: 4-way byte dot products on the integer pipe (hi and lo parts separately);
+//   * mma:  the int8 tensor-core instruction m16n8k32.  Rows 0-7 / 8-15 of the A tile are two
+//           consecutive row tiles; the 32 k-slots are two 16-byte words' worth of nibbles of the four
+//           sub-blocks held by the lane quad; the 8 columns of B are (sub-block of the quad) x
+//           (hi, lo), with a lane's activation bytes in its own sub-block's columns and zeros
+//           elsewhere, so D[row][2t], D[row][2t+1] are exactly lane (row, t)'s hi and lo sums.
+//           With several tokens, one such instruction per token.
 // With RMSNorm fused, x is multiplied by the gain before quantisation and the scalar
 // rsqrt(mean(x^2) + eps) is applied to the fp32 partial.
 //
-// Output.  Each unit yields 8 row partials per token; they are written to
-//   part[(s * n_tok + t) * mpad + row]
-// and summed over s in ascending order by the finisher kernels (finish.cu), which makes the
-// result independent of how the units were split over warps.
+// Output.  A lane's four tile partials of a batch are reduced over the quad with a transposing
+// shuffle (lane t ends with tile t's row sum), the SG warps of the CTA add theirs through shared
+// memory in warp order (one barrier per batch, double-buffered), giving one partial per (column
+// group, row, token):  part[(group * n_tok + tok) * mpad + row].  The finisher kernels (finish.cu)
+// add the groups in ascending order.  No atomics: the bits do not depend on scheduling.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace prima {
-namespace {
 
-constexpr int kWarpsPerCta = 8;
-constexpr int kPipe = 4;   // units in flight per warp
-
-struct UnitRegs {
-  uint4 h, q0, q1;
-};
-
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-  uint4 v;
-  asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
+int gemv_group_size(int64_t n_sb) {
+  for (int sg = 8; sg > 1; --sg)
+    if (n_sb % sg == 0) return sg;
+  return 1;
 }
 
-// 4-way byte dot products: unsigned nibble bytes times signed / unsigned activation bytes.
-__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
+namespace {
+
+constexpr int kMaxWarps = 8;
+constexpr int kBatch = 4;                    // row tiles per batch (= lanes of a quad)
+constexpr int kBatchBytes = kBatch * kUnitBytes;
+constexpr int kRing = 3;                     // batches in flight per warp
+constexpr uint32_t kWaitLimit = 1u << 24;    // polls of one mbarrier wait before the kernel gives up
+
+// ---- asynchronous bulk copies (TMA, 1-D) into a per-warp ring, completion through mbarriers ------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitLimit polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+// ---- integer inner products -----------------------------------------------------------------------
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {   // unsigned bytes x signed bytes
   int d;
   asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-__device__ __forceinline__ uint32_t dp4a_uu(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
+
+// D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col)
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// The 32 activations of one sub-block as bytes: hi[2w + p] / lo[2w + p] hold the high / low bytes of
-// x_q for weights 8w + p, 8w + p + 2, 8w + p + 4, 8w + p + 6 (p = 0 even nibbles, 1 odd nibbles).
+// The 32 activations of one sub-block as signed bytes: hi[2w + p] / lo[2w + p] hold the high / low
+// bytes of x_q for weights 8w + p, 8w + p + 2, 8w + p + 4, 8w + p + 6 (p = 0 even nibbles, 1 odd).
 struct SubX {
   uint32_t hi[8], lo[8];
-  float step;       // s_j
-  float step_sum;   // s_j * sum(x_q)
+  float step;   // s_j
+  int sum;      // sum of x_q
 };
 
-// sum over the 32 weights of q * x_q (exact)
-__device__ __forceinline__ int chunk_dot(const uint4& q, const SubX& x) {
-  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-  int he = 0, ho = 0;
-  uint32_t le = 0, lo = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint32_t e = w[i] & 0x0f0f0f0fu, o = (w[i] >> 4) & 0x0f0f0f0fu;
-    he = dp4a_us(e, x.hi[2 * i], he);
-    ho = dp4a_us(o, x.hi[2 * i + 1], ho);
-    le = dp4a_uu(e, x.lo[2 * i], le);
-    lo = dp4a_uu(o, x.lo[2 * i + 1], lo);
+__device__ __forceinline__ float4 load_x4(const float* __restrict__ xp, const float* __restrict__ gp, int c) {
+  float4 a = *reinterpret_cast<const float4*>(xp + 4 * c);
+  if (gp) {
+    const float4 gv = *reinterpret_cast<const float4*>(gp + 4 * c);
+    a.x *= gv.x; a.y *= gv.y; a.z *= gv.z; a.w *= gv.w;
   }
-  return (he + ho) * 256 + static_cast<int>(le + lo);
+  return a;
 }
 
-// Quantise 32 consecutive activations (times gain, if any) into a SubX.
+// Quantise 32 consecutive activations (times gain, if any).  Two passes over the same 128 bytes
+// (maximum, then rounding) keep the register footprint of this rarely executed step small.
 __device__ __forceinline__ void load_sub(const float* __restrict__ xp, const float* __restrict__ gp, SubX& out) {
-  float v[32];
   float amax = 0.f;
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
-    float4 a = *reinterpret_cast<const float4*>(xp + 4 * c);
-    if (gp) {
-      const float4 gv = *reinterpret_cast<const float4*>(gp + 4 * c);
-      a.x *= gv.x; a.y *= gv.y; a.z *= gv.z; a.w *= gv.w;
-    }
-    v[4 * c] = a.x; v[4 * c + 1] = a.y; v[4 * c + 2] = a.z; v[4 * c + 3] = a.w;
+    const float4 a = load_x4(xp, gp, c);
     amax = fmaxf(amax, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
   }
   const bool ok = amax > 0.f && amax < 3.0e38f;
-  const float inv_step = ok ? 32767.0f / amax : 0.f;
+  const float inv_step = ok ? 32639.0f / amax : 0.f;
   int sum = 0;
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
+    const float4 a = load_x4(xp, gp, 2 * w), b = load_x4(xp, gp, 2 * w + 1);
+    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
 #pragma unroll
-    for (int p = 0; p < 2; ++p) {
-      uint32_t hi = 0, lo = 0;
-#pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        int xq = __float2int_rn(v[8 * w + 2 * b + p] * inv_step);
-        xq = max(-32767, min(32767, xq));
-        sum += xq;
-        hi |= (static_cast<uint32_t>(xq >> 8) & 0xffu) << (8 * b);
-        lo |= (static_cast<uint32_t>(xq) & 0xffu) << (8 * b);
-      }
-      out.hi[2 * w + p] = hi;
-      out.lo[2 * w + p] = lo;
+    for (int i = 0; i < 8; ++i) {
+      int xq = __float2int_rn(v[i] * inv_step);
+      xq = max(-32639, min(32639, xq));
+      sum += xq;
+      const int l = ((xq + 128) & 255) - 128;      // signed low byte
+      const int h = (xq - l) >> 8;                 // signed high byte, |h| <= 127
+      hi[i & 1] |= (static_cast<uint32_t>(h) & 0xffu) << (8 * (i >> 1));
+      lo[i & 1] |= (static_cast<uint32_t>(l) & 0xffu) << (8 * (i >> 1));
     }
+    out.hi[2 * w] = hi[0];
+    out.hi[2 * w + 1] = hi[1];
+    out.lo[2 * w] = lo[0];
+    out.lo[2 * w + 1] = lo[1];
   }
-  out.step = ok ? amax / 32767.0f : 0.f;
-  out.step_sum = out.step * static_cast<float>(sum);
+  out.step = ok ? amax / 32639.0f : 0.f;
+  out.sum = sum;
+}
+
+// What a lane keeps of one sub-block for the multiplications.
+//   dp4a variant: all 16 byte registers.
+//   mma variant:  the B-operand registers of the lane: its hi bytes if it sits in column 2t, its lo
+//                 bytes if in column 2t+1, zeros otherwise (8 registers), plus step and sum.
+template <bool MMA>
+struct LaneX;
+template <>
+struct LaneX<false> {
+  uint32_t hi[8], lo[8];
+  float step;
+  int sum;
+  __device__ __forceinline__ void set(const SubX& s, int, int) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      hi[i] = s.hi[i];
+      lo[i] = s.lo[i];
+    }
+    step = s.step;
+    sum = s.sum;
+  }
+};
+template <>
+struct LaneX<true> {
+  uint32_t b[8];
+  float step;
+  int sum;
+  __device__ __forceinline__ void set(const SubX& s, int g, int t) {
+    const bool mine = (g >> 1) == t;
+    const bool low = g & 1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) b[i] = mine ? (low ? s.lo[i] : s.hi[i]) : 0u;
+    step = s.step;
+    sum = s.sum;
+  }
+};
+
+// I = sum over the 32 weights of one 16-byte chunk of q * x_q, dp4a variant.
+__device__ __forceinline__ int chunk_dot(const uint4& q, const LaneX<false>& x) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  int he = 0, ho = 0, le = 0, lo = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t e = w[i] & 0x0f0f0f0fu, o = w[i] & 0xf0f0f0f0u;
+    he = dp4a_us(e, x.hi[2 * i], he);
+    ho = dp4a_us(o, x.hi[2 * i + 1], ho);
+    le = dp4a_us(e, x.lo[2 * i], le);
+    lo = dp4a_us(o, x.lo[2 * i + 1], lo);
+  }
+  return he * 256 + le + ((ho * 256 + lo) >> 4);
+}
+
+// Two row tiles (u0 -> rows 0-7, u1 -> rows 8-15) of one chunk, mma variant: the lane's I for u0, u1.
+__device__ __forceinline__ void chunk_dot2(const uint4& q_u0, const uint4& q_u1, const LaneX<true>& x, int& i_u0, int& i_u1) {
+  int ce[4] = {0, 0, 0, 0}, co[4] = {0, 0, 0, 0};
+  constexpr uint32_t E = 0x0f0f0f0fu, O = 0xf0f0f0f0u;
+  mma_u8s8(ce, q_u0.x & E, q_u1.x & E, q_u0.y & E, q_u1.y & E, x.b[0], x.b[2]);
+  mma_u8s8(co, q_u0.x & O, q_u1.x & O, q_u0.y & O, q_u1.y & O, x.b[1], x.b[3]);
+  mma_u8s8(ce, q_u0.z & E, q_u1.z & E, q_u0.w & E, q_u1.w & E, x.b[4], x.b[6]);
+  mma_u8s8(co, q_u0.z & O, q_u1.z & O, q_u0.w & O, q_u1.w & O, x.b[5], x.b[7]);
+  i_u0 = ce[0] * 256 + ce[1] + ((co[0] * 256 + co[1]) >> 4);
+  i_u1 = ce[2] * 256 + ce[3] + ((co[2] * 256 + co[3]) >> 4);
+}
+__device__ __forceinline__ void chunk_dot2(const uint4& q_u0, const uint4& q_u1, const LaneX<false>& x, int& i_u0, int& i_u1) {
+  i_u0 = chunk_dot(q_u0, x);
+  i_u1 = chunk_dot(q_u1, x);
 }
 
 // rsqrt(mean(x^2) + eps) of one token from the statistics blocks, reduced the same way in every warp.
@@ -124,33 +235,100 @@ __device__ __forceinline__ float token_inv_rms(const float2* __restrict__ stats,
   return 1.0f / sqrtf(ss / static_cast<float>(cols) + eps);
 }
 
-template <int NTOK>
-__global__ void __launch_bounds__(kWarpsPerCta * 32, (NTOK == 1 ? 2 : 1))
-gemv_partials_kernel(const uint8_t* __restrict__ w, int64_t n_rt, int64_t n_sb, int64_t cols, const float* __restrict__ x,
+// Header of one unit row -> the lane's scale factors.
+struct LaneScales {
+  float d, dmin;
+  int sc_lo, sc_hi, m_lo, m_hi;
+};
+__device__ __forceinline__ LaneScales decode_header(const uint4& h, uint32_t sel_a, uint32_t sel_b) {
+  LaneScales r;
+  const float2 df = __half22float2(*reinterpret_cast<const __half2*>(&h.x));
+  r.d = df.x;
+  r.dmin = df.y;
+  const uint32_t f = __byte_perm(__byte_perm(h.y, h.z, sel_a), h.w, sel_b);
+  r.sc_lo = f & 63u;
+  r.sc_hi = (f >> 6) & 63u;
+  r.m_lo = (f >> 12) & 63u;
+  r.m_hi = (f >> 18) & 63u;
+  return r;
+}
+__device__ __forceinline__ float unit_partial(const LaneScales& s, int i0, int i1, float step_a, int sum_a, float step_b, int sum_b) {
+  const float a0 = static_cast<float>(s.sc_lo * i0), a1 = static_cast<float>(s.sc_hi * i1);
+  const float b0 = static_cast<float>(s.m_lo * sum_a), b1 = static_cast<float>(s.m_hi * sum_b);
+  return step_a * (s.d * a0 - s.dmin * b0) + step_b * (s.d * a1 - s.dmin * b1);
+}
+
+// Walk over the (group, row tile) positions pos .. end-1 in batches of at most kBatch tiles that do
+// not cross a group boundary.
+struct Walk {
+  int pos, end, grp, rt, n_rt;
+  __device__ __forceinline__ void init(int p, int e, int n_rt_) {
+    pos = p;
+    end = e;
+    n_rt = n_rt_;
+    grp = p / n_rt_;
+    rt = p - grp * n_rt_;
+  }
+  __device__ __forceinline__ bool done() const { return pos >= end; }
+  __device__ __forceinline__ int batch() const { return min(kBatch, min(end - pos, n_rt - rt)); }
+  __device__ __forceinline__ void next(int nb) {
+    pos += nb;
+    rt += nb;
+    if (rt == n_rt) {
+      rt = 0;
+      ++grp;
+    }
+  }
+};
+
+template <int NTOK, bool MMA>
+__global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1))
+gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, const float* __restrict__ x,
                      const float* __restrict__ gain, float eps, const float2* __restrict__ stats, int n_stat_blocks, int tok0,
-                     int n_tok_total, float* __restrict__ part, int64_t mpad) {
+                     int n_tok_total, float* __restrict__ part, int64_t mpad, int* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  // layout: [warps][kRing][4608] batches, then [warps][kRing] mbarriers, then the reduction buffer
+  const int n_warps = blockDim.x >> 5;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(n_warps) * kRing * kBatchBytes);
+  float* red = reinterpret_cast<float*>(bars + n_warps * kRing);   // [2][NTOK][kMaxWarps][kBatch][8]
+
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int64_t wg = static_cast<int64_t>(blockIdx.x) * kWarpsPerCta + warp;
-  const int64_t n_warps = static_cast<int64_t>(gridDim.x) * kWarpsPerCta;
-  const int64_t n_units = n_rt * n_sb;
-  const int64_t u0 = n_units * wg / n_warps, u1 = n_units * (wg + 1) / n_warps;
-  if (u0 >= u1) return;
+  const int64_t cols = static_cast<int64_t>(n_sb) * 256;
+  const int n_pos = (n_sb / sg) * n_rt;
+  const int p0 = static_cast<int>(static_cast<int64_t>(n_pos) * blockIdx.x / gridDim.x);
+  const int p1 = static_cast<int>(static_cast<int64_t>(n_pos) * (blockIdx.x + 1) / gridDim.x);
+  if (p0 >= p1) return;
 
-  const uint8_t* lane_h = w + g * 16;
-  const uint8_t* lane_q = w + kUnitHdrBytes + lane * 16;
-
-  UnitRegs buf[kPipe];
+  const uint8_t* my_ring = smem + static_cast<size_t>(warp) * kRing * kBatchBytes;
+  const uint32_t ring_u32 = smem_addr(my_ring);
+  const uint32_t bar_u32 = smem_addr(bars + warp * kRing);
+  if (lane == 0) {
 #pragma unroll
-  for (int i = 0; i < kPipe; ++i) {
-    if (u0 + i < u1) {
-      const int64_t off = (u0 + i) * kUnitBytes;
-      buf[i].h = ldg_stream(lane_h + off);
-      buf[i].q0 = ldg_stream(lane_q + off);
-      buf[i].q1 = ldg_stream(lane_q + off + 512);
-    }
+    for (int i = 0; i < kRing; ++i) mbar_init(bar_u32 + 8 * i, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  __syncwarp();
+
+  Walk pf, cur;                 // next batch to request / batch being computed
+  pf.init(p0, p1, n_rt);
+  cur.init(p0, p1, n_rt);
+  int n_in_flight = 0;          // requested and not yet waited for
+  auto request = [&](int slot) {
+    const int nb = pf.batch();
+    if (lane == 0) {
+      const uint8_t* src = w + (static_cast<int64_t>(pf.grp * sg + warp) * n_rt + pf.rt) * kUnitBytes;
+      mbar_expect_tx(bar_u32 + 8 * slot, nb * kUnitBytes);
+      bulk_load(ring_u32 + slot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * slot);
+    }
+    pf.next(nb);
+    ++n_in_flight;
+  };
+#pragma unroll
+  for (int i = 0; i < kRing; ++i)
+    if (!pf.done()) request(i);
 
   float post[NTOK];
 #pragma unroll
@@ -160,74 +338,153 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int64_t n_rt, int64_t n_sb, 
   const uint32_t sel_a = t == 1 ? 0x7654u : (t == 3 ? 0x0073u : 0x3210u);
   const uint32_t sel_b = t == 2 ? 0x7654u : (t == 3 ? 0x0710u : 0x3210u);
 
-  SubX xa[NTOK], xb[NTOK];   // sub-blocks t and 4 + t of the current column
-  int64_t cur_s = -1;
+  LaneX<MMA> xa[NTOK], xb[NTOK];   // sub-blocks t and 4 + t of the current column
+  int cur_grp = -1;
+  int parity = 0;
+  bool alive = true;
+  int slot = 0;
+  uint32_t phase = 0;
 
-  for (int64_t ub = u0; ub < u1; ub += kPipe) {
+  while (!cur.done()) {
+    const int nb = cur.batch();
+    if (cur.grp != cur_grp) {
+      cur_grp = cur.grp;
+      const int s = cur.grp * sg + warp;
 #pragma unroll
-    for (int i = 0; i < kPipe; ++i) {
-      const int64_t u = ub + i;
-      if (u < u1) {
-        const UnitRegs r = buf[i];
-        if (u + kPipe < u1) {
-          const int64_t off = (u + kPipe) * kUnitBytes;
-          buf[i].h = ldg_stream(lane_h + off);
-          buf[i].q0 = ldg_stream(lane_q + off);
-          buf[i].q1 = ldg_stream(lane_q + off + 512);
-        }
-        const int64_t s = u / n_rt, rt = u - s * n_rt;
-        if (s != cur_s) {
-          cur_s = s;
+      for (int k = 0; k < NTOK; ++k) {
+        const float* xp = x + static_cast<int64_t>(tok0 + k) * cols + s * 256 + 32 * t;
+        const float* gp = gain ? gain + s * 256 + 32 * t : nullptr;
+        SubX tmp;
+        load_sub(xp, gp, tmp);
+        xa[k].set(tmp, g, t);
+        load_sub(xp + 128, gp ? gp + 128 : nullptr, tmp);
+        xb[k].set(tmp, g, t);
+      }
+    }
+    if (alive && !mbar_wait(bar_u32 + 8 * slot, phase)) {
+      alive = false;
+      if (lane == 0) atomicExch(status, 1);
+    }
+    --n_in_flight;
+    const uint8_t* base = my_ring + slot * kBatchBytes;
+    float acc[NTOK][kBatch];
 #pragma unroll
-          for (int k = 0; k < NTOK; ++k) {
-            const float* xp = x + static_cast<int64_t>(tok0 + k) * cols + s * 256 + 32 * t;
-            const float* gp = gain ? gain + s * 256 + 32 * t : nullptr;
-            load_sub(xp, gp, xa[k]);
-            load_sub(xp + 128, gp ? gp + 128 : nullptr, xb[k]);
-          }
-        }
-        const float d = __half2float(__ushort_as_half(static_cast<unsigned short>(r.h.x & 0xffffu)));
-        const float dmin = __half2float(__ushort_as_half(static_cast<unsigned short>(r.h.x >> 16)));
-        const uint32_t f = __byte_perm(__byte_perm(r.h.y, r.h.z, sel_a), r.h.w, sel_b);
-        const float sc_lo = static_cast<float>(f & 63u), sc_hi = static_cast<float>((f >> 6) & 63u);
-        const float m_lo = static_cast<float>((f >> 12) & 63u), m_hi = static_cast<float>((f >> 18) & 63u);
+    for (int pr = 0; pr < kBatch / 2; ++pr) {
+      const uint8_t* u0 = base + (2 * pr) * kUnitBytes;
+      const uint8_t* u1 = u0 + kUnitBytes;
+      const LaneScales s0 = decode_header(*reinterpret_cast<const uint4*>(u0 + g * 16), sel_a, sel_b);
+      const LaneScales s1 = decode_header(*reinterpret_cast<const uint4*>(u1 + g * 16), sel_a, sel_b);
+      const uint4 qa0 = *reinterpret_cast<const uint4*>(u0 + kUnitHdrBytes + lane * 16);
+      const uint4 qa1 = *reinterpret_cast<const uint4*>(u1 + kUnitHdrBytes + lane * 16);
+      const uint4 qb0 = *reinterpret_cast<const uint4*>(u0 + kUnitHdrBytes + 512 + lane * 16);
+      const uint4 qb1 = *reinterpret_cast<const uint4*>(u1 + kUnitHdrBytes + 512 + lane * 16);
 #pragma unroll
-        for (int k = 0; k < NTOK; ++k) {
-          const float i0 = static_cast<float>(chunk_dot(r.q0, xa[k]));
-          const float i1 = static_cast<float>(chunk_dot(r.q1, xb[k]));
-          const float t1 = sc_lo * (xa[k].step * i0) + sc_hi * (xb[k].step * i1);
-          const float t2 = m_lo * xa[k].step_sum + m_hi * xb[k].step_sum;
-          float acc = d * t1 - dmin * t2;
-          acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-          acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-          if (t == 0) part[(s * n_tok_total + tok0 + k) * mpad + rt * kRowsPerTile + g] = acc * post[k];
-        }
+      for (int k = 0; k < NTOK; ++k) {
+        int ia0, ia1, ib0, ib1;
+        chunk_dot2(qa0, qa1, xa[k], ia0, ia1);
+        chunk_dot2(qb0, qb1, xb[k], ib0, ib1);
+        acc[k][2 * pr] = unit_partial(s0, ia0, ib0, xa[k].step, xa[k].sum, xb[k].step, xb[k].sum);
+        acc[k][2 * pr + 1] = unit_partial(s1, ia1, ib1, xa[k].step, xa[k].sum, xb[k].step, xb[k].sum);
+      }
+    }
+    // the whole warp has consumed the slot: hand it back and request the next batch
+    __syncwarp();
+    if (alive && !pf.done()) request(slot);
+
+    // quad reduction with transposition: lane t ends with the row sum of tile t
+#pragma unroll
+    for (int k = 0; k < NTOK; ++k) {
+      const bool odd = t & 1, upper = t & 2;
+      float k0 = odd ? acc[k][1] : acc[k][0];
+      const float s0 = odd ? acc[k][0] : acc[k][1];
+      float k1 = odd ? acc[k][3] : acc[k][2];
+      const float s1 = odd ? acc[k][2] : acc[k][3];
+      k0 += __shfl_xor_sync(0xffffffffu, s0, 1);
+      k1 += __shfl_xor_sync(0xffffffffu, s1, 1);
+      float kk = upper ? k1 : k0;
+      const float ss = upper ? k0 : k1;
+      kk += __shfl_xor_sync(0xffffffffu, ss, 2);
+      red[(((parity * NTOK + k) * kMaxWarps + warp) * kBatch + t) * kRowsPerTile + g] = kk;
+    }
+    __syncthreads();
+    // warp-ordered sum of the SG warps' partials: one thread per (token, tile of the batch, row)
+    for (int idx = threadIdx.x; idx < NTOK * kBatch * kRowsPerTile; idx += blockDim.x) {
+      const int k = idx / (kBatch * kRowsPerTile);
+      const int i = (idx / kRowsPerTile) % kBatch;
+      const int row = idx % kRowsPerTile;
+      if (i < nb) {
+        const float* src = red + ((parity * NTOK + k) * kMaxWarps * kBatch + i) * kRowsPerTile + row;
+        float sum = src[0];
+        for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile];
+        part[(static_cast<int64_t>(cur.grp) * n_tok_total + tok0 + k) * mpad + (cur.rt + i) * kRowsPerTile + row] = sum * post[k];
+      }
+    }
+    parity ^= 1;
+    if (++slot == kRing) {
+      slot = 0;
+      phase ^= 1u;
+    }
+    cur.next(nb);
+  }
+  // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
+  // outstanding slot one more bounded wait before the memory is released.
+  if (!alive) {
+    for (int i = 0; i < n_in_flight && i < kRing; ++i) {
+      mbar_wait(bar_u32 + 8 * slot, phase);
+      if (++slot == kRing) {
+        slot = 0;
+        phase ^= 1u;
       }
     }
   }
 }
 
+size_t gemv_smem_bytes(int sg, int n_tok) {
+  return static_cast<size_t>(sg) * kRing * kBatchBytes + static_cast<size_t>(sg) * kRing * 8 +
+         static_cast<size_t>(2) * n_tok * kMaxWarps * kBatch * kRowsPerTile * sizeof(float);
+}
+
+template <int NTOK, bool MMA>
+cudaError_t launch_one(const TiledMat& w, const GemvIn& in, int sg, int64_t grid, int tok, int n_tok, float* part, cudaStream_t st) {
+  auto kern = gemv_partials_kernel<NTOK, MMA>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_smem_bytes(kMaxWarps, NTOK)));
+  if (e != cudaSuccess) return e;
+  kern<<<static_cast<unsigned>(grid), sg * 32, gemv_smem_bytes(sg, NTOK), st>>>(
+      w.data, static_cast<int>(w.n_rt), static_cast<int>(w.n_sb), sg, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok,
+      n_tok, part, w.mpad(), in.status);
+  return cudaGetLastError();
+}
+
 }  // namespace
+
+// Which inner product the GEMV uses.  Environment variable PRIMA_GEMV_KERNEL = "dp4a" or "mma"
+// (read once per process); default below.
+bool gemv_uses_tensor_cores() {
+  static const bool mma = [] {
+    const char* v = getenv("PRIMA_GEMV_KERNEL");
+    if (v && v[0] == 'd') return false;
+    if (v && v[0] == 'm') return true;
+    return true;
+  }();
+  return mma;
+}
 
 int launch_gemv_partials(const TiledMat& w, const GemvIn& in, int n_tok, float* part, int sm_count, cudaStream_t st) {
   if (w.n_rt == 0 || w.n_sb == 0) return 0;
-  const int64_t n_units = w.n_rt * w.n_sb;
+  if (w.n_rt * w.n_sb >= (int64_t(1) << 31)) return cuda_rc(cudaErrorInvalidValue);
+  const int sg = gemv_group_size(w.n_sb);
+  const int64_t n_pos = (w.n_sb / sg) * w.n_rt;
   int launches = 0;
-  const int block = kWarpsPerCta * 32;
   int tok = 0;
   while (tok < n_tok) {
     const int chunk = (n_tok - tok >= 2) ? 2 : 1;
-    const int ctas_per_sm = chunk == 1 ? 2 : 1;
-    int64_t grid = static_cast<int64_t>(sm_count) * ctas_per_sm;
-    const int64_t max_useful = (n_units + kWarpsPerCta - 1) / kWarpsPerCta;
-    if (grid > max_useful) grid = max_useful;
-    if (chunk == 1)
-      gemv_partials_kernel<1><<<static_cast<unsigned>(grid), block, 0, st>>>(
-          w.data, w.n_rt, w.n_sb, w.cols, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok, n_tok, part, w.mpad());
-    else
-      gemv_partials_kernel<2><<<static_cast<unsigned>(grid), block, 0, st>>>(
-          w.data, w.n_rt, w.n_sb, w.cols, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok, n_tok, part, w.mpad());
-    cudaError_t e = cudaGetLastError();
+    const int warps_per_sm = chunk == 1 ? 16 : 8;
+    int64_t grid = static_cast<int64_t>(sm_count) * std::max(1, warps_per_sm / sg);
+    if (grid > n_pos) grid = n_pos;
+    cudaError_t e;
+    const bool mma = gemv_uses_tensor_cores();
+    if (chunk == 1) e = mma ? launch_one<1, true>(w, in, sg, grid, tok, n_tok, part, st) : launch_one<1, false>(w, in, sg, grid, tok, n_tok, part, st);
+    else e = mma ? launch_one<2, true>(w, in, sg, grid, tok, n_tok, part, st) : launch_one<2, false>(w, in, sg, grid, tok, n_tok, part, st);
     if (e != cudaSuccess) return cuda_rc(e);
     ++launches;
     tok += chunk;
