@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(kThreads)
 attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_cache, const __half* __restrict__ v_cache,
                     int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks,
                     float* __restrict__ o_part, float2* __restrict__ ml_part) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int group = n_q_heads / n_kv_heads;
   const int n_q = n_tok * group;                       // query rows served by this CTA
@@ -125,6 +127,8 @@ attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_ca
 // One block of 128 threads per (token, head): merge the chunks in ascending order.
 __global__ void attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks,
                                   int n_q_heads, float* __restrict__ o, float2* __restrict__ stats) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x;            // tok * H + head
   const int d = threadIdx.x;
   const float2* ml = ml_part + static_cast<int64_t>(row) * n_chunks;
@@ -173,19 +177,13 @@ int launch_attention(const float* q, const __half* k_cache, const __half* v_cach
   const int group = n_q_heads / n_kv_heads;
   const int n_q = n_tok * group;
   const size_t smem = 2 * kChunk * kRowHalves * sizeof(__half) + static_cast<size_t>(n_q) * (kHeadDim + kChunk) * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-    if (e != cudaSuccess) return cuda_rc(e);
-    attr_set = true;
-  }
-  dim3 grid(n_chunks, n_kv_heads);
-  attn_partial_kernel<<<grid, kThreads, smem, st>>>(q, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok,
-                                                    n_chunks, scr.o_part, scr.ml_part);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
   if (e != cudaSuccess) return cuda_rc(e);
-  attn_merge_kernel<<<n_tok * n_q_heads, kHeadDim, 0, st>>>(scr.o_part, scr.ml_part, n_chunks, n_q_heads, o, stats->data);
-  e = cudaGetLastError();
+  dim3 grid(n_chunks, n_kv_heads);
+  e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), smem, st, q, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok,
+                                                    n_chunks, scr.o_part, scr.ml_part);
+  if (e != cudaSuccess) return cuda_rc(e);
+  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), 0, st, scr.o_part, scr.ml_part, n_chunks, n_q_heads, o, stats->data);
   if (e != cudaSuccess) return cuda_rc(e);
   stats->n_blocks = n_q_heads;
   return 2;

@@ -136,4 +136,30 @@ constexpr int kArgmaxBlocks = 128;
 
 inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? 0 : -static_cast<int>(e); }
 
+// ---- programmatic dependent launch -------------------------------------------------------------
+// Every kernel of the forward pass is launched with programmatic stream serialisation: it may
+// start while its predecessor in the stream is still running.  A kernel calls pdl_trigger() first
+// thing (its successor may then be scheduled as soon as resources free up) and pdl_wait() before
+// it reads anything a predecessor wrote or writes anything a predecessor may still read; what it
+// does before pdl_wait() (set-up, prefetching immutable weights) overlaps the predecessor's tail.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 }  // namespace prima

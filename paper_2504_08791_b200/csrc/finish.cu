@@ -41,6 +41,8 @@ __device__ __forceinline__ float column_sum(const float* __restrict__ part, int6
 
 __global__ void finish_plain_kernel(const float* __restrict__ part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok,
                                     float* __restrict__ y) {
+  pdl_trigger();
+  pdl_wait();
   const int tok = blockIdx.y;
   const int64_t stride = static_cast<int64_t>(n_tok) * mpad;
   for (int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; r < rows; r += static_cast<int64_t>(gridDim.x) * kBlock)
@@ -49,6 +51,8 @@ __global__ void finish_plain_kernel(const float* __restrict__ part, int64_t n_sb
 
 __global__ void finish_residual_kernel(const float* __restrict__ part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok,
                                        float* __restrict__ h, float2* __restrict__ stats) {
+  pdl_trigger();
+  pdl_wait();
   const int tok = blockIdx.y;
   const int64_t stride = static_cast<int64_t>(n_tok) * mpad;
   float ss = 0.f, am = 0.f;
@@ -63,6 +67,8 @@ __global__ void finish_residual_kernel(const float* __restrict__ part, int64_t n
 
 __global__ void finish_swiglu_kernel(const float* __restrict__ part, int64_t n_sb, int64_t mpad, int64_t ffn, int n_tok,
                                      float* __restrict__ act, float2* __restrict__ stats) {
+  pdl_trigger();
+  pdl_wait();
   const int tok = blockIdx.y;
   const int64_t stride = static_cast<int64_t>(n_tok) * mpad;
   float ss = 0.f, am = 0.f;
@@ -86,6 +92,8 @@ __global__ void finish_swiglu_kernel(const float* __restrict__ part, int64_t n_s
 __global__ void finish_qkv_kernel(const float* __restrict__ part, int64_t n_sb, int64_t mpad, int n_q_heads, int n_kv_heads,
                                   int n_tok, const float2* __restrict__ rope_tab, int rope_mode, float* __restrict__ q_out,
                                   __half* __restrict__ k_cache, __half* __restrict__ v_cache, int kv_capacity, int pos) {
+  pdl_trigger();
+  pdl_wait();
   const int head = blockIdx.x, tok = blockIdx.y, i = threadIdx.x;
   const int64_t stride = static_cast<int64_t>(n_tok) * mpad;
   const int a = rope_mode == 0 ? i : 2 * i;
@@ -115,6 +123,8 @@ __global__ void finish_qkv_kernel(const float* __restrict__ part, int64_t n_sb, 
 
 __global__ void copy_stats_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t width,
                                   float2* __restrict__ stats) {
+  pdl_trigger();
+  pdl_wait();
   const int tok = blockIdx.y;
   float ss = 0.f, am = 0.f;
   for (int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; r < width; r += static_cast<int64_t>(gridDim.x) * kBlock) {
@@ -127,6 +137,8 @@ __global__ void copy_stats_kernel(const float* __restrict__ src, float* __restri
 }
 
 __global__ void rope_table_kernel(float2* __restrict__ tab, int pos, int n_tok, double theta) {
+  pdl_trigger();
+  pdl_wait();
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_tok * (kHeadDim / 2)) return;
   const int tok = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
@@ -168,6 +180,8 @@ __device__ __forceinline__ void block_argmax(float v, int i, float* out_v, int32
 
 __global__ void argmax_stage1_kernel(const float* __restrict__ logits, int64_t vocab, float* __restrict__ val,
                                      int32_t* __restrict__ idx) {
+  pdl_trigger();
+  pdl_wait();
   const int tok = blockIdx.y;
   float v = -INFINITY;
   int i = 0x7fffffff;
@@ -178,6 +192,8 @@ __global__ void argmax_stage1_kernel(const float* __restrict__ logits, int64_t v
 
 __global__ void argmax_stage2_kernel(const float* __restrict__ val, const int32_t* __restrict__ idx, int n_blocks,
                                      int32_t* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   const int tok = blockIdx.x;
   float v = -INFINITY;
   int i = 0x7fffffff;
@@ -205,7 +221,7 @@ inline int done(int launches) {
 
 int launch_finish_plain(const float* part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok, float* y, cudaStream_t st) {
   dim3 grid(static_cast<unsigned>((rows + kBlock - 1) / kBlock > 1024 ? 1024 : (rows + kBlock - 1) / kBlock), n_tok);
-  finish_plain_kernel<<<grid, kBlock, 0, st>>>(part, n_sb, mpad, rows, n_tok, y);
+  launch_pdl(finish_plain_kernel, dim3(grid), dim3(kBlock), 0, st, part, n_sb, mpad, rows, n_tok, y);
   return done(1);
 }
 
@@ -213,7 +229,7 @@ int launch_finish_residual(const float* part, int64_t n_sb, int64_t mpad, int64_
                            cudaStream_t st) {
   const int nb = stat_blocks_for(rows);
   dim3 grid(nb, n_tok);
-  finish_residual_kernel<<<grid, kBlock, 0, st>>>(part, n_sb, mpad, rows, n_tok, h, stats->data);
+  launch_pdl(finish_residual_kernel, dim3(grid), dim3(kBlock), 0, st, part, n_sb, mpad, rows, n_tok, h, stats->data);
   stats->n_blocks = nb;
   return done(1);
 }
@@ -222,7 +238,7 @@ int launch_finish_swiglu(const float* part, int64_t n_sb, int64_t mpad, int64_t 
                          cudaStream_t st) {
   const int nb = stat_blocks_for(ffn);
   dim3 grid(nb, n_tok);
-  finish_swiglu_kernel<<<grid, kBlock, 0, st>>>(part, n_sb, mpad, ffn, n_tok, act, stats->data);
+  launch_pdl(finish_swiglu_kernel, dim3(grid), dim3(kBlock), 0, st, part, n_sb, mpad, ffn, n_tok, act, stats->data);
   stats->n_blocks = nb;
   return done(1);
 }
@@ -231,7 +247,7 @@ int launch_finish_qkv(const float* part, int64_t n_sb, int64_t mpad, int n_q_hea
                       const float2* rope_tab, int rope_mode, float* q_out, __half* k_cache, __half* v_cache, int kv_capacity,
                       int pos, cudaStream_t st) {
   dim3 grid(n_q_heads + 2 * n_kv_heads, n_tok);
-  finish_qkv_kernel<<<grid, kHeadDim / 2, 0, st>>>(part, n_sb, mpad, n_q_heads, n_kv_heads, n_tok, rope_tab, rope_mode, q_out,
+  launch_pdl(finish_qkv_kernel, dim3(grid), dim3(kHeadDim / 2), 0, st, part, n_sb, mpad, n_q_heads, n_kv_heads, n_tok, rope_tab, rope_mode, q_out,
                                                    k_cache, v_cache, kv_capacity, pos);
   return done(1);
 }
@@ -239,14 +255,14 @@ int launch_finish_qkv(const float* part, int64_t n_sb, int64_t mpad, int n_q_hea
 int launch_copy_stats(const float* src, float* dst, int64_t width, int n_tok, VecStats* stats, cudaStream_t st) {
   const int nb = stat_blocks_for(width);
   dim3 grid(nb, n_tok);
-  copy_stats_kernel<<<grid, kBlock, 0, st>>>(src, dst, width, stats->data);
+  launch_pdl(copy_stats_kernel, dim3(grid), dim3(kBlock), 0, st, src, dst, width, stats->data);
   stats->n_blocks = nb;
   return done(1);
 }
 
 int launch_rope_table(float2* tab, int pos, int n_tok, float theta, cudaStream_t st) {
   const int n = n_tok * (kHeadDim / 2);
-  rope_table_kernel<<<(n + 127) / 128, 128, 0, st>>>(tab, pos, n_tok, static_cast<double>(theta));
+  launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, tab, pos, n_tok, static_cast<double>(theta));
   return done(1);
 }
 
@@ -255,8 +271,8 @@ int launch_argmax(const float* logits, int64_t vocab, int n_tok, float* scratch_
   int nb = static_cast<int>((vocab + kBlock - 1) / kBlock);
   if (nb > kArgmaxBlocks) nb = kArgmaxBlocks;
   dim3 grid(nb, n_tok);
-  argmax_stage1_kernel<<<grid, kBlock, 0, st>>>(logits, vocab, scratch_val, scratch_idx);
-  argmax_stage2_kernel<<<n_tok, kBlock, 0, st>>>(scratch_val, scratch_idx, nb, dev_out);
+  launch_pdl(argmax_stage1_kernel, dim3(grid), dim3(kBlock), 0, st, logits, vocab, scratch_val, scratch_idx);
+  launch_pdl(argmax_stage2_kernel, dim3(n_tok), dim3(kBlock), 0, st, scratch_val, scratch_idx, nb, dev_out);
   return done(2);
 }
 

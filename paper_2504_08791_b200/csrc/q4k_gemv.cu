@@ -286,6 +286,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1))
 gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, const float* __restrict__ x,
                      const float* __restrict__ gain, float eps, const float2* __restrict__ stats, int n_stat_blocks, int tok0,
                      int n_tok_total, float* __restrict__ part, int64_t mpad, int* __restrict__ status) {
+  pdl_trigger();
   extern __shared__ __align__(128) uint8_t smem[];
   // layout: [warps][kRing][4608] batches, then [warps][kRing] mbarriers, then the reduction buffer
   const int n_warps = blockDim.x >> 5;
@@ -329,6 +330,9 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
 #pragma unroll
   for (int i = 0; i < kRing; ++i)
     if (!pf.done()) request(i);
+
+  // the first weight batches are on their way; everything below depends on the predecessor kernel
+  pdl_wait();
 
   float post[NTOK];
 #pragma unroll
@@ -449,10 +453,9 @@ cudaError_t launch_one(const TiledMat& w, const GemvIn& in, int sg, int64_t grid
   auto kern = gemv_partials_kernel<NTOK, MMA>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_smem_bytes(kMaxWarps, NTOK)));
   if (e != cudaSuccess) return e;
-  kern<<<static_cast<unsigned>(grid), sg * 32, gemv_smem_bytes(sg, NTOK), st>>>(
-      w.data, static_cast<int>(w.n_rt), static_cast<int>(w.n_sb), sg, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok,
-      n_tok, part, w.mpad(), in.status);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(static_cast<unsigned>(grid)), dim3(sg * 32), gemv_smem_bytes(sg, NTOK), st, w.data, static_cast<int>(w.n_rt),
+                    static_cast<int>(w.n_sb), sg, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok, n_tok, part, w.mpad(),
+                    in.status);
 }
 
 }  // namespace
