@@ -1,148 +1,236 @@
 // Grouped-query decode attention over the fp16 KV cache, split along the context.
 //
-// One CTA per (context chunk of 64 positions, KV head).  The CTA stages its 64 keys and 64 values
-// (256 bytes each) in shared memory once and serves all query rows that share the KV head: the
-// H/G query heads of every token of the step.  It produces, per query row, the chunk's running
-// maximum m, the sum l of exp(s - m), and the un-normalised output sum exp(s - m) V.  A second
-// kernel merges the chunks of a row in ascending order: M = max m_c,
-// o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c.  Token t of the step attends positions
-// 0 .. pos + t (causal inside the step); positions beyond that get weight zero.
+// One CTA of 4 warps per (context chunk of 64 positions, KV head); each warp owns 16 positions.
+// The query rows that share the KV head -- the H/G heads of every token of the step, at most 64
+// rows -- are processed 16 at a time (one m16n8k16 tile of rows).  Per tile a warp computes
+//   S = Q K^T   with  A = Q (16 rows x 16 dims, fp16, pre-scaled by 1/sqrt(128)),  B = K,
+//   P = exp(S - max),   O = P V   with  A = P (fp16),  B = V,
+// all with fp32 accumulation on the tensor cores.  K and V go from global memory straight into
+// the B-operand registers with fully used 16-byte loads: the instruction's k index is only a
+// label, so each lane is given the head dimensions (for K) or positions (for V) that make its
+// bytes contiguous in the cache, and Q / P are arranged to match.  The four warps' (max, sum, O)
+// are combined through shared memory, giving per query row and chunk the running maximum m, the
+// sum l of exp(s - m) and the un-normalised output.  A second kernel merges the chunks of a row in
+// ascending order:  M = max m_c,  o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c.
+// Token t of the step attends positions 0 .. pos + t (causal inside the step).
 #include "common.cuh"
 
 namespace prima {
 namespace {
 
 constexpr int kChunk = 64;
-constexpr int kThreads = 256;
-constexpr int kRowHalves = kHeadDim + 8;   // padded row: conflict-free 16-byte reads down a column of rows
+constexpr int kWarps = 4;
+constexpr int kThreads = kWarps * 32;
 
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_h2(float a, float b) {
+  const __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Lane (g, t) = (lane / 4, lane % 4).
+//  * S tile: instruction column n = g is position (block base + g); the lane's k slots of step ks are
+//    head dims  32 (ks / 2) + 8 t + 4 (ks % 2) + {0, 1}  (first register) and  + {2, 3}  (second).
+//  * O tile: instruction d of 16 has column n = g at head dim  64 (d / 8) + 8 g + (d % 8); the lane's
+//    k slots are the positions  2t, 2t+1, 2t+8, 2t+9  of the warp's 16.
 __global__ void __launch_bounds__(kThreads)
 attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_cache, const __half* __restrict__ v_cache,
                     int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks,
                     float* __restrict__ o_part, float2* __restrict__ ml_part) {
   pdl_trigger();
-  pdl_wait();
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ float s_o[kWarps][16][kHeadDim];
+  __shared__ float s_m[kWarps][16], s_l[kWarps][16];
+
   const int group = n_q_heads / n_kv_heads;
-  const int n_q = n_tok * group;                       // query rows served by this CTA
-  __half* ks = reinterpret_cast<__half*>(smem_raw);    // [64][136]
-  __half* vs = ks + kChunk * kRowHalves;               // [64][136]
-  float* qs = reinterpret_cast<float*>(vs + kChunk * kRowHalves);  // [n_q][128]
-  float* sc = qs + n_q * kHeadDim;                     // [n_q][64]
-
-  const int chunk = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
-  const int c0 = chunk * kChunk;
+  const int n_rows = n_tok * group;                  // query rows served by this CTA
+  const int chunk = blockIdx.x, kv = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
   const int n_ctx = pos + n_tok;
-  const int valid = min(kChunk, n_ctx - c0);
+  const int wbase = chunk * kChunk + warp * 16;      // first position of this warp
 
-  for (int idx = tid; idx < n_q * kHeadDim; idx += kThreads) {
-    const int qi = idx >> 7, d = idx & 127;
-    const int tok = qi / group, head = g * group + qi % group;
-    qs[idx] = q[(static_cast<int64_t>(tok) * n_q_heads + head) * kHeadDim + d];
+  // ---- K and V of the warp's 16 positions (independent of the predecessor only for old positions;
+  //      the newest entries were written by the previous kernel, so wait first)
+  pdl_wait();
+  uint4 kreg[2][4];      // [position block of 8][32-dim slice]
+  uint4 vreg[4][2];      // [k-slot position][64-dim half]
+  const __half* kbase = k_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
+  const __half* vbase = v_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
+#pragma unroll
+  for (int pb = 0; pb < 2; ++pb) {
+    const int p = wbase + 8 * pb + g;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      kreg[pb][j] = p < n_ctx ? *reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t) : make_uint4(0, 0, 0, 0);
   }
-  for (int idx = tid; idx < kChunk * 16; idx += kThreads) {
-    const int row = idx >> 4, col = idx & 15;
-    uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-    if (row < valid) {
-      const int64_t off = (static_cast<int64_t>(g) * kv_capacity + c0 + row) * kHeadDim + col * 8;
-      kv = *reinterpret_cast<const uint4*>(k_cache + off);
-      vv = *reinterpret_cast<const uint4*>(v_cache + off);
-    }
-    *reinterpret_cast<uint4*>(ks + row * kRowHalves + col * 8) = kv;
-    *reinterpret_cast<uint4*>(vs + row * kRowHalves + col * 8) = vv;
+#pragma unroll
+  for (int pi = 0; pi < 4; ++pi) {
+    const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf)
+      vreg[pi][hf] = p < n_ctx ? *reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g) : make_uint4(0, 0, 0, 0);
   }
-  __syncthreads();
 
-  // scores
   const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
-  for (int idx = tid; idx < n_q * kChunk; idx += kThreads) {
-    const int qi = idx >> 6, j = idx & 63;
-    const int tok = qi / group;
-    float s = -INFINITY;
-    if (j < valid && c0 + j <= pos + tok) {
-      const __half* kr = ks + j * kRowHalves;
-      const float* qr = qs + qi * kHeadDim;
-      float acc = 0.f;
+  for (int tile = 0; tile * 16 < n_rows; ++tile) {
+    // ---- Q fragments of rows (tile*16 + g) and (+ 8)
+    uint32_t qa[8][4];
+    int row_tok[2];
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const uint4 kv = *reinterpret_cast<const uint4*>(kr + c * 8);
-        const float4 q0 = *reinterpret_cast<const float4*>(qr + c * 8);
-        const float4 q1 = *reinterpret_cast<const float4*>(qr + c * 8 + 4);
-        const float2 k0 = __half22float2(*reinterpret_cast<const __half2*>(&kv.x));
-        const float2 k1 = __half22float2(*reinterpret_cast<const __half2*>(&kv.y));
-        const float2 k2 = __half22float2(*reinterpret_cast<const __half2*>(&kv.z));
-        const float2 k3 = __half22float2(*reinterpret_cast<const __half2*>(&kv.w));
-        acc = fmaf(q0.x, k0.x, acc); acc = fmaf(q0.y, k0.y, acc);
-        acc = fmaf(q0.z, k1.x, acc); acc = fmaf(q0.w, k1.y, acc);
-        acc = fmaf(q1.x, k2.x, acc); acc = fmaf(q1.y, k2.y, acc);
-        acc = fmaf(q1.z, k3.x, acc); acc = fmaf(q1.w, k3.y, acc);
+    for (int hr = 0; hr < 2; ++hr) {
+      const int r = tile * 16 + g + 8 * hr;
+      const bool live = r < n_rows;
+      const int tok = live ? r / group : 0, head = kv * group + (live ? r % group : 0);
+      row_tok[hr] = live ? tok : -1;
+      const float* qr = q + (static_cast<int64_t>(tok) * n_q_heads + head) * kHeadDim;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (live) {
+          a = *reinterpret_cast<const float4*>(qr + 32 * j + 8 * t);
+          b = *reinterpret_cast<const float4*>(qr + 32 * j + 8 * t + 4);
+        }
+        qa[2 * j][hr] = pack_h2(a.x * scale, a.y * scale);
+        qa[2 * j][2 + hr] = pack_h2(a.z * scale, a.w * scale);
+        qa[2 * j + 1][hr] = pack_h2(b.x * scale, b.y * scale);
+        qa[2 * j + 1][2 + hr] = pack_h2(b.z * scale, b.w * scale);
       }
-      s = acc * scale;
     }
-    sc[idx] = s;
-  }
-  __syncthreads();
-
-  // per-row maximum, exponentials and their sum: one warp per query row
-  const int warp = tid >> 5, lane = tid & 31;
-  for (int qi = warp; qi < n_q; qi += kThreads / 32) {
-    const float s0 = sc[qi * kChunk + lane], s1 = sc[qi * kChunk + lane + 32];
-    float m = fmaxf(s0, s1);
+    // ---- scores of the 16 positions: two blocks of 8
+    float sc[2][4];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float p0 = 0.f, p1 = 0.f;
-    if (m > -INFINITY) {
-      p0 = expf(s0 - m);
-      p1 = expf(s1 - m);
-    }
-    float l = p0 + p1;
+    for (int pb = 0; pb < 2; ++pb) {
+      sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    sc[qi * kChunk + lane] = p0;
-    sc[qi * kChunk + lane + 32] = p1;
-    if (lane == 0) {
-      const int tok = qi / group, head = g * group + qi % group;
-      ml_part[(static_cast<int64_t>(tok) * n_q_heads + head) * n_chunks + chunk] = make_float2(m, l);
+      for (int j = 0; j < 4; ++j) {
+        mma_f16(sc[pb], qa[2 * j][0], qa[2 * j][1], qa[2 * j][2], qa[2 * j][3], kreg[pb][j].x, kreg[pb][j].y);
+        mma_f16(sc[pb], qa[2 * j + 1][0], qa[2 * j + 1][1], qa[2 * j + 1][2], qa[2 * j + 1][3], kreg[pb][j].z, kreg[pb][j].w);
+      }
     }
-  }
-  __syncthreads();
-
-  // weighted values: each thread owns two adjacent output lanes of one query row at a time
-  for (int idx = tid; idx < n_q * (kHeadDim / 2); idx += kThreads) {
-    const int qi = idx >> 6, d = (idx & 63) * 2;
-    const float* pr = sc + qi * kChunk;
-    float ax = 0.f, ay = 0.f;
-    for (int j = 0; j < valid; ++j) {
-      const float2 v = __half22float2(*reinterpret_cast<const __half2*>(vs + j * kRowHalves + d));
-      const float p = pr[j];
-      ax = fmaf(p, v.x, ax);
-      ay = fmaf(p, v.y, ay);
+    // ---- mask, row maxima, exponentials
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int hr = e >> 1;
+        const int p = wbase + 8 * pb + 2 * t + (e & 1);
+        const bool ok = row_tok[hr] >= 0 && p <= pos + row_tok[hr];
+        sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
+        mx[hr] = fmaxf(mx[hr], sc[pb][e]);
+      }
+    float lsum[2];
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+      mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
+      mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
+      lsum[hr] = 0.f;
     }
-    const int tok = qi / group, head = g * group + qi % group;
-    float* dst = o_part + ((static_cast<int64_t>(tok) * n_q_heads + head) * n_chunks + chunk) * kHeadDim + d;
-    *reinterpret_cast<float2*>(dst) = make_float2(ax, ay);
+    uint32_t pa[4];
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) {
+      float pv[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int hr = e >> 1;
+        pv[e] = mx[hr] > -INFINITY ? expf(sc[pb][e] - mx[hr]) : 0.f;
+        lsum[hr] += pv[e];
+      }
+      pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g,   k slots of this block
+      pa[2 * pb + 1] = pack_h2(pv[2], pv[3]);    // row g+8
+    }
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+      lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 1);
+      lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 2);
+    }
+    // ---- O = P V, 16 instructions of 8 head dims each
+#pragma unroll
+    for (int d = 0; d < 16; ++d) {
+      const int hf = d >> 3, j = (d & 7) >> 1;
+      const uint32_t sel = (d & 1) ? 0x7632u : 0x5410u;
+      const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
+      const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
+      const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
+      const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
+      const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
+      const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
+      float oc[4] = {0.f, 0.f, 0.f, 0.f};
+      mma_f16(oc, pa[0], pa[1], pa[2], pa[3], b0, b1);
+      const int dim = 64 * hf + (d & 7);
+      s_o[warp][g][dim + 16 * t] = oc[0];
+      s_o[warp][g][dim + 16 * t + 8] = oc[1];
+      s_o[warp][g + 8][dim + 16 * t] = oc[2];
+      s_o[warp][g + 8][dim + 16 * t + 8] = oc[3];
+    }
+    if (t == 0) {
+      s_m[warp][g] = mx[0];
+      s_m[warp][g + 8] = mx[1];
+      s_l[warp][g] = lsum[0];
+      s_l[warp][g + 8] = lsum[1];
+    }
+    __syncthreads();
+    // ---- combine the four warps: thread d of 128 owns head dim d of every row of the tile
+    {
+      const int d = threadIdx.x;
+      for (int r = 0; r < 16 && tile * 16 + r < n_rows; ++r) {
+        float big = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) big = fmaxf(big, s_m[w][r]);
+        float l = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+          const float f = s_m[w][r] > -INFINITY ? expf(s_m[w][r] - big) : 0.f;
+          l += f * s_l[w][r];
+          acc += f * s_o[w][r][d];
+        }
+        const int rr = tile * 16 + r;
+        const int tok = rr / group, head = kv * group + rr % group;
+        const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * n_chunks + chunk;
+        o_part[slot * kHeadDim + d] = acc;
+        if (d == 0) ml_part[slot] = make_float2(big, l);
+      }
+    }
+    __syncthreads();
   }
 }
 
-// One block of 128 threads per (token, head): merge the chunks in ascending order.
-__global__ void attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks,
-                                  int n_q_heads, float* __restrict__ o, float2* __restrict__ stats) {
+// One block of 128 threads per (token, head): merge the chunks in ascending order.  The weights
+// e^(m_c - M) / L of all chunks are prepared first, in parallel; then thread d sums its head dim.
+__global__ void __launch_bounds__(kHeadDim)
+attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks, int n_q_heads,
+                  float* __restrict__ o, float2* __restrict__ stats) {
   pdl_trigger();
   pdl_wait();
+  extern __shared__ float s_w[];         // [n_chunks]
+  __shared__ float s_red[4];
   const int row = blockIdx.x;            // tok * H + head
   const int d = threadIdx.x;
   const float2* ml = ml_part + static_cast<int64_t>(row) * n_chunks;
   float big = -INFINITY;
-  for (int c = 0; c < n_chunks; ++c) big = fmaxf(big, ml[c].x);
-  float denom = 0.f, acc = 0.f;
-  for (int c = 0; c < n_chunks; ++c) {
+  for (int c = d; c < n_chunks; c += kHeadDim) big = fmaxf(big, ml[c].x);
+#pragma unroll
+  for (int of = 16; of > 0; of >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, of));
+  if ((d & 31) == 0) s_red[d >> 5] = big;
+  __syncthreads();
+  big = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+  for (int c = d; c < n_chunks; c += kHeadDim) {
     const float2 v = ml[c];
-    if (v.x > -INFINITY) {
-      const float w = expf(v.x - big);
-      denom += w * v.y;
-      acc += w * o_part[(static_cast<int64_t>(row) * n_chunks + c) * kHeadDim + d];
-    }
+    s_w[c] = v.x > -INFINITY ? expf(v.x - big) : 0.f;
   }
+  __syncthreads();
+  // every thread forms the same denominator in chunk order
+  float denom = 0.f;
+  for (int c = 0; c < n_chunks; ++c) denom += s_w[c] * ml[c].y;
+  float acc = 0.f;
+  const float* op = o_part + static_cast<int64_t>(row) * n_chunks * kHeadDim + d;
+#pragma unroll 8
+  for (int c = 0; c < n_chunks; ++c) acc += s_w[c] * op[static_cast<int64_t>(c) * kHeadDim];
   const float out = acc / denom;
   o[static_cast<int64_t>(row) * kHeadDim + d] = out;
 
@@ -174,16 +262,12 @@ int launch_attention(const float* q, const __half* k_cache, const __half* v_cach
   const int n_ctx = pos + n_tok;
   const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
   if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
-  const int group = n_q_heads / n_kv_heads;
-  const int n_q = n_tok * group;
-  const size_t smem = 2 * kChunk * kRowHalves * sizeof(__half) + static_cast<size_t>(n_q) * (kHeadDim + kChunk) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-  if (e != cudaSuccess) return cuda_rc(e);
   dim3 grid(n_chunks, n_kv_heads);
-  e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), smem, st, q, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok,
-                                                    n_chunks, scr.o_part, scr.ml_part);
+  cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), 0, st, q, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok,
+                             n_chunks, scr.o_part, scr.ml_part);
   if (e != cudaSuccess) return cuda_rc(e);
-  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), 0, st, scr.o_part, scr.ml_part, n_chunks, n_q_heads, o, stats->data);
+  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(n_chunks) * sizeof(float), st, scr.o_part,
+                 scr.ml_part, n_chunks, n_q_heads, o, stats->data);
   if (e != cudaSuccess) return cuda_rc(e);
   stats->n_blocks = n_q_heads;
   return 2;
