@@ -54,9 +54,11 @@ attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_ca
   const int n_ctx = pos + n_tok;
   const int wbase = chunk * kChunk + warp * 16;      // first position of this warp
 
-  // ---- K and V of the warp's 16 positions (independent of the predecessor only for old positions;
-  //      the newest entries were written by the previous kernel, so wait first)
-  pdl_wait();
+  // ---- K and V of the warp's 16 positions.  Entries below `pos` were written by earlier steps and do
+  //      not change, so a warp whose positions are all old loads them before waiting for the
+  //      predecessor kernel (which writes the newest entries and the queries).
+  const bool old_only = wbase + 16 <= pos;
+  if (!old_only) pdl_wait();
   uint4 kreg[2][4];      // [position block of 8][32-dim slice]
   uint4 vreg[4][2];      // [k-slot position][64-dim half]
   const __half* kbase = k_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
@@ -75,6 +77,8 @@ attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_ca
     for (int hf = 0; hf < 2; ++hf)
       vreg[pi][hf] = p < n_ctx ? *reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g) : make_uint4(0, 0, 0, 0);
   }
+
+  if (old_only) pdl_wait();
 
   const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
   for (int tile = 0; tile * 16 < n_rows; ++tile) {

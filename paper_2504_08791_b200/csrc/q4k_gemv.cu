@@ -297,9 +297,23 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
   const int warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int64_t cols = static_cast<int64_t>(n_sb) * 256;
-  const int n_pos = (n_sb / sg) * n_rt;
-  const int p0 = static_cast<int>(static_cast<int64_t>(n_pos) * blockIdx.x / gridDim.x);
-  const int p1 = static_cast<int>(static_cast<int64_t>(n_pos) * (blockIdx.x + 1) / gridDim.x);
+  // This CTA's range of (group, row tile) positions.  When the grid has at least one CTA per column
+  // group, every group gets the same number of CTAs and a range never crosses a group boundary (a
+  // crossing costs a second activation load in mid-stream, which only that CTA pays and everybody
+  // waits for); otherwise the positions are cut evenly.
+  const int n_groups = n_sb / sg;
+  const int n_pos = n_groups * n_rt;
+  int p0, p1;
+  const int per_group = gridDim.x / n_groups;
+  if (per_group >= 1) {
+    const int grp = blockIdx.x / per_group, i = blockIdx.x - grp * per_group;
+    if (grp >= n_groups) return;
+    p0 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * i / per_group);
+    p1 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * (i + 1) / per_group);
+  } else {
+    p0 = static_cast<int>(static_cast<int64_t>(n_pos) * blockIdx.x / gridDim.x);
+    p1 = static_cast<int>(static_cast<int64_t>(n_pos) * (blockIdx.x + 1) / gridDim.x);
+  }
   if (p0 >= p1) return;
 
   const uint8_t* my_ring = smem + static_cast<size_t>(warp) * kRing * kBatchBytes;
@@ -335,8 +349,6 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
   pdl_wait();
 
   float post[NTOK];
-#pragma unroll
-  for (int k = 0; k < NTOK; ++k) post[k] = gain ? token_inv_rms(stats, n_stat_blocks, tok0 + k, cols, eps) : 1.0f;
 
   // lane-constant byte selectors that pull this lane's 24-bit field group out of header words 1..3
   const uint32_t sel_a = t == 1 ? 0x7654u : (t == 3 ? 0x0073u : 0x3210u);
@@ -344,6 +356,7 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
 
   LaneX<MMA> xa[NTOK], xb[NTOK];   // sub-blocks t and 4 + t of the current column
   int cur_grp = -1;
+  bool first = true;
   int parity = 0;
   bool alive = true;
   int slot = 0;
@@ -363,6 +376,11 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
         xa[k].set(tmp, g, t);
         load_sub(xp + 128, gp ? gp + 128 : nullptr, tmp);
         xb[k].set(tmp, g, t);
+      }
+      if (first) {      // after the activation loads, so that the two round trips overlap
+        first = false;
+#pragma unroll
+        for (int k = 0; k < NTOK; ++k) post[k] = gain ? token_inv_rms(stats, n_stat_blocks, tok0 + k, cols, eps) : 1.0f;
       }
     }
     if (alive && !mbar_wait(bar_u32 + 8 * slot, phase)) {
