@@ -52,13 +52,12 @@ struct prima_ctx {
   uint8_t* embd = nullptr;
   bool have_out_norm = false, have_head = false, have_embd = false;
 
-  float* part = nullptr;
-  size_t part_floats = 0;
-  float* h = nullptr;
-  float* qbuf = nullptr;
+  float* part_a = nullptr;   // partial sums of the QKV, gate/up and head products
+  float* part_b = nullptr;   // partial sums of the O and down products
+  float* h_a = nullptr;      // residual stream entering a layer / leaving its feed-forward block
+  float* h_b = nullptr;      // residual stream after the attention block
   float* obuf = nullptr;
-  float* act = nullptr;
-  VecStats st_h, st_o, st_act;
+  SumSq ssq_attn, ssq_ffn, ssq_out;
   float2* rope_tab = nullptr;
   AttnScratch attn{};
   uint8_t* staging = nullptr;
@@ -85,7 +84,6 @@ struct prima_gemv_plan {
   int max_n_cols = 1;
   TiledMat w;
   float* part = nullptr;
-  VecStats stats;
   int* status = nullptr;
 };
 
@@ -237,26 +235,25 @@ int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx
   const int64_t n = g.max_n_tok;
   const int64_t e_ = g.hidden, H = g.n_q_heads, G = g.n_kv_heads, F = g.ffn;
   auto pad8 = [](int64_t r) { return (r + 7) / 8 * 8; };
-  int64_t part = 0;
-  part = std::max(part, (e_ / 256) * n * pad8((H + 2 * G) * kHeadDim));
-  part = std::max(part, (H * kHeadDim / 256) * n * pad8(e_));
-  part = std::max(part, (e_ / 256) * n * pad8(2 * F));
-  part = std::max(part, (F / 256) * n * pad8(e_));
-  part = std::max(part, (e_ / 256) * n * pad8(g.vocab));
-  c->part_floats = static_cast<size_t>(part);
+  int64_t part_a = 0, part_b = 0;
+  part_a = std::max(part_a, (e_ / 256) * n * pad8((H + 2 * G) * kHeadDim));
+  part_a = std::max(part_a, (e_ / 256) * n * pad8(2 * F));
+  part_a = std::max(part_a, (e_ / 256) * n * pad8(g.vocab));
+  part_b = std::max(part_b, (H * kHeadDim / 256) * n * pad8(e_));
+  part_b = std::max(part_b, (F / 256) * n * pad8(e_));
   c->attn.max_chunks = (g.kv_capacity + attention_chunk_len() - 1) / attention_chunk_len();
   c->staging_bytes = 256u << 20;
 
   int rc = PRIMA_OK;
   auto A = [&](int r) { if (rc == PRIMA_OK) rc = r; };
-  A(dev_alloc(c, &c->part, c->part_floats));
-  A(dev_alloc(c, &c->h, static_cast<size_t>(n * e_)));
-  A(dev_alloc(c, &c->qbuf, static_cast<size_t>(n * H * kHeadDim)));
+  A(dev_alloc(c, &c->part_a, static_cast<size_t>(part_a)));
+  A(dev_alloc(c, &c->part_b, static_cast<size_t>(part_b)));
+  A(dev_alloc(c, &c->h_a, static_cast<size_t>(n * e_)));
+  A(dev_alloc(c, &c->h_b, static_cast<size_t>(n * e_)));
   A(dev_alloc(c, &c->obuf, static_cast<size_t>(n * H * kHeadDim)));
-  A(dev_alloc(c, &c->act, static_cast<size_t>(n * F)));
-  A(dev_alloc(c, &c->st_h.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
-  A(dev_alloc(c, &c->st_o.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
-  A(dev_alloc(c, &c->st_act.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
+  A(dev_alloc(c, &c->ssq_attn.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
+  A(dev_alloc(c, &c->ssq_ffn.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
+  A(dev_alloc(c, &c->ssq_out.data, static_cast<size_t>(kMaxTok) * kMaxStatBlocks, true));
   A(dev_alloc(c, &c->rope_tab, static_cast<size_t>(kMaxTok) * (kHeadDim / 2)));
   A(dev_alloc(c, &c->attn.o_part, static_cast<size_t>(n * H) * c->attn.max_chunks * kHeadDim));
   A(dev_alloc(c, &c->attn.ml_part, static_cast<size_t>(n * H) * c->attn.max_chunks));
@@ -380,28 +377,49 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
   const int64_t e_ = g.hidden;
   const int H = g.n_q_heads, G = g.n_kv_heads;
 
-  LAUNCH(c, launch_copy_stats(hidden_in, c->h, e_, n_tok, &c->st_h, st), "copy_stats");
-  if (layer_begin < layer_end) LAUNCH(c, launch_rope_table(c->rope_tab, pos, n_tok, g.rope_theta, st), "rope_table");
+  if (layer_begin == layer_end) {
+    if (hidden_out != hidden_in) {
+      cudaError_t e = cudaMemcpyAsync(hidden_out, hidden_in, static_cast<size_t>(n_tok) * e_ * 4, cudaMemcpyDeviceToDevice, st);
+      if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(hidden_out)");
+    }
+    return PRIMA_OK;
+  }
+  LAUNCH(c, launch_rope_table(c->rope_tab, pos, n_tok, g.rope_theta, st), "rope_table");
+  const int64_t mpad_e = (e_ + 7) / 8 * 8;
+  // The residual stream entering a layer is h_in plus the still unsummed partial sums of the previous
+  // down projection (none for the first layer of the call); each product's CTAs finish what they
+  // need of their producer's output while staging their activations.
+  const float* h_in = hidden_in;
+  int n_parts_prev = 0;
   for (int l = layer_begin; l < layer_end; ++l) {
     Layer& L = c->layers[l];
-    GemvIn in{c->h, L.g_attn, L.gmax_attn, g.rms_eps, c->st_h, c->status};
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->part, c->sm_count, st), "gemv(qkv)");
-    LAUNCH(c, launch_finish_qkv(c->part, gemv_n_parts(L.qkv.n_sb), L.qkv.mpad(), H, G, n_tok, c->rope_tab, g.rope_mode, c->qbuf, L.k, L.v,
-                                g.kv_capacity, pos, st), "finish_qkv");
+    GemvIn in;                                   // QKV: residual (+ down partials of layer l-1) -> h_b
+    in.kind = kResidual; in.h_in = h_in; in.h_out = c->h_b; in.part_in = c->part_b; in.n_parts_in = n_parts_prev; in.mpad_in = mpad_e;
+    in.gain = L.g_attn; in.ssq_out = c->ssq_attn; in.status = c->status;
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->part_a, c->sm_count, st), "gemv(qkv)");
+    c->ssq_attn = in.ssq_out;
+    c->ssq_attn.eps = g.rms_eps;
     LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos + n_tok),
-             launch_attention(c->qbuf, L.k, L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, &c->st_o, st), "attention");
-    GemvIn in_o{c->obuf, nullptr, 1.f, 0.f, c->st_o, c->status};
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->part, c->sm_count, st), "gemv(o)");
-    LAUNCH(c, launch_finish_residual(c->part, gemv_n_parts(L.o.n_sb), L.o.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(o)");
-    GemvIn in_f{c->h, L.g_ffn, L.gmax_ffn, g.rms_eps, c->st_h, c->status};
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->part, c->sm_count, st), "gemv(gate/up)");
-    LAUNCH(c, launch_finish_swiglu(c->part, gemv_n_parts(L.gu.n_sb), L.gu.mpad(), g.ffn, n_tok, c->act, &c->st_act, st), "finish_swiglu");
-    GemvIn in_d{c->act, nullptr, 1.f, 0.f, c->st_act, c->status};
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->part, c->sm_count, st), "gemv(down)");
-    LAUNCH(c, launch_finish_residual(c->part, gemv_n_parts(L.down.n_sb), L.down.mpad(), e_, n_tok, c->h, &c->st_h, st), "finish_residual(down)");
+             launch_attention(c->part_a, static_cast<int>(gemv_n_parts(L.qkv.n_sb)), L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k,
+                              L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, st), "attention");
+    GemvIn in_o;                                 // O: plain attention output
+    in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status;
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->part_b, c->sm_count, st), "gemv(o)");
+    GemvIn in_f;                                 // gate/up: h_b + O partials -> h_a
+    in_f.kind = kResidual; in_f.h_in = c->h_b; in_f.h_out = c->h_a; in_f.part_in = c->part_b;
+    in_f.n_parts_in = static_cast<int>(gemv_n_parts(L.o.n_sb)); in_f.mpad_in = L.o.mpad();
+    in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status;
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->part_a, c->sm_count, st), "gemv(gate/up)");
+    c->ssq_ffn = in_f.ssq_out;
+    c->ssq_ffn.eps = g.rms_eps;
+    GemvIn in_d;                                 // down: SwiGLU of the gate/up partials
+    in_d.kind = kSwiglu; in_d.part_in = c->part_a; in_d.n_parts_in = static_cast<int>(gemv_n_parts(L.gu.n_sb)); in_d.mpad_in = L.gu.mpad();
+    in_d.ssq_in = c->ssq_ffn; in_d.status = c->status;
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->part_b, c->sm_count, st), "gemv(down)");
+    h_in = c->h_a;
+    n_parts_prev = static_cast<int>(gemv_n_parts(L.down.n_sb));
   }
-  cudaError_t e = cudaMemcpyAsync(hidden_out, c->h, static_cast<size_t>(n_tok) * e_ * 4, cudaMemcpyDeviceToDevice, st);
-  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(hidden_out)");
+  LAUNCH(c, launch_finish_residual(c->part_b, n_parts_prev, mpad_e, e_, n_tok, c->h_a, hidden_out, st), "finish_residual");
   return PRIMA_OK;
 }
 
@@ -412,10 +430,13 @@ int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
   if (!c->have_out_norm || !c->have_head) return fail(c, PRIMA_ERR_STATE, "output norm or head not loaded");
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = c->stream;
-  LAUNCH(c, launch_copy_stats(hidden, nullptr, c->cfg.hidden, n_tok, &c->st_h, st), "copy_stats");
-  GemvIn in{hidden, c->g_out, c->gmax_out, c->cfg.rms_eps, c->st_h, c->status};
-  LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->part, c->sm_count, st), "gemv(head)");
-  LAUNCH(c, launch_finish_plain(c->part, gemv_n_parts(c->head.n_sb), c->head.mpad(), c->cfg.vocab, n_tok, logits, st), "finish_plain");
+  GemvIn in;        // the head stages hidden itself (no partial sums to add) and leaves its sums of squares
+  in.kind = kResidual; in.h_in = hidden; in.h_out = c->h_b; in.n_parts_in = 0; in.part_in = c->part_b;
+  in.mpad_in = (c->cfg.hidden + 7) / 8 * 8; in.gain = c->g_out; in.ssq_out = c->ssq_out; in.status = c->status;
+  LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->part_a, c->sm_count, st), "gemv(head)");
+  c->ssq_out = in.ssq_out;
+  c->ssq_out.eps = c->cfg.rms_eps;
+  LAUNCH(c, launch_finish_plain(c->part_a, gemv_n_parts(c->head.n_sb), c->head.mpad(), c->cfg.vocab, n_tok, logits, c->ssq_out, st), "finish_plain");
   return PRIMA_OK;
 }
 
@@ -576,7 +597,6 @@ int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int ma
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&p->w.data), p->w.bytes());
   if (e == cudaSuccess) e = cudaMemset(p->w.data, 0, p->w.bytes());
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->part), static_cast<size_t>(p->w.n_sb) * max_n_cols * p->w.mpad() * 4);
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->stats.data), sizeof(float2) * kMaxTok * kMaxStatBlocks);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->status), sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(int));
   if (e == cudaSuccess) {
@@ -595,12 +615,11 @@ int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int ma
 int prima_gemv_plan_run(prima_gemv_plan* p, const float* dev_x, int n_cols, float* dev_y, void* stream) {
   if (!p || !dev_x || !dev_y || n_cols < 1 || n_cols > p->max_n_cols) return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_plan_run: bad argument");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int k = launch_copy_stats(dev_x, nullptr, p->w.cols, n_cols, &p->stats, st);
-  if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "copy_stats");
-  GemvIn in{dev_x, nullptr, 1.f, 0.f, p->stats, p->status};
-  k = launch_gemv_partials(p->w, in, n_cols, p->part, p->sm_count, st);
+  GemvIn in;
+  in.kind = kPlain; in.x = dev_x; in.status = p->status;
+  int k = launch_gemv_partials(p->w, in, n_cols, p->part, p->sm_count, st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "gemv kernel");
-  k = launch_finish_plain(p->part, gemv_n_parts(p->w.n_sb), p->w.mpad(), p->w.rows, n_cols, dev_y, st);
+  k = launch_finish_plain(p->part, gemv_n_parts(p->w.n_sb), p->w.mpad(), p->w.rows, n_cols, dev_y, SumSq(), st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "finish kernel");
   return PRIMA_OK;
 }
@@ -609,7 +628,6 @@ int prima_gemv_plan_destroy(prima_gemv_plan* p) {
   if (!p) return PRIMA_OK;
   cudaFree(p->w.data);
   cudaFree(p->part);
-  cudaFree(p->stats.data);
   cudaFree(p->status);
   delete p;
   return PRIMA_OK;

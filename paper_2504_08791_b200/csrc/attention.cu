@@ -13,6 +13,11 @@
 // sum l of exp(s - m) and the un-normalised output.  A second kernel merges the chunks of a row in
 // ascending order:  M = max m_c,  o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c.
 // Token t of the step attends positions 0 .. pos + t (causal inside the step).
+//
+// The kernel also finishes the fused QKV product that precedes it: every CTA forms the queries of
+// its KV head from that product's partial sums (sum, RMSNorm factor, rotation), and the CTA whose
+// chunk contains a new position forms that position's key and value, rounds them to binary16 and
+// appends them to the cache before its warps read the chunk.
 #include "common.cuh"
 
 namespace prima {
@@ -39,12 +44,14 @@ __device__ __forceinline__ uint32_t pack_h2(float a, float b) {
 //  * O tile: instruction d of 16 has column n = g at head dim  64 (d / 8) + 8 g + (d % 8); the lane's
 //    k slots are the positions  2t, 2t+1, 2t+8, 2t+9  of the warp's 16.
 __global__ void __launch_bounds__(kThreads)
-attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_cache, const __half* __restrict__ v_cache,
-                    int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks,
+attn_partial_kernel(const float* __restrict__ part, int n_parts, int64_t mpad, const float* __restrict__ ssq, int n_groups,
+                    float inv_width, float eps, const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache,
+                    __half* __restrict__ v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks,
                     float* __restrict__ o_part, float2* __restrict__ ml_part) {
   pdl_trigger();
   __shared__ float s_o[kWarps][16][kHeadDim];
   __shared__ float s_m[kWarps][16], s_l[kWarps][16];
+  extern __shared__ float q_s[];                     // [n_rows][128] rotated queries of this KV head
 
   const int group = n_q_heads / n_kv_heads;
   const int n_rows = n_tok * group;                  // query rows served by this CTA
@@ -56,29 +63,93 @@ attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_ca
 
   // ---- K and V of the warp's 16 positions.  Entries below `pos` were written by earlier steps and do
   //      not change, so a warp whose positions are all old loads them before waiting for the
-  //      predecessor kernel (which writes the newest entries and the queries).
+  //      predecessor kernel; the others load after the new entries have been appended below.
   const bool old_only = wbase + 16 <= pos;
-  if (!old_only) pdl_wait();
   uint4 kreg[2][4];      // [position block of 8][32-dim slice]
   uint4 vreg[4][2];      // [k-slot position][64-dim half]
   const __half* kbase = k_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
   const __half* vbase = v_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
+  auto load_kv = [&]() {
 #pragma unroll
-  for (int pb = 0; pb < 2; ++pb) {
-    const int p = wbase + 8 * pb + g;
+    for (int pb = 0; pb < 2; ++pb) {
+      const int p = wbase + 8 * pb + g;
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-      kreg[pb][j] = p < n_ctx ? *reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t) : make_uint4(0, 0, 0, 0);
-  }
+      for (int j = 0; j < 4; ++j)
+        kreg[pb][j] = p < n_ctx ? __ldcg(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t)) : make_uint4(0, 0, 0, 0);
+    }
 #pragma unroll
-  for (int pi = 0; pi < 4; ++pi) {
-    const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
+    for (int pi = 0; pi < 4; ++pi) {
+      const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
 #pragma unroll
-    for (int hf = 0; hf < 2; ++hf)
-      vreg[pi][hf] = p < n_ctx ? *reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g) : make_uint4(0, 0, 0, 0);
-  }
+      for (int hf = 0; hf < 2; ++hf)
+        vreg[pi][hf] = p < n_ctx ? __ldcg(reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g)) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  if (old_only) load_kv();
+  pdl_wait();
 
-  if (old_only) pdl_wait();
+  // ---- finish the QKV product for this KV head: one thread per rotation pair
+  const int64_t pstride = static_cast<int64_t>(n_tok) * mpad;
+  auto pair_sum = [&](int tok, int64_t row_a, int64_t row_b, float& va, float& vb) {
+    va = vb = 0.f;
+    int p = 0;
+    for (; p + 4 <= n_parts; p += 4) {      // four loads in flight per row, additions in ascending order
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        a[i] = part[(p + i) * pstride + tok * mpad + row_a];
+        b[i] = part[(p + i) * pstride + tok * mpad + row_b];
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        va += a[i];
+        vb += b[i];
+      }
+    }
+    for (; p < n_parts; ++p) {
+      va += part[p * pstride + tok * mpad + row_a];
+      vb += part[p * pstride + tok * mpad + row_b];
+    }
+  };
+  auto token_scale = [&](int tok) {
+    float ss = 0.f;
+    for (int gi = 0; gi < n_groups; ++gi) ss += ssq[tok * kMaxStatBlocks + gi];
+    return 1.0f / sqrtf(ss * inv_width + eps);
+  };
+  const int chunk0 = chunk * kChunk;
+  for (int idx = threadIdx.x; idx < n_tok * (kHeadDim / 2); idx += kThreads) {   // new keys and values
+    const int tok = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
+    const int p = pos + tok;
+    if (p < chunk0 || p >= chunk0 + kChunk) continue;
+    const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
+    const float inv = token_scale(tok);
+    float ka, kb, va, vb;
+    pair_sum(tok, static_cast<int64_t>(n_q_heads + kv) * kHeadDim + a, static_cast<int64_t>(n_q_heads + kv) * kHeadDim + b, ka, kb);
+    pair_sum(tok, static_cast<int64_t>(n_q_heads + n_kv_heads + kv) * kHeadDim + a,
+             static_cast<int64_t>(n_q_heads + n_kv_heads + kv) * kHeadDim + b, va, vb);
+    ka *= inv; kb *= inv; va *= inv; vb *= inv;
+    const float2 cs = rope_tab[tok * (kHeadDim / 2) + i];
+    __half* kd = k_cache + (static_cast<int64_t>(kv) * kv_capacity + p) * kHeadDim;
+    __half* vd = v_cache + (static_cast<int64_t>(kv) * kv_capacity + p) * kHeadDim;
+    kd[a] = __float2half_rn(ka * cs.x - kb * cs.y);
+    kd[b] = __float2half_rn(kb * cs.x + ka * cs.y);
+    vd[a] = __float2half_rn(va);
+    vd[b] = __float2half_rn(vb);
+  }
+  for (int idx = threadIdx.x; idx < n_rows * (kHeadDim / 2); idx += kThreads) {   // queries
+    const int r = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
+    const int tok = r / group, head = kv * group + r % group;
+    const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
+    float qa_, qb_;
+    pair_sum(tok, static_cast<int64_t>(head) * kHeadDim + a, static_cast<int64_t>(head) * kHeadDim + b, qa_, qb_);
+    const float inv = token_scale(tok);
+    qa_ *= inv; qb_ *= inv;
+    const float2 cs = rope_tab[tok * (kHeadDim / 2) + i];
+    q_s[r * kHeadDim + a] = qa_ * cs.x - qb_ * cs.y;
+    q_s[r * kHeadDim + b] = qb_ * cs.x + qa_ * cs.y;
+  }
+  __syncthreads();
+  if (!old_only) load_kv();
 
   const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
   for (int tile = 0; tile * 16 < n_rows; ++tile) {
@@ -89,9 +160,8 @@ attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_ca
     for (int hr = 0; hr < 2; ++hr) {
       const int r = tile * 16 + g + 8 * hr;
       const bool live = r < n_rows;
-      const int tok = live ? r / group : 0, head = kv * group + (live ? r % group : 0);
-      row_tok[hr] = live ? tok : -1;
-      const float* qr = q + (static_cast<int64_t>(tok) * n_q_heads + head) * kHeadDim;
+      row_tok[hr] = live ? r / group : -1;
+      const float* qr = q_s + (live ? r : 0) * kHeadDim;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
@@ -207,8 +277,7 @@ attn_partial_kernel(const float* __restrict__ q, const __half* __restrict__ k_ca
 // One block of 128 threads per (token, head): merge the chunks in ascending order.  The weights
 // e^(m_c - M) / L of all chunks are prepared first, in parallel; then thread d sums its head dim.
 __global__ void __launch_bounds__(kHeadDim)
-attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks, int n_q_heads,
-                  float* __restrict__ o, float2* __restrict__ stats) {
+attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks, float* __restrict__ o) {
   pdl_trigger();
   pdl_wait();
   extern __shared__ float s_w[];         // [n_chunks]
@@ -237,43 +306,30 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
   for (int c = 0; c < n_chunks; ++c) acc += s_w[c] * op[static_cast<int64_t>(c) * kHeadDim];
   const float out = acc / denom;
   o[static_cast<int64_t>(row) * kHeadDim + d] = out;
-
-  __shared__ float s_ss[4], s_am[4];
-  float ss = out * out, am = fabsf(out);
-#pragma unroll
-  for (int of = 16; of > 0; of >>= 1) {
-    ss += __shfl_xor_sync(0xffffffffu, ss, of);
-    am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, of));
-  }
-  if ((d & 31) == 0) {
-    s_ss[d >> 5] = ss;
-    s_am[d >> 5] = am;
-  }
-  __syncthreads();
-  if (d == 0) {
-    const int tok = row / n_q_heads, head = row % n_q_heads;
-    stats[tok * kMaxStatBlocks + head] =
-        make_float2((s_ss[0] + s_ss[1]) + (s_ss[2] + s_ss[3]), fmaxf(fmaxf(s_am[0], s_am[1]), fmaxf(s_am[2], s_am[3])));
-  }
 }
 
 }  // namespace
 
 int attention_chunk_len() { return kChunk; }
 
-int launch_attention(const float* q, const __half* k_cache, const __half* v_cache, int kv_capacity, int n_q_heads,
-                     int n_kv_heads, int pos, int n_tok, const AttnScratch& scr, float* o, VecStats* stats, cudaStream_t st) {
+int launch_attention(const float* part_qkv, int n_parts, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode,
+                     __half* k_cache, __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok,
+                     const AttnScratch& scr, float* o, cudaStream_t st) {
   const int n_ctx = pos + n_tok;
   const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
   if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
+  const int n_rows = n_tok * (n_q_heads / n_kv_heads);
+  const size_t q_bytes = static_cast<size_t>(n_rows) * kHeadDim * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * kHeadDim * 4);
+  if (e != cudaSuccess) return cuda_rc(e);
   dim3 grid(n_chunks, n_kv_heads);
-  cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), 0, st, q, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok,
-                             n_chunks, scr.o_part, scr.ml_part);
+  e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), q_bytes, st, part_qkv, n_parts, mpad, static_cast<const float*>(ssq.data),
+                 ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps, rope_tab, rope_mode, k_cache, v_cache,
+                 kv_capacity, n_q_heads, n_kv_heads, pos, n_tok, n_chunks, scr.o_part, scr.ml_part);
   if (e != cudaSuccess) return cuda_rc(e);
   e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(n_chunks) * sizeof(float), st, scr.o_part,
-                 scr.ml_part, n_chunks, n_q_heads, o, stats->data);
+                 scr.ml_part, n_chunks, o);
   if (e != cudaSuccess) return cuda_rc(e);
-  stats->n_blocks = n_q_heads;
   return 2;
 }
 

@@ -53,11 +53,15 @@ struct TiledMat {
   int64_t mpad() const { return n_rt * kRowsPerTile; }
 };
 
-// Per-token activation statistics written by whichever kernel produced a vector and read by the
-// GEMV that consumes it: stats[tok][block] = (sum of squares, max |x|) over the block's slice.
-struct VecStats {
-  float2* data = nullptr;    // device, [kMaxTok][kMaxStatBlocks]
-  int n_blocks = 0;
+// Sums of squares of a vector, one per column group of the product that consumed it first:
+// ssq[tok * kMaxStatBlocks + group].  rsqrt(sum over groups / width + eps) is the RMSNorm factor.
+// Normalisation is *deferred*: a product with a normalised input multiplies by gain only and leaves
+// partial sums that still lack the scalar factor; whoever consumes those partial sums applies it.
+struct SumSq {
+  float* data = nullptr;     // device, [kMaxTok][kMaxStatBlocks]
+  int n_groups = 0;
+  int64_t width = 0;         // length of the vector the sums belong to
+  float eps = 0.f;
 };
 
 // ---- launch interfaces (definitions in the .cu files) ----------------------------------------
@@ -79,52 +83,56 @@ inline int64_t gemv_n_parts(int64_t n_sb) { return n_sb / gemv_group_size(n_sb);
 
 // Partial products of every (row, column group p of gemv_group_size(n_sb) super-block columns):
 //   part[(p * n_tok + t) * mpad + r] = sum over the weights of group p of W[r][k] * xhat[t][k]
-// where xhat = x * gain * rsqrt(mean(x^2) + eps) if gain != nullptr, else x.  x: [n_tok][cols].
+// A CTA stages the 256*SG activations of its column group in shared memory, finishing the
+// producer's output on the way (GemvIn.kind):
+//   kPlain    xhat = x
+//   kResidual v = h_in + sum over the n_parts_in partial sums of the previous product (ascending);
+//             v is written to h_out (the new residual stream), its sum of squares over the group to
+//             ssq_out, and xhat = v * gain (the RMSNorm scalar is left to the consumer of `part`)
+//   kSwiglu   xhat[k] = silu(G) * U with G, U = inv * the sums of the partial sums of fused rows
+//             2k, 2k+1 of the previous (gate/up) product, inv from ssq_in
+enum GemvKind { kPlain = 0, kResidual = 1, kSwiglu = 2 };
 struct GemvIn {
-  const float* x;        // [n_tok][cols] fp32
-  const float* gain;     // [cols] or nullptr (no normalisation)
-  float gain_max;        // max |gain| (1 if gain == nullptr)
-  float eps;
-  VecStats stats;        // statistics of x
-  int* status;           // device word raised if a bounded wait inside the kernel gives up
+  int kind = kPlain;
+  const float* x = nullptr;        // kPlain: [n_tok][cols]
+  const float* h_in = nullptr;     // kResidual: [n_tok][cols]
+  float* h_out = nullptr;          // kResidual: [n_tok][cols], must not alias h_in
+  const float* part_in = nullptr;  // kResidual / kSwiglu: partial sums of the previous product
+  int n_parts_in = 0;
+  int64_t mpad_in = 0;
+  const float* gain = nullptr;     // kResidual: [cols]
+  SumSq ssq_out;                   // kResidual: written (n_groups is set by the launcher)
+  SumSq ssq_in;                    // kSwiglu: read
+  int* status = nullptr;           // device word raised if a bounded wait inside the kernel gives up
 };
-int launch_gemv_partials(const TiledMat& w, const GemvIn& in, int n_tok, float* part, int sm_count,
-                         cudaStream_t st);
+int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, float* part, int sm_count, cudaStream_t st);
 
-// Finishers: sum the partials of a row over the super-block columns in ascending order, then
-//   plain:    y[t][r] = sum
-//   residual: h[t][r] = h[t][r] + sum, and statistics of the new h
-//   swiglu:   act[t][r] = silu(sum of fused row 2r) * (sum of fused row 2r+1), statistics of act
-//   qkv:      rows are [q heads | k heads | v heads] x 128; rotate q and k with the cos/sin table,
-//             write q (fp32, [n_tok][H*128]) and append k, v as binary16 to the cache at pos + t
-int launch_finish_plain(const float* part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok, float* y,
+// y[t][r] = scale_t * sum over the n_parts partial sums (ascending), scale_t = the RMSNorm factor
+// from ssq when ssq.data != nullptr, else 1.
+int launch_finish_plain(const float* part, int64_t n_parts, int64_t mpad, int64_t rows, int n_tok, float* y, const SumSq& ssq,
                         cudaStream_t st);
-int launch_finish_residual(const float* part, int64_t n_sb, int64_t mpad, int64_t rows, int n_tok, float* h,
-                           VecStats* stats, cudaStream_t st);
-int launch_finish_swiglu(const float* part, int64_t n_sb, int64_t mpad, int64_t ffn, int n_tok, float* act,
-                         VecStats* stats, cudaStream_t st);
-int launch_finish_qkv(const float* part, int64_t n_sb, int64_t mpad, int n_q_heads, int n_kv_heads, int n_tok,
-                      const float2* rope_tab, int rope_mode, float* q_out, __half* k_cache, __half* v_cache,
-                      int kv_capacity, int pos, cudaStream_t st);
-
-// Statistics of an arbitrary vector (used for the hidden state entering a window) and copy.
-int launch_copy_stats(const float* src, float* dst, int64_t width, int n_tok, VecStats* stats, cudaStream_t st);
+// out[t][r] = h[t][r] + sum over the partial sums (the residual stream leaving a window).
+int launch_finish_residual(const float* part, int64_t n_parts, int64_t mpad, int64_t rows, int n_tok, const float* h, float* out,
+                           cudaStream_t st);
 
 // cos/sin table for positions pos..pos+n_tok-1: tab[t][i] = (cos, sin)(pos_t * theta^(-2i/128)),
 // evaluated in double precision.
 int launch_rope_table(float2* tab, int pos, int n_tok, float theta, cudaStream_t st);
 
 // Grouped-query decode attention over the fp16 cache, split along the context, merged by
-// log-sum-exp.  q: [n_tok][H*128] fp32 (rotated).  Cache layout [G][capacity][128] binary16.
-// o: [n_tok][H*128] fp32 with statistics (max |o| per head).
+// log-sum-exp.  The queries, and the new keys and values, are taken from the partial sums of the
+// fused QKV product (rows [q heads | k heads | v heads] x 128): summed, scaled by the RMSNorm factor
+// from ssq, rotated with the cos/sin table; the new K and V are appended to the cache (binary16) at
+// positions pos + t by the CTAs whose chunk holds them.  Cache layout [G][capacity][128].
+// o: [n_tok][H*128] fp32.
 struct AttnScratch {
   float* o_part;    // [n_tok*H][n_chunks][128]
   float2* ml_part;  // [n_tok*H][n_chunks]  (running max, running sum)
   int max_chunks;
 };
-int launch_attention(const float* q, const __half* k_cache, const __half* v_cache, int kv_capacity, int n_q_heads,
-                     int n_kv_heads, int pos, int n_tok, const AttnScratch& scr, float* o, VecStats* stats,
-                     cudaStream_t st);
+int launch_attention(const float* part_qkv, int n_parts, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode,
+                     __half* k_cache, __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok,
+                     const AttnScratch& scr, float* o, cudaStream_t st);
 int attention_chunk_len();
 
 // Embedding lookup from a standard-layout table, and greedy argmax.

@@ -129,7 +129,7 @@ int prima_gemv_q4k_noalloc(const void* dev_w, int64_t rows, int64_t cols, const 
     snprintf(g_noalloc_error, sizeof(g_noalloc_error), "prima_gemv_q4k_noalloc: launch failed: %s", cudaGetErrorString(e));
     return PRIMA_ERR_CUDA;
   }
-  const int k = prima::launch_finish_plain(scratch, n_sb, rows, rows, n_cols, dev_y, st);
+  const int k = prima::launch_finish_plain(scratch, n_sb, rows, rows, n_cols, dev_y, prima::SumSq(), st);
   if (k < 0) return noalloc_fail(PRIMA_ERR_CUDA, "prima_gemv_q4k_noalloc: finishing kernel failed to launch");
   return PRIMA_OK;
 }

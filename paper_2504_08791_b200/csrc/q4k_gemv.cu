@@ -113,22 +113,12 @@ struct SubX {
   int sum;      // sum of x_q
 };
 
-__device__ __forceinline__ float4 load_x4(const float* __restrict__ xp, const float* __restrict__ gp, int c) {
-  float4 a = *reinterpret_cast<const float4*>(xp + 4 * c);
-  if (gp) {
-    const float4 gv = *reinterpret_cast<const float4*>(gp + 4 * c);
-    a.x *= gv.x; a.y *= gv.y; a.z *= gv.z; a.w *= gv.w;
-  }
-  return a;
-}
-
-// Quantise 32 consecutive activations (times gain, if any).  Two passes over the same 128 bytes
-// (maximum, then rounding) keep the register footprint of this rarely executed step small.
-__device__ __forceinline__ void load_sub(const float* __restrict__ xp, const float* __restrict__ gp, SubX& out) {
+// Quantise 32 consecutive staged activations (fp32 in shared memory).
+__device__ __forceinline__ void load_sub(const float* __restrict__ xs, SubX& out) {
   float amax = 0.f;
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
-    const float4 a = load_x4(xp, gp, c);
+    const float4 a = *reinterpret_cast<const float4*>(xs + 4 * c);
     amax = fmaxf(amax, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
   }
   const bool ok = amax > 0.f && amax < 3.0e38f;
@@ -136,7 +126,7 @@ __device__ __forceinline__ void load_sub(const float* __restrict__ xp, const flo
   int sum = 0;
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    const float4 a = load_x4(xp, gp, 2 * w), b = load_x4(xp, gp, 2 * w + 1);
+    const float4 a = *reinterpret_cast<const float4*>(xs + 8 * w), b = *reinterpret_cast<const float4*>(xs + 8 * w + 4);
     const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
 #pragma unroll
@@ -225,14 +215,100 @@ __device__ __forceinline__ void chunk_dot2(const uint4& q_u0, const uint4& q_u1,
   i_u1 = chunk_dot(q_u1, x);
 }
 
-// rsqrt(mean(x^2) + eps) of one token from the statistics blocks, reduced the same way in every warp.
-__device__ __forceinline__ float token_inv_rms(const float2* __restrict__ stats, int n_blocks, int tok, int64_t cols, float eps) {
-  const int lane = threadIdx.x & 31;
+// Kernel parameters (see GemvIn in common.cuh).
+struct GemvParams {
+  const uint8_t* w;
+  int n_rt, n_sb, sg;
+  int kind;
+  const float* x;
+  const float* h_in;
+  float* h_out;
+  const float* part_in;
+  int n_parts_in;
+  int64_t mpad_in;
+  const float* gain;
+  float* ssq_out;
+  const float* ssq_in;
+  int n_ssq_in;
+  float inv_width_in, eps_in;
+  int tok0, n_tok_total;
+  float* part;
+  int64_t mpad;
+  int* status;
+};
+
+// RMSNorm factor of one token from per-group sums of squares, groups added in ascending order.
+__device__ __forceinline__ float inv_rms(const float* __restrict__ ssq, int n_groups, int tok, float inv_width, float eps) {
   float ss = 0.f;
-  for (int b = lane; b < n_blocks; b += 32) ss += stats[tok * kMaxStatBlocks + b].x;
+  for (int gidx = 0; gidx < n_groups; ++gidx) ss += ssq[tok * kMaxStatBlocks + gidx];
+  return 1.0f / sqrtf(ss * inv_width + eps);
+}
+
+// Sum of n float4 partial sums at base + p * stride, p ascending.  Loads are issued eight at a time
+// so that their latencies overlap; the additions keep the ascending order.
+__device__ __forceinline__ float4 sum_parts4(const float* __restrict__ base, int64_t stride, int n) {
+  float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+  int p = 0;
+  for (; p + 8 <= n; p += 8) {
+    float4 a[8];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  return 1.0f / sqrtf(ss / static_cast<float>(cols) + eps);
+    for (int i = 0; i < 8; ++i) a[i] = *reinterpret_cast<const float4*>(base + (p + i) * stride);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      sum.x += a[i].x; sum.y += a[i].y; sum.z += a[i].z; sum.w += a[i].w;
+    }
+  }
+  float4 a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (p + i < n) a[i] = *reinterpret_cast<const float4*>(base + (p + i) * stride);
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (p + i < n) {
+      sum.x += a[i].x; sum.y += a[i].y; sum.z += a[i].z; sum.w += a[i].w;
+    }
+  return sum;
+}
+
+// A warp stages the 256 activations of its column s for NTOK tokens into xs[NTOK][256] (a ring slot
+// that is free at that moment), finishing the producer's output on the way; lane l owns columns
+// 8l .. 8l+7.  ss[k] receives the lane's share of the sum of squares (kResidual).
+template <int NTOK>
+__device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float* __restrict__ xs, float (&ss)[NTOK]) {
+  const int lane = threadIdx.x & 31;
+  const int64_t cols = static_cast<int64_t>(P.n_sb) * 256;
+  const int64_t k0 = static_cast<int64_t>(s) * 256 + 8 * lane;
+  const int64_t pstride = static_cast<int64_t>(P.n_tok_total) * P.mpad_in;
+#pragma unroll
+  for (int k = 0; k < NTOK; ++k) {
+    const int64_t row = static_cast<int64_t>(P.tok0 + k);
+    float* dst = xs + k * 256 + 8 * lane;
+    ss[k] = 0.f;
+    if (P.kind == kPlain) {
+      *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(P.x + row * cols + k0);
+      *reinterpret_cast<float4*>(dst + 4) = *reinterpret_cast<const float4*>(P.x + row * cols + k0 + 4);
+    } else if (P.kind == kResidual) {
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int64_t kk = k0 + 4 * hf;
+        const float4 sum = sum_parts4(P.part_in + row * P.mpad_in + kk, pstride, P.n_parts_in);
+        const float4 h = *reinterpret_cast<const float4*>(P.h_in + row * cols + kk);
+        const float4 v = make_float4(h.x + sum.x, h.y + sum.y, h.z + sum.z, h.w + sum.w);
+        *reinterpret_cast<float4*>(P.h_out + row * cols + kk) = v;
+        ss[k] += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+        const float4 gv = *reinterpret_cast<const float4*>(P.gain + kk);
+        *reinterpret_cast<float4*>(dst + 4 * hf) = make_float4(v.x * gv.x, v.y * gv.y, v.z * gv.z, v.w * gv.w);
+      }
+    } else {   // kSwiglu: the previous product's fused rows 2k (gate) and 2k+1 (up)
+      const float inv = inv_rms(P.ssq_in, P.n_ssq_in, P.tok0 + k, P.inv_width_in, P.eps_in);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 sum = sum_parts4(P.part_in + row * P.mpad_in + 2 * (k0 + 2 * q), pstride, P.n_parts_in);   // (G0, U0, G1, U1)
+        const float g0 = sum.x * inv, u0 = sum.y * inv, g1 = sum.z * inv, u1 = sum.w * inv;
+        *reinterpret_cast<float2*>(dst + 2 * q) = make_float2(g0 / (1.0f + expf(-g0)) * u0, g1 / (1.0f + expf(-g1)) * u1);
+      }
+    }
+  }
 }
 
 // Header of one unit row -> the lane's scale factors.
@@ -282,21 +358,24 @@ struct Walk {
 };
 
 template <int NTOK, bool MMA>
-__global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1))
-gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, const float* __restrict__ x,
-                     const float* __restrict__ gain, float eps, const float2* __restrict__ stats, int n_stat_blocks, int tok0,
-                     int n_tok_total, float* __restrict__ part, int64_t mpad, int* __restrict__ status) {
+__global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_partials_kernel(const GemvParams P) {
   pdl_trigger();
   extern __shared__ __align__(128) uint8_t smem[];
-  // layout: [warps][kRing][4608] batches, then [warps][kRing] mbarriers, then the reduction buffer
+  // layout: [warps][kRing][4608] batches, [warps][kRing] mbarriers, the reduction buffer
+  // [2][NTOK][kMaxWarps][kBatch][8], a small scratch for the sums of squares
   const int n_warps = blockDim.x >> 5;
+  const uint8_t* __restrict__ w = P.w;
+  const int n_rt = P.n_rt, n_sb = P.n_sb, sg = P.sg, tok0 = P.tok0, n_tok_total = P.n_tok_total;
+  float* __restrict__ part = P.part;
+  const int64_t mpad = P.mpad;
+  int* __restrict__ status = P.status;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(n_warps) * kRing * kBatchBytes);
-  float* red = reinterpret_cast<float*>(bars + n_warps * kRing);   // [2][NTOK][kMaxWarps][kBatch][8]
+  float* red = reinterpret_cast<float*>(bars + ((n_warps * kRing + 15) & ~15));   // keeps what follows 128-byte aligned
+  float* s_red = red + 2 * NTOK * kMaxWarps * kBatch * kRowsPerTile;   // [warps][NTOK]
 
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int64_t cols = static_cast<int64_t>(n_sb) * 256;
   // This CTA's range of (group, row tile) positions.  When the grid has at least one CTA per column
   // group, every group gets the same number of CTAs and a range never crosses a group boundary (a
   // crossing costs a second activation load in mid-stream, which only that CTA pays and everybody
@@ -328,61 +407,80 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
   __syncwarp();
 
   Walk pf, cur;                 // next batch to request / batch being computed
-  pf.init(p0, p1, n_rt);
   cur.init(p0, p1, n_rt);
   int n_in_flight = 0;          // requested and not yet waited for
-  auto request = [&](int slot) {
+  int rslot = 0;                // ring slot of the next request (requests and waits go round the ring in step)
+  auto request = [&]() {
     const int nb = pf.batch();
     if (lane == 0) {
       const uint8_t* src = w + (static_cast<int64_t>(pf.grp * sg + warp) * n_rt + pf.rt) * kUnitBytes;
-      mbar_expect_tx(bar_u32 + 8 * slot, nb * kUnitBytes);
-      bulk_load(ring_u32 + slot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * slot);
+      mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
+      bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot);
     }
     pf.next(nb);
     ++n_in_flight;
+    if (++rslot == kRing) rslot = 0;
   };
-#pragma unroll
-  for (int i = 0; i < kRing; ++i)
-    if (!pf.done()) request(i);
-
-  // the first weight batches are on their way; everything below depends on the predecessor kernel
-  pdl_wait();
-
-  float post[NTOK];
 
   // lane-constant byte selectors that pull this lane's 24-bit field group out of header words 1..3
   const uint32_t sel_a = t == 1 ? 0x7654u : (t == 3 ? 0x0073u : 0x3210u);
   const uint32_t sel_b = t == 2 ? 0x7654u : (t == 3 ? 0x0710u : 0x3210u);
 
   LaneX<MMA> xa[NTOK], xb[NTOK];   // sub-blocks t and 4 + t of the current column
-  int cur_grp = -1;
-  bool first = true;
   int parity = 0;
   bool alive = true;
-  int slot = 0;
+  bool waited = false;
+  int slot = 0;                  // ring slot of the next wait
   uint32_t phase = 0;
 
   while (!cur.done()) {
-    const int nb = cur.batch();
-    if (cur.grp != cur_grp) {
-      cur_grp = cur.grp;
-      const int s = cur.grp * sg + warp;
+    // ---- a segment: the positions of one column group.  The ring is empty here.  Request all
+    //      slots but one, use the free one as scratch for staging this column's activations,
+    //      then request it too.
+    const int seg_end = min(p1, (cur.grp + 1) * n_rt);
+    pf.init(cur.pos, seg_end, n_rt);
+#pragma unroll
+    for (int i = 0; i < kRing - 1; ++i)
+      if (!pf.done()) request();
+    if (!waited) {      // the first weight batches are on their way; everything below depends on the predecessor kernel
+      pdl_wait();
+      waited = true;
+    }
+    {
+      float* xs = reinterpret_cast<float*>(const_cast<uint8_t*>(my_ring) + rslot * kBatchBytes);
+      float ss[NTOK];
+      stage_warp<NTOK>(P, cur.grp * sg + warp, xs, ss);
+      __syncwarp();
 #pragma unroll
       for (int k = 0; k < NTOK; ++k) {
-        const float* xp = x + static_cast<int64_t>(tok0 + k) * cols + s * 256 + 32 * t;
-        const float* gp = gain ? gain + s * 256 + 32 * t : nullptr;
         SubX tmp;
-        load_sub(xp, gp, tmp);
+        load_sub(xs + k * 256 + 32 * t, tmp);
         xa[k].set(tmp, g, t);
-        load_sub(xp + 128, gp ? gp + 128 : nullptr, tmp);
+        load_sub(xs + k * 256 + 128 + 32 * t, tmp);
         xb[k].set(tmp, g, t);
       }
-      if (first) {      // after the activation loads, so that the two round trips overlap
-        first = false;
+      // the scratch is handed to the asynchronous copy engine next: order our accesses before it
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (!pf.done()) request();
+      if (P.kind == kResidual) {   // sums of squares of the group: lanes, then warps, in a fixed order
 #pragma unroll
-        for (int k = 0; k < NTOK; ++k) post[k] = gain ? token_inv_rms(stats, n_stat_blocks, tok0 + k, cols, eps) : 1.0f;
+        for (int k = 0; k < NTOK; ++k) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) ss[k] += __shfl_xor_sync(0xffffffffu, ss[k], o);
+          if (lane == 0) s_red[warp * NTOK + k] = ss[k];
+        }
+        __syncthreads();
+        if (threadIdx.x < NTOK) {
+          float a = 0.f;
+          for (int ww = 0; ww < n_warps; ++ww) a += s_red[ww * NTOK + threadIdx.x];
+          P.ssq_out[(tok0 + threadIdx.x) * kMaxStatBlocks + cur.grp] = a;
+        }
+        __syncthreads();
       }
     }
+    while (cur.pos < seg_end) {
+    const int nb = cur.batch();
     if (alive && !mbar_wait(bar_u32 + 8 * slot, phase)) {
       alive = false;
       if (lane == 0) atomicExch(status, 1);
@@ -411,7 +509,7 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
     }
     // the whole warp has consumed the slot: hand it back and request the next batch
     __syncwarp();
-    if (alive && !pf.done()) request(slot);
+    if (alive && !pf.done()) request();
 
     // quad reduction with transposition: lane t ends with the row sum of tile t
 #pragma unroll
@@ -438,7 +536,7 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
         const float* src = red + ((parity * NTOK + k) * kMaxWarps * kBatch + i) * kRowsPerTile + row;
         float sum = src[0];
         for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile];
-        part[(static_cast<int64_t>(cur.grp) * n_tok_total + tok0 + k) * mpad + (cur.rt + i) * kRowsPerTile + row] = sum * post[k];
+        part[(static_cast<int64_t>(cur.grp) * n_tok_total + tok0 + k) * mpad + (cur.rt + i) * kRowsPerTile + row] = sum;
       }
     }
     parity ^= 1;
@@ -447,6 +545,7 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
       phase ^= 1u;
     }
     cur.next(nb);
+    }
   }
   // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
   // outstanding slot one more bounded wait before the memory is released.
@@ -462,50 +561,66 @@ gemv_partials_kernel(const uint8_t* __restrict__ w, int n_rt, int n_sb, int sg, 
 }
 
 size_t gemv_smem_bytes(int sg, int n_tok) {
-  return static_cast<size_t>(sg) * kRing * kBatchBytes + static_cast<size_t>(sg) * kRing * 8 +
-         static_cast<size_t>(2) * n_tok * kMaxWarps * kBatch * kRowsPerTile * sizeof(float);
+  return static_cast<size_t>(sg) * kRing * kBatchBytes + static_cast<size_t>((sg * kRing + 15) & ~15) * 8 +
+         static_cast<size_t>(2) * n_tok * kMaxWarps * kBatch * kRowsPerTile * sizeof(float) +
+         static_cast<size_t>(kMaxWarps) * n_tok * sizeof(float);
 }
 
 template <int NTOK, bool MMA>
-cudaError_t launch_one(const TiledMat& w, const GemvIn& in, int sg, int64_t grid, int tok, int n_tok, float* part, cudaStream_t st) {
+cudaError_t launch_one(const GemvParams& P, int64_t grid, cudaStream_t st) {
   auto kern = gemv_partials_kernel<NTOK, MMA>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_smem_bytes(kMaxWarps, NTOK)));
   if (e != cudaSuccess) return e;
-  return launch_pdl(kern, dim3(static_cast<unsigned>(grid)), dim3(sg * 32), gemv_smem_bytes(sg, NTOK), st, w.data, static_cast<int>(w.n_rt),
-                    static_cast<int>(w.n_sb), sg, in.x, in.gain, in.eps, in.stats.data, in.stats.n_blocks, tok, n_tok, part, w.mpad(),
-                    in.status);
+  return launch_pdl(kern, dim3(static_cast<unsigned>(grid)), dim3(P.sg * 32), gemv_smem_bytes(P.sg, NTOK), st, P);
+}
+
+template <bool MMA>
+cudaError_t launch_n(int n, const GemvParams& P, int64_t grid, cudaStream_t st) {
+  switch (n) {
+    case 1: return launch_one<1, MMA>(P, grid, st);
+    case 2: return launch_one<2, MMA>(P, grid, st);
+    case 3: return launch_one<3, MMA>(P, grid, st);
+    default: return launch_one<4, MMA>(P, grid, st);
+  }
 }
 
 }  // namespace
 
 // Which inner product the GEMV uses.  Environment variable PRIMA_GEMV_KERNEL = "dp4a" or "mma"
-// (read once per process); default below.
+// (read once per process); the tensor-core variant is the default.
 bool gemv_uses_tensor_cores() {
   static const bool mma = [] {
     const char* v = getenv("PRIMA_GEMV_KERNEL");
-    if (v && v[0] == 'd') return false;
-    if (v && v[0] == 'm') return true;
-    return true;
+    return !(v && v[0] == 'd');
   }();
   return mma;
 }
 
-int launch_gemv_partials(const TiledMat& w, const GemvIn& in, int n_tok, float* part, int sm_count, cudaStream_t st) {
+int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, float* part, int sm_count, cudaStream_t st) {
   if (w.n_rt == 0 || w.n_sb == 0) return 0;
   if (w.n_rt * w.n_sb >= (int64_t(1) << 31)) return cuda_rc(cudaErrorInvalidValue);
   const int sg = gemv_group_size(w.n_sb);
   const int64_t n_pos = (w.n_sb / sg) * w.n_rt;
+  in.ssq_out.n_groups = static_cast<int>(w.n_sb / sg);
+  in.ssq_out.width = w.cols;
+  GemvParams P;
+  P.w = w.data; P.n_rt = static_cast<int>(w.n_rt); P.n_sb = static_cast<int>(w.n_sb); P.sg = sg;
+  P.kind = in.kind; P.x = in.x; P.h_in = in.h_in; P.h_out = in.h_out; P.part_in = in.part_in; P.n_parts_in = in.n_parts_in;
+  P.mpad_in = in.mpad_in; P.gain = in.gain; P.ssq_out = in.ssq_out.data; P.ssq_in = in.ssq_in.data; P.n_ssq_in = in.ssq_in.n_groups;
+  P.inv_width_in = in.ssq_in.width > 0 ? 1.0f / static_cast<float>(in.ssq_in.width) : 0.f;
+  P.eps_in = in.ssq_in.eps;
+  P.n_tok_total = n_tok; P.part = part; P.mpad = w.mpad(); P.status = in.status;
   int launches = 0;
   int tok = 0;
   while (tok < n_tok) {
-    const int chunk = (n_tok - tok >= 2) ? 2 : 1;
+    // up to 4 tokens per pass; 5..8 tokens are split as evenly as possible over two passes
+    const int left = n_tok - tok;
+    const int chunk = left <= 4 ? left : (left + 1) / 2;
     const int warps_per_sm = chunk == 1 ? 16 : 8;
     int64_t grid = static_cast<int64_t>(sm_count) * std::max(1, warps_per_sm / sg);
     if (grid > n_pos) grid = n_pos;
-    cudaError_t e;
-    const bool mma = gemv_uses_tensor_cores();
-    if (chunk == 1) e = mma ? launch_one<1, true>(w, in, sg, grid, tok, n_tok, part, st) : launch_one<1, false>(w, in, sg, grid, tok, n_tok, part, st);
-    else e = mma ? launch_one<2, true>(w, in, sg, grid, tok, n_tok, part, st) : launch_one<2, false>(w, in, sg, grid, tok, n_tok, part, st);
+    P.tok0 = tok;
+    const cudaError_t e = gemv_uses_tensor_cores() ? launch_n<true>(chunk, P, grid, st) : launch_n<false>(chunk, P, grid, st);
     if (e != cudaSuccess) return cuda_rc(e);
     ++launches;
     tok += chunk;
