@@ -110,6 +110,23 @@ class ClockSampler:
         return out
 
 
+# ------------------------------------------------------------------------------------ multi-rank
+def aggregate_over_ranks(ms_local: float, dist, device=None) -> float:
+    """Max over ranks of a rank's device time (ranks are independent replicas; the job takes as long
+    as its slowest rank).  `dist` is torch.distributed or None for a single process."""
+    if dist is None:
+        return ms_local
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(ms_per_step_max: float, world: int) -> dict:
+    """Whole-job numbers of N replicas that each decode one token per step."""
+    return {"ms_per_token": ms_per_step_max / world, "tokens_per_s": world * 1e3 / ms_per_step_max}
+
+
 # ------------------------------------------------------------------------------------ the GPU arm
 def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None):
     import torch
@@ -173,11 +190,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return aggregate_over_ranks(ms, dist, "cuda")
 
     for _ in range(args.warmup):
         device_step(n_ctx)
@@ -232,7 +245,7 @@ def run_ours(args, rank, world, local_rank):
 
     result = {
         "metric": "decode_ms_per_token",
-        "value": ms_step / world,
+        "value": job_value(ms_step, world)["ms_per_token"],
         "unit": "ms/token",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step,
@@ -241,7 +254,7 @@ def run_ours(args, rank, world, local_rank):
         "vs_baseline": None,
         "dtype": "q4_k weights x int16 activations, int32/fp32 accumulate",
         "data": "synthetic",
-        "tokens_per_s": world * 1e3 / ms_step,
+        "tokens_per_s": job_value(ms_step, world)["tokens_per_s"],
         "config": {"workload": desc, "layers": L, "windows": n_windows, "n_ctx": n_ctx, "n_tok": 1,
                    "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs larger than L2 (>= 4.9 GB per step)",
                    "bytes_per_token": bpt["total"]},
