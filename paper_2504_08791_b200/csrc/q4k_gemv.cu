@@ -113,39 +113,53 @@ struct SubX {
   int sum;      // sum of x_q
 };
 
-// Quantise 32 consecutive staged activations (fp32 in shared memory).
-__device__ __forceinline__ void load_sub(const float* __restrict__ xs, SubX& out) {
-  float amax = 0.f;
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    const float4 a = *reinterpret_cast<const float4*>(xs + 4 * c);
-    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
-  }
+// Quantise the warp's 256 staged activations (fp32, xs[256]) in place, every lane its own 8 values:
+// lane l holds quarter l % 4 of sub-block l / 4, i.e. exactly word l % 4 of that sub-block's byte
+// registers.  The sub-block's maximum and sum are formed over the 4 lanes with shuffles.  Afterwards
+// the lane's 32 bytes hold [hi even, hi odd, lo even, lo odd, step, sum, -, -].
+__device__ __forceinline__ void quantise_warp(float* __restrict__ xs) {
+  const int lane = threadIdx.x & 31;
+  float* mine = xs + 8 * lane;
+  const float4 a = *reinterpret_cast<const float4*>(mine), b = *reinterpret_cast<const float4*>(mine + 4);
+  const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  float amax = fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
+                     fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w))));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
   const bool ok = amax > 0.f && amax < 3.0e38f;
   const float inv_step = ok ? 32639.0f / amax : 0.f;
   int sum = 0;
+  uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    int xq = __float2int_rn(v[i] * inv_step);
+    xq = max(-32639, min(32639, xq));
+    sum += xq;
+    const int l = ((xq + 128) & 255) - 128;      // signed low byte
+    const int h = (xq - l) >> 8;                 // signed high byte, |h| <= 127
+    hi[i & 1] |= (static_cast<uint32_t>(h) & 0xffu) << (8 * (i >> 1));
+    lo[i & 1] |= (static_cast<uint32_t>(l) & 0xffu) << (8 * (i >> 1));
+  }
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+  __syncwarp();
+  *reinterpret_cast<uint4*>(mine) = make_uint4(hi[0], hi[1], lo[0], lo[1]);
+  mine[4] = ok ? amax / 32639.0f : 0.f;
+  reinterpret_cast<int*>(mine)[5] = sum;
+}
+
+// Collect sub-block j (0..7) of a quantised xs[256] into byte registers.
+__device__ __forceinline__ void gather_sub(const float* __restrict__ xs, int j, SubX& out) {
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    const float4 a = *reinterpret_cast<const float4*>(xs + 8 * w), b = *reinterpret_cast<const float4*>(xs + 8 * w + 4);
-    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      int xq = __float2int_rn(v[i] * inv_step);
-      xq = max(-32639, min(32639, xq));
-      sum += xq;
-      const int l = ((xq + 128) & 255) - 128;      // signed low byte
-      const int h = (xq - l) >> 8;                 // signed high byte, |h| <= 127
-      hi[i & 1] |= (static_cast<uint32_t>(h) & 0xffu) << (8 * (i >> 1));
-      lo[i & 1] |= (static_cast<uint32_t>(l) & 0xffu) << (8 * (i >> 1));
-    }
-    out.hi[2 * w] = hi[0];
-    out.hi[2 * w + 1] = hi[1];
-    out.lo[2 * w] = lo[0];
-    out.lo[2 * w + 1] = lo[1];
+    const uint4 q = *reinterpret_cast<const uint4*>(xs + 8 * (4 * j + w));
+    out.hi[2 * w] = q.x;
+    out.hi[2 * w + 1] = q.y;
+    out.lo[2 * w] = q.z;
+    out.lo[2 * w + 1] = q.w;
   }
-  out.step = ok ? amax / 32639.0f : 0.f;
-  out.sum = sum;
+  out.step = xs[8 * 4 * j + 4];
+  out.sum = reinterpret_cast<const int*>(xs)[8 * 4 * j + 5];
 }
 
 // What a lane keeps of one sub-block for the multiplications.
@@ -452,11 +466,14 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
       stage_warp<NTOK>(P, cur.grp * sg + warp, xs, ss);
       __syncwarp();
 #pragma unroll
+      for (int k = 0; k < NTOK; ++k) quantise_warp(xs + k * 256);
+      __syncwarp();
+#pragma unroll
       for (int k = 0; k < NTOK; ++k) {
         SubX tmp;
-        load_sub(xs + k * 256 + 32 * t, tmp);
+        gather_sub(xs + k * 256, t, tmp);
         xa[k].set(tmp, g, t);
-        load_sub(xs + k * 256 + 128 + 32 * t, tmp);
+        gather_sub(xs + k * 256, 4 + t, tmp);
         xb[k].set(tmp, g, t);
       }
       // the scratch is handed to the asynchronous copy engine next: order our accesses before it
