@@ -113,17 +113,18 @@ struct SubX {
   int sum;      // sum of x_q
 };
 
-// Quantise the warp's 256 staged activations (fp32, xs[256]) in place, every lane its own 8 values:
-// lane l holds quarter l % 4 of sub-block l / 4, i.e. exactly word l % 4 of that sub-block's byte
-// registers.  The sub-block's maximum and sum are formed over the 4 lanes with shuffles.  Afterwards
-// the lane's 32 bytes hold [hi even, hi odd, lo even, lo odd, step, sum, -, -].
-__device__ __forceinline__ void quantise_warp(float* __restrict__ xs) {
-  const int lane = threadIdx.x & 31;
-  float* mine = xs + 8 * lane;
-  const float4 a = *reinterpret_cast<const float4*>(mine), b = *reinterpret_cast<const float4*>(mine + 4);
-  const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-  float amax = fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
-                     fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w))));
+// Quantise the warp's 256 staged activations, every lane its own 8 values: lane l holds quarter
+// l % 4 of sub-block l / 4, i.e. exactly word l % 4 of that sub-block's byte registers
+// (q = [hi even, hi odd, lo even, lo odd]).  Maximum and sum over the sub-block come from shuffles.
+struct LaneQuant {
+  uint4 q;
+  float step;
+  int sum;
+};
+__device__ __forceinline__ LaneQuant quantise_lane(const float (&v)[8]) {
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
   const bool ok = amax > 0.f && amax < 3.0e38f;
@@ -142,24 +143,25 @@ __device__ __forceinline__ void quantise_warp(float* __restrict__ xs) {
   }
   sum += __shfl_xor_sync(0xffffffffu, sum, 1);
   sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-  __syncwarp();
-  *reinterpret_cast<uint4*>(mine) = make_uint4(hi[0], hi[1], lo[0], lo[1]);
-  mine[4] = ok ? amax / 32639.0f : 0.f;
-  reinterpret_cast<int*>(mine)[5] = sum;
+  LaneQuant r;
+  r.q = make_uint4(hi[0], hi[1], lo[0], lo[1]);
+  r.step = ok ? amax / 32639.0f : 0.f;
+  r.sum = sum;
+  return r;
 }
 
-// Collect sub-block j (0..7) of a quantised xs[256] into byte registers.
-__device__ __forceinline__ void gather_sub(const float* __restrict__ xs, int j, SubX& out) {
+// Collect sub-block j (0..7) from the lanes 4j .. 4j+3 that quantised it.
+__device__ __forceinline__ void gather_sub(const LaneQuant& mine, int j, SubX& out) {
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    const uint4 q = *reinterpret_cast<const uint4*>(xs + 8 * (4 * j + w));
-    out.hi[2 * w] = q.x;
-    out.hi[2 * w + 1] = q.y;
-    out.lo[2 * w] = q.z;
-    out.lo[2 * w + 1] = q.w;
+    const int src = 4 * j + w;
+    out.hi[2 * w] = __shfl_sync(0xffffffffu, mine.q.x, src);
+    out.hi[2 * w + 1] = __shfl_sync(0xffffffffu, mine.q.y, src);
+    out.lo[2 * w] = __shfl_sync(0xffffffffu, mine.q.z, src);
+    out.lo[2 * w + 1] = __shfl_sync(0xffffffffu, mine.q.w, src);
   }
-  out.step = xs[8 * 4 * j + 4];
-  out.sum = reinterpret_cast<const int*>(xs)[8 * 4 * j + 5];
+  out.step = __shfl_sync(0xffffffffu, mine.step, 4 * j);
+  out.sum = __shfl_sync(0xffffffffu, mine.sum, 4 * j);
 }
 
 // What a lane keeps of one sub-block for the multiplications.
@@ -284,11 +286,10 @@ __device__ __forceinline__ float4 sum_parts4(const float* __restrict__ base, int
   return sum;
 }
 
-// A warp stages the 256 activations of its column s for NTOK tokens into xs[NTOK][256] (a ring slot
-// that is free at that moment), finishing the producer's output on the way; lane l owns columns
-// 8l .. 8l+7.  ss[k] receives the lane's share of the sum of squares (kResidual).
+// A warp stages the 256 activations of its column s for NTOK tokens in registers, finishing the
+// producer's output on the way; lane l owns columns 8l .. 8l+7 (v[k][0..7]).  ss[k] receives the lane's share of the sum of squares (kResidual).
 template <int NTOK>
-__device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float* __restrict__ xs, float (&ss)[NTOK]) {
+__device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float (&v)[NTOK][8], float (&ss)[NTOK]) {
   const int lane = threadIdx.x & 31;
   const int64_t cols = static_cast<int64_t>(P.n_sb) * 256;
   const int64_t k0 = static_cast<int64_t>(s) * 256 + 8 * lane;
@@ -296,7 +297,7 @@ __device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float* __
 #pragma unroll
   for (int k = 0; k < NTOK; ++k) {
     const int64_t row = static_cast<int64_t>(P.tok0 + k);
-    float* dst = xs + k * 256 + 8 * lane;
+    float* dst = v[k];
     ss[k] = 0.f;
     if (P.kind == kPlain) {
       *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(P.x + row * cols + k0);
@@ -448,38 +449,30 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   uint32_t phase = 0;
 
   while (!cur.done()) {
-    // ---- a segment: the positions of one column group.  The ring is empty here.  Request all
-    //      slots but one, use the free one as scratch for staging this column's activations,
-    //      then request it too.
+    // ---- a segment: the positions of one column group.  The ring is empty here: fill it, then
+    //      (after the dependency wait) stage and quantise this column's activations in registers.
     const int seg_end = min(p1, (cur.grp + 1) * n_rt);
     pf.init(cur.pos, seg_end, n_rt);
 #pragma unroll
-    for (int i = 0; i < kRing - 1; ++i)
+    for (int i = 0; i < kRing; ++i)
       if (!pf.done()) request();
     if (!waited) {      // the first weight batches are on their way; everything below depends on the predecessor kernel
       pdl_wait();
       waited = true;
     }
     {
-      float* xs = reinterpret_cast<float*>(const_cast<uint8_t*>(my_ring) + rslot * kBatchBytes);
+      float v[NTOK][8];
       float ss[NTOK];
-      stage_warp<NTOK>(P, cur.grp * sg + warp, xs, ss);
-      __syncwarp();
-#pragma unroll
-      for (int k = 0; k < NTOK; ++k) quantise_warp(xs + k * 256);
-      __syncwarp();
+      stage_warp<NTOK>(P, cur.grp * sg + warp, v, ss);
 #pragma unroll
       for (int k = 0; k < NTOK; ++k) {
+        const LaneQuant lq = quantise_lane(v[k]);
         SubX tmp;
-        gather_sub(xs + k * 256, t, tmp);
+        gather_sub(lq, t, tmp);
         xa[k].set(tmp, g, t);
-        gather_sub(xs + k * 256, 4 + t, tmp);
+        gather_sub(lq, 4 + t, tmp);
         xb[k].set(tmp, g, t);
       }
-      // the scratch is handed to the asynchronous copy engine next: order our accesses before it
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (!pf.done()) request();
       if (P.kind == kResidual) {   // sums of squares of the group: lanes, then warps, in a fixed order
 #pragma unroll
         for (int k = 0; k < NTOK; ++k) {
