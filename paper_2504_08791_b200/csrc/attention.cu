@@ -1,6 +1,6 @@
 // Grouped-query decode attention over the fp16 KV cache, split along the context.
 //
-// One CTA of 4 warps per (context chunk of 64 positions, KV head); each warp owns 16 positions.
+// One CTA of 8 warps per (context chunk of 128 positions, KV head); each warp owns 16 positions.
 // The query rows that share the KV head -- the H/G heads of every token of the step, at most 64
 // rows -- are processed 16 at a time (one m16n8k16 tile of rows).  Per tile a warp computes
 //   S = Q K^T   with  A = Q (16 rows x 16 dims, fp16, pre-scaled by 1/sqrt(128)),  B = K,
@@ -8,7 +8,7 @@
 // all with fp32 accumulation on the tensor cores.  K and V go from global memory straight into
 // the B-operand registers with fully used 16-byte loads: the instruction's k index is only a
 // label, so each lane is given the head dimensions (for K) or positions (for V) that make its
-// bytes contiguous in the cache, and Q / P are arranged to match.  The four warps' (max, sum, O)
+// bytes contiguous in the cache, and Q / P are arranged to match.  The eight warps' (max, sum, O)
 // are combined through shared memory, giving per query row and chunk the running maximum m, the
 // sum l of exp(s - m) and the un-normalised output.  A second kernel merges the chunks of a row in
 // ascending order:  M = max m_c,  o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c.
@@ -23,8 +23,8 @@
 namespace prima {
 namespace {
 
-constexpr int kChunk = 64;
-constexpr int kWarps = 4;
+constexpr int kChunk = 128;
+constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -49,9 +49,11 @@ attn_partial_kernel(const float* __restrict__ part, int n_parts, int64_t mpad, c
                     __half* __restrict__ v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks,
                     float* __restrict__ o_part, float2* __restrict__ ml_part) {
   pdl_trigger();
-  __shared__ float s_o[kWarps][16][kHeadDim];
+  extern __shared__ float dyn_smem[];
+  float (*s_o)[16][kHeadDim] = reinterpret_cast<float (*)[16][kHeadDim]>(dyn_smem);   // [kWarps][16][128]
+  float* q_s = dyn_smem + kWarps * 16 * kHeadDim;    // [n_rows][128] rotated queries of this KV head
   __shared__ float s_m[kWarps][16], s_l[kWarps][16];
-  extern __shared__ float q_s[];                     // [n_rows][128] rotated queries of this KV head
+  __shared__ float s_inv[kMaxTok];
 
   const int group = n_q_heads / n_kv_heads;
   const int n_rows = n_tok * group;                  // query rows served by this CTA
@@ -111,18 +113,19 @@ attn_partial_kernel(const float* __restrict__ part, int n_parts, int64_t mpad, c
       vb += part[p * pstride + tok * mpad + row_b];
     }
   };
-  auto token_scale = [&](int tok) {
+  if (threadIdx.x < n_tok) {
     float ss = 0.f;
-    for (int gi = 0; gi < n_groups; ++gi) ss += ssq[tok * kMaxStatBlocks + gi];
-    return 1.0f / sqrtf(ss * inv_width + eps);
-  };
+    for (int gi = 0; gi < n_groups; ++gi) ss += ssq[threadIdx.x * kMaxStatBlocks + gi];
+    s_inv[threadIdx.x] = 1.0f / sqrtf(ss * inv_width + eps);
+  }
+  __syncthreads();
   const int chunk0 = chunk * kChunk;
   for (int idx = threadIdx.x; idx < n_tok * (kHeadDim / 2); idx += kThreads) {   // new keys and values
     const int tok = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
     const int p = pos + tok;
     if (p < chunk0 || p >= chunk0 + kChunk) continue;
     const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
-    const float inv = token_scale(tok);
+    const float inv = s_inv[tok];
     float ka, kb, va, vb;
     pair_sum(tok, static_cast<int64_t>(n_q_heads + kv) * kHeadDim + a, static_cast<int64_t>(n_q_heads + kv) * kHeadDim + b, ka, kb);
     pair_sum(tok, static_cast<int64_t>(n_q_heads + n_kv_heads + kv) * kHeadDim + a,
@@ -136,17 +139,35 @@ attn_partial_kernel(const float* __restrict__ part, int n_parts, int64_t mpad, c
     vd[a] = __float2half_rn(va);
     vd[b] = __float2half_rn(vb);
   }
-  for (int idx = threadIdx.x; idx < n_rows * (kHeadDim / 2); idx += kThreads) {   // queries
-    const int r = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
-    const int tok = r / group, head = kv * group + r % group;
-    const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
-    float qa_, qb_;
-    pair_sum(tok, static_cast<int64_t>(head) * kHeadDim + a, static_cast<int64_t>(head) * kHeadDim + b, qa_, qb_);
-    const float inv = token_scale(tok);
-    qa_ *= inv; qb_ *= inv;
-    const float2 cs = rope_tab[tok * (kHeadDim / 2) + i];
-    q_s[r * kHeadDim + a] = qa_ * cs.x - qb_ * cs.y;
-    q_s[r * kHeadDim + b] = qb_ * cs.x + qa_ * cs.y;
+  // queries: four rotation pairs per thread and trip, their loads issued together
+  const int n_pairs = n_rows * (kHeadDim / 2);
+  for (int base = threadIdx.x; base < n_pairs; base += 4 * kThreads) {
+    float qa_[4], qb_[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = base + u * kThreads;
+      qa_[u] = qb_[u] = 0.f;
+      if (idx < n_pairs) {
+        const int r = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
+        const int tok = r / group, head = kv * group + r % group;
+        const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
+        pair_sum(tok, static_cast<int64_t>(head) * kHeadDim + a, static_cast<int64_t>(head) * kHeadDim + b, qa_[u], qb_[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = base + u * kThreads;
+      if (idx < n_pairs) {
+        const int r = idx / (kHeadDim / 2), i = idx % (kHeadDim / 2);
+        const int tok = r / group;
+        const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
+        const float inv = s_inv[tok];
+        const float x = qa_[u] * inv, y = qb_[u] * inv;
+        const float2 cs = rope_tab[tok * (kHeadDim / 2) + i];
+        q_s[r * kHeadDim + a] = x * cs.x - y * cs.y;
+        q_s[r * kHeadDim + b] = y * cs.x + x * cs.y;
+      }
+    }
   }
   __syncthreads();
   if (!old_only) load_kv();
@@ -249,10 +270,11 @@ attn_partial_kernel(const float* __restrict__ part, int n_parts, int64_t mpad, c
       s_l[warp][g + 8] = lsum[1];
     }
     __syncthreads();
-    // ---- combine the four warps: thread d of 128 owns head dim d of every row of the tile
+    // ---- combine the warps: each group of 128 threads takes every (kThreads/128)-th row of the
+    //      tile, thread d of the group owning head dim d
     {
-      const int d = threadIdx.x;
-      for (int r = 0; r < 16 && tile * 16 + r < n_rows; ++r) {
+      const int d = threadIdx.x % kHeadDim;
+      for (int r = threadIdx.x / kHeadDim; r < 16 && tile * 16 + r < n_rows; r += kThreads / kHeadDim) {
         float big = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) big = fmaxf(big, s_m[w][r]);
@@ -319,8 +341,8 @@ int launch_attention(const float* part_qkv, int n_parts, int64_t mpad, const Sum
   const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
   if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
   const int n_rows = n_tok * (n_q_heads / n_kv_heads);
-  const size_t q_bytes = static_cast<size_t>(n_rows) * kHeadDim * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * kHeadDim * 4);
+  const size_t q_bytes = static_cast<size_t>(kWarps * 16 + n_rows) * kHeadDim * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (kWarps * 16 + 64) * kHeadDim * 4);
   if (e != cudaSuccess) return cuda_rc(e);
   dim3 grid(n_chunks, n_kv_heads);
   e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), q_bytes, st, part_qkv, n_parts, mpad, static_cast<const float*>(ssq.data),
