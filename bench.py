@@ -157,6 +157,8 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     shape, n_ctx, n_windows, desc = WORKLOADS[args.workload]
+    if args.ctx:
+        n_ctx = args.ctx
     cfg = synth.model_config(shape)
     if args.layers:
         cfg["n_layers"] = args.layers
@@ -338,6 +340,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="70b", choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
+    ap.add_argument("--ctx", type=int, default=0, help="override the KV context length (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

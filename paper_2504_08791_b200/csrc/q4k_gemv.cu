@@ -70,9 +70,17 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar)
+// The weights are read once per token and never again before hundreds of MB of other weights have
+// passed: they are marked evict-first in L2, so that the small arrays the kernels hand to each other
+// (partial sums, the residual stream, gains, statistics) stay resident instead of being pushed out.
+__device__ __forceinline__ uint64_t stream_once_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar), "l"(policy)
                : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
@@ -430,7 +438,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     if (lane == 0) {
       const uint8_t* src = w + (static_cast<int64_t>(pf.grp * sg + warp) * n_rt + pf.rt) * kUnitBytes;
       mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
-      bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot);
+      bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot, stream_once_policy());
     }
     pf.next(nb);
     ++n_in_flight;
