@@ -52,8 +52,12 @@ struct prima_ctx {
   uint8_t* embd = nullptr;
   bool have_out_norm = false, have_head = false, have_embd = false;
 
-  float* part_a = nullptr;   // partial sums of the QKV, gate/up and head products
-  float* part_b = nullptr;   // partial sums of the O and down products
+  // fixed-point accumulators of the products, [max_n_tok][padded rows] each; all zero between calls
+  acc_t* acc_qkv = nullptr;  // QKV and head products
+  acc_t* acc_o = nullptr;    // O product
+  acc_t* acc_gu = nullptr;   // gate/up product
+  acc_t* acc_down = nullptr; // down product
+  int64_t n_acc_qkv = 0, n_acc_o = 0, n_acc_gu = 0, n_acc_down = 0;
   float* h_a = nullptr;      // residual stream entering a layer / leaving its feed-forward block
   float* h_b = nullptr;      // residual stream after the attention block
   float* obuf = nullptr;
@@ -83,7 +87,7 @@ struct prima_gemv_plan {
   int sm_count = 0;
   int max_n_cols = 1;
   TiledMat w;
-  float* part = nullptr;
+  acc_t* acc = nullptr;
   int* status = nullptr;
 };
 
@@ -235,19 +239,19 @@ int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx
   const int64_t n = g.max_n_tok;
   const int64_t e_ = g.hidden, H = g.n_q_heads, G = g.n_kv_heads, F = g.ffn;
   auto pad8 = [](int64_t r) { return (r + 7) / 8 * 8; };
-  int64_t part_a = 0, part_b = 0;
-  part_a = std::max(part_a, (e_ / 256) * n * pad8((H + 2 * G) * kHeadDim));
-  part_a = std::max(part_a, (e_ / 256) * n * pad8(2 * F));
-  part_a = std::max(part_a, (e_ / 256) * n * pad8(g.vocab));
-  part_b = std::max(part_b, (H * kHeadDim / 256) * n * pad8(e_));
-  part_b = std::max(part_b, (F / 256) * n * pad8(e_));
+  c->n_acc_qkv = n * std::max(pad8((H + 2 * G) * kHeadDim), pad8(g.vocab));
+  c->n_acc_o = n * pad8(e_);
+  c->n_acc_gu = n * pad8(2 * F);
+  c->n_acc_down = n * pad8(e_);
   c->attn.max_chunks = (g.kv_capacity + attention_chunk_len() - 1) / attention_chunk_len();
   c->staging_bytes = 256u << 20;
 
   int rc = PRIMA_OK;
   auto A = [&](int r) { if (rc == PRIMA_OK) rc = r; };
-  A(dev_alloc(c, &c->part_a, static_cast<size_t>(part_a)));
-  A(dev_alloc(c, &c->part_b, static_cast<size_t>(part_b)));
+  A(dev_alloc(c, &c->acc_qkv, static_cast<size_t>(c->n_acc_qkv), true));
+  A(dev_alloc(c, &c->acc_o, static_cast<size_t>(c->n_acc_o), true));
+  A(dev_alloc(c, &c->acc_gu, static_cast<size_t>(c->n_acc_gu), true));
+  A(dev_alloc(c, &c->acc_down, static_cast<size_t>(c->n_acc_down), true));
   A(dev_alloc(c, &c->h_a, static_cast<size_t>(n * e_)));
   A(dev_alloc(c, &c->h_b, static_cast<size_t>(n * e_)));
   A(dev_alloc(c, &c->obuf, static_cast<size_t>(n * H * kHeadDim)));
@@ -386,40 +390,46 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
   }
   LAUNCH(c, launch_rope_table(c->rope_tab, pos, n_tok, g.rope_theta, st), "rope_table");
   const int64_t mpad_e = (e_ + 7) / 8 * 8;
-  // The residual stream entering a layer is h_in plus the still unsummed partial sums of the previous
-  // down projection (none for the first layer of the call); each product's CTAs finish what they
-  // need of their producer's output while staging their activations.
+  // The residual stream entering a layer is h_in plus the value of the previous down projection's
+  // accumulators (nothing for the first layer of the call); each product's CTAs finish what they
+  // need of their producer's output while staging their activations.  Every accumulator array is
+  // cleared by the kernel that follows its last reader: gate/up's by the next QKV product (or the
+  // closing kernel), QKV's and down's by the O product, O's by the down product.
   const float* h_in = hidden_in;
-  int n_parts_prev = 0;
+  const acc_t* acc_prev = nullptr;
   for (int l = layer_begin; l < layer_end; ++l) {
     Layer& L = c->layers[l];
-    GemvIn in;                                   // QKV: residual (+ down partials of layer l-1) -> h_b
-    in.kind = kResidual; in.h_in = h_in; in.h_out = c->h_b; in.part_in = c->part_b; in.n_parts_in = n_parts_prev; in.mpad_in = mpad_e;
+    GemvIn in;                                   // QKV: residual (+ down projection of layer l-1) -> h_b
+    in.kind = kResidual; in.h_in = h_in; in.h_out = c->h_b; in.acc_in = acc_prev; in.mpad_in = mpad_e;
     in.gain = L.g_attn; in.ssq_out = c->ssq_attn; in.status = c->status;
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->part_a, c->sm_count, st), "gemv(qkv)");
+    in.zero0 = c->acc_gu; in.zero0_n = static_cast<int64_t>(n_tok) * L.gu.mpad();
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(qkv)");
     c->ssq_attn = in.ssq_out;
     c->ssq_attn.eps = g.rms_eps;
     LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos + n_tok),
-             launch_attention(c->part_a, static_cast<int>(gemv_n_parts(L.qkv.n_sb)), L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k,
-                              L.v, g.kv_capacity, H, G, pos, n_tok, c->attn, c->obuf, st), "attention");
+             launch_attention(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k, L.v, g.kv_capacity, H, G, pos, n_tok,
+                              c->attn, c->obuf, c->sm_count, st), "attention");
     GemvIn in_o;                                 // O: plain attention output
     in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status;
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->part_b, c->sm_count, st), "gemv(o)");
-    GemvIn in_f;                                 // gate/up: h_b + O partials -> h_a
-    in_f.kind = kResidual; in_f.h_in = c->h_b; in_f.h_out = c->h_a; in_f.part_in = c->part_b;
-    in_f.n_parts_in = static_cast<int>(gemv_n_parts(L.o.n_sb)); in_f.mpad_in = L.o.mpad();
+    in_o.zero0 = c->acc_qkv; in_o.zero0_n = static_cast<int64_t>(n_tok) * L.qkv.mpad();
+    in_o.zero1 = c->acc_down; in_o.zero1_n = static_cast<int64_t>(n_tok) * mpad_e;
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->acc_o, c->sm_count, st), "gemv(o)");
+    GemvIn in_f;                                 // gate/up: h_b + O projection -> h_a
+    in_f.kind = kResidual; in_f.h_in = c->h_b; in_f.h_out = c->h_a; in_f.acc_in = c->acc_o; in_f.mpad_in = L.o.mpad();
     in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status;
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->part_a, c->sm_count, st), "gemv(gate/up)");
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->acc_gu, c->sm_count, st), "gemv(gate/up)");
     c->ssq_ffn = in_f.ssq_out;
     c->ssq_ffn.eps = g.rms_eps;
-    GemvIn in_d;                                 // down: SwiGLU of the gate/up partials
-    in_d.kind = kSwiglu; in_d.part_in = c->part_a; in_d.n_parts_in = static_cast<int>(gemv_n_parts(L.gu.n_sb)); in_d.mpad_in = L.gu.mpad();
+    GemvIn in_d;                                 // down: SwiGLU of the gate/up product
+    in_d.kind = kSwiglu; in_d.acc_in = c->acc_gu; in_d.mpad_in = L.gu.mpad();
     in_d.ssq_in = c->ssq_ffn; in_d.status = c->status;
-    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->part_b, c->sm_count, st), "gemv(down)");
+    in_d.zero0 = c->acc_o; in_d.zero0_n = static_cast<int64_t>(n_tok) * L.o.mpad();
+    LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->acc_down, c->sm_count, st), "gemv(down)");
     h_in = c->h_a;
-    n_parts_prev = static_cast<int>(gemv_n_parts(L.down.n_sb));
+    acc_prev = c->acc_down;
   }
-  LAUNCH(c, launch_finish_residual(c->part_b, n_parts_prev, mpad_e, e_, n_tok, c->h_a, hidden_out, st), "finish_residual");
+  LAUNCH(c, launch_finish_residual(c->acc_down, mpad_e, e_, n_tok, c->h_a, hidden_out, c->acc_gu,
+                                   static_cast<int64_t>(n_tok) * c->layers[layer_end - 1].gu.mpad(), st), "finish_residual");
   return PRIMA_OK;
 }
 
@@ -431,12 +441,12 @@ int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = c->stream;
   GemvIn in;        // the head stages hidden itself (no partial sums to add) and leaves its sums of squares
-  in.kind = kResidual; in.h_in = hidden; in.h_out = c->h_b; in.n_parts_in = 0; in.part_in = c->part_b;
+  in.kind = kResidual; in.h_in = hidden; in.h_out = c->h_b; in.acc_in = nullptr;
   in.mpad_in = (c->cfg.hidden + 7) / 8 * 8; in.gain = c->g_out; in.ssq_out = c->ssq_out; in.status = c->status;
-  LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->part_a, c->sm_count, st), "gemv(head)");
+  LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(head)");
   c->ssq_out = in.ssq_out;
   c->ssq_out.eps = c->cfg.rms_eps;
-  LAUNCH(c, launch_finish_plain(c->part_a, gemv_n_parts(c->head.n_sb), c->head.mpad(), c->cfg.vocab, n_tok, logits, c->ssq_out, st), "finish_plain");
+  LAUNCH(c, launch_finish_acc(c->acc_qkv, c->head.mpad(), c->cfg.vocab, n_tok, logits, c->ssq_out, st), "finish_acc");
   return PRIMA_OK;
 }
 
@@ -596,7 +606,9 @@ int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int ma
   p->w = shape_tiled(rows, cols);
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&p->w.data), p->w.bytes());
   if (e == cudaSuccess) e = cudaMemset(p->w.data, 0, p->w.bytes());
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->part), static_cast<size_t>(p->w.n_sb) * max_n_cols * p->w.mpad() * 4);
+  const size_t acc_bytes = static_cast<size_t>(max_n_cols) * p->w.mpad() * sizeof(acc_t);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->acc), acc_bytes);
+  if (e == cudaSuccess) e = cudaMemset(p->acc, 0, acc_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&p->status), sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(p->status, 0, sizeof(int));
   if (e == cudaSuccess) {
@@ -617,9 +629,9 @@ int prima_gemv_plan_run(prima_gemv_plan* p, const float* dev_x, int n_cols, floa
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   GemvIn in;
   in.kind = kPlain; in.x = dev_x; in.status = p->status;
-  int k = launch_gemv_partials(p->w, in, n_cols, p->part, p->sm_count, st);
+  int k = launch_gemv_partials(p->w, in, n_cols, p->acc, p->sm_count, st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "gemv kernel");
-  k = launch_finish_plain(p->part, gemv_n_parts(p->w.n_sb), p->w.mpad(), p->w.rows, n_cols, dev_y, SumSq(), st);
+  k = launch_finish_acc(p->acc, p->w.mpad(), p->w.rows, n_cols, dev_y, SumSq(), st);
   if (k < 0) return cuda_fail(nullptr, static_cast<cudaError_t>(-k), "finish kernel");
   return PRIMA_OK;
 }
@@ -627,7 +639,7 @@ int prima_gemv_plan_run(prima_gemv_plan* p, const float* dev_x, int n_cols, floa
 int prima_gemv_plan_destroy(prima_gemv_plan* p) {
   if (!p) return PRIMA_OK;
   cudaFree(p->w.data);
-  cudaFree(p->part);
+  cudaFree(p->acc);
   cudaFree(p->status);
   delete p;
   return PRIMA_OK;

@@ -75,53 +75,74 @@ int launch_dequant_std(const uint8_t* blocks, int64_t n_sb, float* out, cudaStre
 int launch_retile(const uint8_t* src, int64_t rows_src, int64_t n_sb, TiledMat dst, int64_t dst_row0,
                   int64_t dst_row_stride, cudaStream_t st);
 
+// ---- fixed-point accumulators --------------------------------------------------------------------
+// A product is computed as partial sums over groups of super-block columns by different CTAs.  The
+// partial sums of one output element are added into a 64-bit fixed-point accumulator (two's
+// complement, 32 fractional bits) with integer atomics: integer addition is associative, so the
+// result does not depend on the order in which the CTAs arrive -- the bits are the same from run
+// to run and under any split into windows -- and whoever consumes the product reads ONE word per
+// element instead of one per group.  Range +-2^31, resolution 2^-32 per partial sum; a partial sum
+// outside +-2^27 raises the device status word.  An accumulator array must be all zero when the
+// product that adds into it starts; the kernels clear the arrays behind their readers.
+using acc_t = unsigned long long;
+constexpr float kAccScale = 4294967296.0f;                 // 2^32
+constexpr float kAccInvScale = 2.3283064365386963e-10f;    // 2^-32
+constexpr float kAccLimit = 134217728.0f;                  // 2^27
+
 // Number of adjacent super-block columns one CTA of the GEMV works on (largest divisor of n_sb
-// that is <= 8), and the number of partial sums per row that the GEMV leaves for the finishers.
+// that is <= 8).
 int gemv_group_size(int64_t n_sb);
 bool gemv_uses_tensor_cores();
-inline int64_t gemv_n_parts(int64_t n_sb) { return n_sb / gemv_group_size(n_sb); }
 
-// Partial products of every (row, column group p of gemv_group_size(n_sb) super-block columns):
-//   part[(p * n_tok + t) * mpad + r] = sum over the weights of group p of W[r][k] * xhat[t][k]
-// A CTA stages the 256*SG activations of its column group in shared memory, finishing the
-// producer's output on the way (GemvIn.kind):
+// acc[t * mpad + r] += sum over the weights of column group p of W[r][k] * xhat[t][k], for every
+// group p.  A warp stages the 256 activations of its column in registers, finishing the producer's
+// output on the way (GemvIn.kind):
 //   kPlain    xhat = x
-//   kResidual v = h_in + sum over the n_parts_in partial sums of the previous product (ascending);
+//   kResidual v = h_in + value(acc_in) (acc_in = the accumulators of the previous product, or null);
 //             v is written to h_out (the new residual stream), its sum of squares over the group to
-//             ssq_out, and xhat = v * gain (the RMSNorm scalar is left to the consumer of `part`)
-//   kSwiglu   xhat[k] = silu(G) * U with G, U = inv * the sums of the partial sums of fused rows
-//             2k, 2k+1 of the previous (gate/up) product, inv from ssq_in
+//             ssq_out, and xhat = v * gain (the RMSNorm scalar is left to the consumer of `acc`)
+//   kSwiglu   xhat[k] = silu(G) * U with G, U = inv * the values of acc_in for fused rows 2k, 2k+1 of
+//             the previous (gate/up) product, inv from ssq_in
+// After its dependency wait the kernel also clears the accumulator arrays zero0 / zero1 (arrays
+// whose last reader was the predecessor kernel or an earlier one).
 enum GemvKind { kPlain = 0, kResidual = 1, kSwiglu = 2 };
 struct GemvIn {
   int kind = kPlain;
   const float* x = nullptr;        // kPlain: [n_tok][cols]
   const float* h_in = nullptr;     // kResidual: [n_tok][cols]
   float* h_out = nullptr;          // kResidual: [n_tok][cols], must not alias h_in
-  const float* part_in = nullptr;  // kResidual / kSwiglu: partial sums of the previous product
-  int n_parts_in = 0;
+  const acc_t* acc_in = nullptr;   // kResidual (optional) / kSwiglu: [n_tok][mpad_in]
   int64_t mpad_in = 0;
   const float* gain = nullptr;     // kResidual: [cols]
   SumSq ssq_out;                   // kResidual: written (n_groups is set by the launcher)
   SumSq ssq_in;                    // kSwiglu: read
-  int* status = nullptr;           // device word raised if a bounded wait inside the kernel gives up
+  acc_t* zero0 = nullptr;          // accumulator arrays to clear, with their lengths
+  int64_t zero0_n = 0;
+  acc_t* zero1 = nullptr;
+  int64_t zero1_n = 0;
+  int* status = nullptr;           // device word raised if a bounded wait gives up (1) or a partial sum is out of range (2)
 };
-int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, float* part, int sm_count, cudaStream_t st);
+int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, int sm_count, cudaStream_t st);
+
+// y[t][r] = scale_t * value(acc[t * mpad + r]), scale_t = the RMSNorm factor from ssq when
+// ssq.data != nullptr, else 1; every accumulator is cleared after it has been read.
+int launch_finish_acc(acc_t* acc, int64_t mpad, int64_t rows, int n_tok, float* y, const SumSq& ssq, cudaStream_t st);
+// out[t][r] = h[t][r] + value(acc[t * mpad + r]) (the residual stream leaving a window); clears acc
+// behind the read and the array zero0.
+int launch_finish_residual(acc_t* acc, int64_t mpad, int64_t rows, int n_tok, const float* h, float* out, acc_t* zero0, int64_t zero0_n,
+                           cudaStream_t st);
 
 // y[t][r] = scale_t * sum over the n_parts partial sums (ascending), scale_t = the RMSNorm factor
 // from ssq when ssq.data != nullptr, else 1.
 int launch_finish_plain(const float* part, int64_t n_parts, int64_t mpad, int64_t rows, int n_tok, float* y, const SumSq& ssq,
                         cudaStream_t st);
-// out[t][r] = h[t][r] + sum over the partial sums (the residual stream leaving a window).
-int launch_finish_residual(const float* part, int64_t n_parts, int64_t mpad, int64_t rows, int n_tok, const float* h, float* out,
-                           cudaStream_t st);
-
 // cos/sin table for positions pos..pos+n_tok-1: tab[t][i] = (cos, sin)(pos_t * theta^(-2i/128)),
 // evaluated in double precision.
 int launch_rope_table(float2* tab, int pos, int n_tok, float theta, cudaStream_t st);
 
 // Grouped-query decode attention over the fp16 cache, split along the context, merged by
-// log-sum-exp.  The queries, and the new keys and values, are taken from the partial sums of the
-// fused QKV product (rows [q heads | k heads | v heads] x 128): summed, scaled by the RMSNorm factor
+// log-sum-exp.  The queries, and the new keys and values, are taken from the accumulators of the
+// fused QKV product (rows [q heads | k heads | v heads] x 128): scaled by the RMSNorm factor
 // from ssq, rotated with the cos/sin table; the new K and V are appended to the cache (binary16) at
 // positions pos + t by the CTAs whose chunk holds them.  Cache layout [G][capacity][128].
 // o: [n_tok][H*128] fp32.
@@ -130,9 +151,9 @@ struct AttnScratch {
   float2* ml_part;  // [n_tok*H][n_chunks]  (running max, running sum)
   int max_chunks;
 };
-int launch_attention(const float* part_qkv, int n_parts, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode,
+int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode,
                      __half* k_cache, __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok,
-                     const AttnScratch& scr, float* o, cudaStream_t st);
+                     const AttnScratch& scr, float* o, int sm_count, cudaStream_t st);
 int attention_chunk_len();
 
 // Embedding lookup from a standard-layout table, and greedy argmax.
@@ -151,6 +172,9 @@ inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? 0 : -static_cast<i
 // it reads anything a predecessor wrote or writes anything a predecessor may still read; what it
 // does before pdl_wait() (set-up, prefetching immutable weights) overlaps the predecessor's tail.
 #ifdef __CUDACC__
+__device__ __forceinline__ float acc_value(acc_t a) { return static_cast<float>(static_cast<long long>(a)) * kAccInvScale; }
+__device__ __forceinline__ acc_t acc_from(float v) { return static_cast<acc_t>(__float2ll_rn(v * kAccScale)); }
+
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -1,5 +1,6 @@
-// Finishers of the streaming GEMV that are still separate kernels (logits, and the residual stream
-// leaving a window), the rotary table and the greedy argmax.
+// Finishers that are separate kernels (logits, the residual stream leaving a window, the sum over
+// per-column partial sums used by the entry point that allocates nothing), the rotary table and the
+// greedy argmax.
 #include "common.cuh"
 
 namespace prima {
@@ -31,16 +32,39 @@ __global__ void finish_plain_kernel(const float* __restrict__ part, int64_t n_pa
     y[tok * rows + r] = scale * column_sum(part, n_parts, stride, tok * mpad + r);
 }
 
-// out[t][r] = h[t][r] + sum of the partial sums (same expression as the staging step of the GEMV,
-// so a window boundary changes no bits).
-__global__ void finish_residual_kernel(const float* __restrict__ part, int64_t n_parts, int64_t mpad, int64_t rows, int n_tok,
-                                       const float* __restrict__ h, float* __restrict__ out) {
+// y[t][r] = scale_t * value(acc[t * mpad + r]); the accumulator is cleared behind the read.
+__global__ void finish_acc_kernel(acc_t* __restrict__ acc, int64_t mpad, int64_t rows, int n_tok, float* __restrict__ y,
+                                  const float* __restrict__ ssq, int n_groups, float inv_width, float eps) {
   pdl_trigger();
   pdl_wait();
   const int tok = blockIdx.y;
-  const int64_t stride = static_cast<int64_t>(n_tok) * mpad;
-  for (int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; r < rows; r += static_cast<int64_t>(gridDim.x) * kBlock)
-    out[tok * rows + r] = h[tok * rows + r] + column_sum(part, n_parts, stride, tok * mpad + r);
+  float scale = 1.0f;
+  if (ssq) {
+    float ss = 0.f;
+    for (int gi = 0; gi < n_groups; ++gi) ss += ssq[tok * kMaxStatBlocks + gi];
+    scale = 1.0f / sqrtf(ss * inv_width + eps);
+  }
+  for (int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; r < mpad; r += static_cast<int64_t>(gridDim.x) * kBlock) {
+    const acc_t a = __ldcg(acc + tok * mpad + r);
+    acc[tok * mpad + r] = 0;
+    if (r < rows) y[tok * rows + r] = scale * acc_value(a);
+  }
+}
+
+// out[t][r] = h[t][r] + value(acc[t * mpad + r]) (same expression as the staging step of the GEMV,
+// so a window boundary changes no bits); clears the accumulator behind the read, and zero0.
+__global__ void finish_residual_kernel(acc_t* __restrict__ acc, int64_t mpad, int64_t rows, int n_tok, const float* __restrict__ h,
+                                       float* __restrict__ out, acc_t* __restrict__ zero0, int64_t zero0_n) {
+  pdl_trigger();
+  pdl_wait();
+  const int tok = blockIdx.y;
+  for (int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; r < mpad; r += static_cast<int64_t>(gridDim.x) * kBlock) {
+    const acc_t a = __ldcg(acc + tok * mpad + r);
+    acc[tok * mpad + r] = 0;
+    if (r < rows) out[tok * rows + r] = h[tok * rows + r] + acc_value(a);
+  }
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * gridDim.y * kBlock;
+  for (int64_t i = (static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x) * kBlock + threadIdx.x; i < zero0_n; i += stride) zero0[i] = 0;
 }
 
 __global__ void rope_table_kernel(float2* __restrict__ tab, int pos, int n_tok, double theta) {
@@ -127,10 +151,17 @@ int launch_finish_plain(const float* part, int64_t n_parts, int64_t mpad, int64_
   return done(1);
 }
 
-int launch_finish_residual(const float* part, int64_t n_parts, int64_t mpad, int64_t rows, int n_tok, const float* h, float* out,
+int launch_finish_acc(acc_t* acc, int64_t mpad, int64_t rows, int n_tok, float* y, const SumSq& ssq, cudaStream_t st) {
+  dim3 grid(static_cast<unsigned>(std::min<int64_t>(1024, (mpad + kBlock - 1) / kBlock)), n_tok);
+  launch_pdl(finish_acc_kernel, grid, dim3(kBlock), 0, st, acc, mpad, rows, n_tok, y, static_cast<const float*>(ssq.data), ssq.n_groups,
+             ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps);
+  return done(1);
+}
+
+int launch_finish_residual(acc_t* acc, int64_t mpad, int64_t rows, int n_tok, const float* h, float* out, acc_t* zero0, int64_t zero0_n,
                            cudaStream_t st) {
-  dim3 grid(static_cast<unsigned>(std::min<int64_t>(1024, (rows + kBlock - 1) / kBlock)), n_tok);
-  launch_pdl(finish_residual_kernel, grid, dim3(kBlock), 0, st, part, n_parts, mpad, rows, n_tok, h, out);
+  dim3 grid(static_cast<unsigned>(std::min<int64_t>(1024, (mpad + kBlock - 1) / kBlock)), n_tok);
+  launch_pdl(finish_residual_kernel, grid, dim3(kBlock), 0, st, acc, mpad, rows, n_tok, h, out, zero0, zero0_n);
   return done(1);
 }
 

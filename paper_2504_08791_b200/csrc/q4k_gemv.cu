@@ -38,9 +38,10 @@
 //
 // Output.  A lane's four tile partials of a batch are reduced over the quad with a transposing
 // shuffle (lane t ends with tile t's row sum), the SG warps of the CTA add theirs through shared
-// memory in warp order (one barrier per batch, double-buffered), giving one partial per (column
-// group, row, token):  part[(group * n_tok + tok) * mpad + row].  The finisher kernels (finish.cu)
-// add the groups in ascending order.  No atomics: the bits do not depend on scheduling.
+// memory in warp order (one barrier per batch, double-buffered), giving one partial sum per (column
+// group, row, token), which is added into the row's 64-bit fixed-point accumulator
+// acc[tok * mpad + row] with an integer atomic (see common.cuh): the sum over the column groups is
+// exact in the integers, so the bits do not depend on the order in which CTAs arrive.
 #include <cstdlib>
 
 #include "common.cuh"
@@ -247,8 +248,7 @@ struct GemvParams {
   const float* x;
   const float* h_in;
   float* h_out;
-  const float* part_in;
-  int n_parts_in;
+  const acc_t* acc_in;
   int64_t mpad_in;
   const float* gain;
   float* ssq_out;
@@ -256,79 +256,79 @@ struct GemvParams {
   int n_ssq_in;
   float inv_width_in, eps_in;
   int tok0, n_tok_total;
-  float* part;
+  acc_t* acc;
   int64_t mpad;
+  acc_t* zero0;
+  int64_t zero0_n;
+  acc_t* zero1;
+  int64_t zero1_n;
   int* status;
 };
 
-// RMSNorm factor of one token from per-group sums of squares, groups added in ascending order.
-__device__ __forceinline__ float inv_rms(const float* __restrict__ ssq, int n_groups, int tok, float inv_width, float eps) {
-  float ss = 0.f;
-  for (int gidx = 0; gidx < n_groups; ++gidx) ss += ssq[tok * kMaxStatBlocks + gidx];
-  return 1.0f / sqrtf(ss * inv_width + eps);
-}
-
-// Sum of n float4 partial sums at base + p * stride, p ascending.  Loads are issued eight at a time
-// so that their latencies overlap; the additions keep the ascending order.
-__device__ __forceinline__ float4 sum_parts4(const float* __restrict__ base, int64_t stride, int n) {
-  float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-  int p = 0;
-  for (; p + 8 <= n; p += 8) {
-    float4 a[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) a[i] = *reinterpret_cast<const float4*>(base + (p + i) * stride);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      sum.x += a[i].x; sum.y += a[i].y; sum.z += a[i].z; sum.w += a[i].w;
-    }
-  }
-  float4 a[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-    if (p + i < n) a[i] = *reinterpret_cast<const float4*>(base + (p + i) * stride);
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-    if (p + i < n) {
-      sum.x += a[i].x; sum.y += a[i].y; sum.z += a[i].z; sum.w += a[i].w;
-    }
-  return sum;
-}
+// Loads of what another kernel wrote go to L2 directly.
+__device__ __forceinline__ float4 ld_l2(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ ulonglong2 ld_l2(const acc_t* p) { return __ldcg(reinterpret_cast<const ulonglong2*>(p)); }
 
 // A warp stages the 256 activations of its column s for NTOK tokens in registers, finishing the
-// producer's output on the way; lane l owns columns 8l .. 8l+7 (v[k][0..7]).  ss[k] receives the lane's share of the sum of squares (kResidual).
+// producer's output on the way; lane l owns columns 8l .. 8l+7 (v[k][0..7]).  ss[k] receives the
+// lane's share of the sum of squares (kResidual).  This step sits on the critical path between two
+// products and a round trip to L2 takes about a microsecond, so every load of a token is issued
+// before any is used.
 template <int NTOK>
 __device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float (&v)[NTOK][8], float (&ss)[NTOK]) {
   const int lane = threadIdx.x & 31;
   const int64_t cols = static_cast<int64_t>(P.n_sb) * 256;
   const int64_t k0 = static_cast<int64_t>(s) * 256 + 8 * lane;
-  const int64_t pstride = static_cast<int64_t>(P.n_tok_total) * P.mpad_in;
 #pragma unroll
   for (int k = 0; k < NTOK; ++k) {
     const int64_t row = static_cast<int64_t>(P.tok0 + k);
-    float* dst = v[k];
     ss[k] = 0.f;
     if (P.kind == kPlain) {
-      *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(P.x + row * cols + k0);
-      *reinterpret_cast<float4*>(dst + 4) = *reinterpret_cast<const float4*>(P.x + row * cols + k0 + 4);
+      const float4 a = ld_l2(P.x + row * cols + k0), b = ld_l2(P.x + row * cols + k0 + 4);
+      v[k][0] = a.x; v[k][1] = a.y; v[k][2] = a.z; v[k][3] = a.w;
+      v[k][4] = b.x; v[k][5] = b.y; v[k][6] = b.z; v[k][7] = b.w;
     } else if (P.kind == kResidual) {
+      const float4 h0 = ld_l2(P.h_in + row * cols + k0), h1 = ld_l2(P.h_in + row * cols + k0 + 4);
+      const float4 g0 = __ldg(reinterpret_cast<const float4*>(P.gain + k0)), g1 = __ldg(reinterpret_cast<const float4*>(P.gain + k0 + 4));
+      float r[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+      if (P.acc_in) {
+        const acc_t* ain = P.acc_in + row * P.mpad_in + k0;
+        ulonglong2 a[4];
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        const int64_t kk = k0 + 4 * hf;
-        const float4 sum = sum_parts4(P.part_in + row * P.mpad_in + kk, pstride, P.n_parts_in);
-        const float4 h = *reinterpret_cast<const float4*>(P.h_in + row * cols + kk);
-        const float4 v = make_float4(h.x + sum.x, h.y + sum.y, h.z + sum.z, h.w + sum.w);
-        *reinterpret_cast<float4*>(P.h_out + row * cols + kk) = v;
-        ss[k] += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
-        const float4 gv = *reinterpret_cast<const float4*>(P.gain + kk);
-        *reinterpret_cast<float4*>(dst + 4 * hf) = make_float4(v.x * gv.x, v.y * gv.y, v.z * gv.z, v.w * gv.w);
+        for (int i = 0; i < 4; ++i) a[i] = ld_l2(ain + 2 * i);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          r[2 * i] += acc_value(a[i].x);
+          r[2 * i + 1] += acc_value(a[i].y);
+        }
       }
-    } else {   // kSwiglu: the previous product's fused rows 2k (gate) and 2k+1 (up)
-      const float inv = inv_rms(P.ssq_in, P.n_ssq_in, P.tok0 + k, P.inv_width_in, P.eps_in);
+      *reinterpret_cast<float4*>(P.h_out + row * cols + k0) = make_float4(r[0], r[1], r[2], r[3]);
+      *reinterpret_cast<float4*>(P.h_out + row * cols + k0 + 4) = make_float4(r[4], r[5], r[6], r[7]);
+      ss[k] = ((r[0] * r[0] + r[1] * r[1]) + (r[2] * r[2] + r[3] * r[3])) + ((r[4] * r[4] + r[5] * r[5]) + (r[6] * r[6] + r[7] * r[7]));
+      const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float4 sum = sum_parts4(P.part_in + row * P.mpad_in + 2 * (k0 + 2 * q), pstride, P.n_parts_in);   // (G0, U0, G1, U1)
-        const float g0 = sum.x * inv, u0 = sum.y * inv, g1 = sum.z * inv, u1 = sum.w * inv;
-        *reinterpret_cast<float2*>(dst + 2 * q) = make_float2(g0 / (1.0f + expf(-g0)) * u0, g1 / (1.0f + expf(-g1)) * u1);
+      for (int i = 0; i < 8; ++i) v[k][i] = r[i] * gg[i];
+    } else {   // kSwiglu: the previous product's fused rows 2c (gate) and 2c+1 (up): 16 consecutive accumulators
+      const acc_t* ain = P.acc_in + row * P.mpad_in + 2 * k0;
+      ulonglong2 a[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] = ld_l2(ain + 2 * i);
+      float ssq = 0.f;
+      const float* sp = P.ssq_in + (P.tok0 + k) * kMaxStatBlocks;
+      for (int g0 = 0; g0 < P.n_ssq_in; g0 += 8) {     // groups added in ascending order
+        float sq[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (g0 + i < P.n_ssq_in) sq[i] = __ldcg(sp + g0 + i);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (g0 + i < P.n_ssq_in) ssq += sq[i];
+      }
+      const float inv = 1.0f / sqrtf(ssq * P.inv_width_in + P.eps_in);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float gt = acc_value(a[i].x) * inv, up = acc_value(a[i].y) * inv;
+        v[k][i] = gt / (1.0f + expf(-gt)) * up;
       }
     }
   }
@@ -388,8 +388,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   // [2][NTOK][kMaxWarps][kBatch][8], a small scratch for the sums of squares
   const int n_warps = blockDim.x >> 5;
   const uint8_t* __restrict__ w = P.w;
-  const int n_rt = P.n_rt, n_sb = P.n_sb, sg = P.sg, tok0 = P.tok0, n_tok_total = P.n_tok_total;
-  float* __restrict__ part = P.part;
+  const int n_rt = P.n_rt, n_sb = P.n_sb, sg = P.sg, tok0 = P.tok0;
+  acc_t* __restrict__ acc_out = P.acc;
   const int64_t mpad = P.mpad;
   int* __restrict__ status = P.status;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(n_warps) * kRing * kBatchBytes);
@@ -405,18 +405,30 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   // waits for); otherwise the positions are cut evenly.
   const int n_groups = n_sb / sg;
   const int n_pos = n_groups * n_rt;
-  int p0, p1;
+  int p0 = 0, p1 = 0;
   const int per_group = gridDim.x / n_groups;
   if (per_group >= 1) {
     const int grp = blockIdx.x / per_group, i = blockIdx.x - grp * per_group;
-    if (grp >= n_groups) return;
-    p0 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * i / per_group);
-    p1 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * (i + 1) / per_group);
+    if (grp < n_groups) {
+      p0 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * i / per_group);
+      p1 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * (i + 1) / per_group);
+    }
   } else {
     p0 = static_cast<int>(static_cast<int64_t>(n_pos) * blockIdx.x / gridDim.x);
     p1 = static_cast<int>(static_cast<int64_t>(n_pos) * (blockIdx.x + 1) / gridDim.x);
   }
-  if (p0 >= p1) return;
+  // Every CTA of the grid, also one without positions, clears its share of the accumulator arrays
+  // whose readers are done once the predecessor kernel is.
+  auto clear_arrays = [&]() {
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < P.zero0_n; i += stride) P.zero0[i] = 0;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < P.zero1_n; i += stride) P.zero1[i] = 0;
+  };
+  if (p0 >= p1) {
+    pdl_wait();
+    clear_arrays();
+    return;
+  }
 
   const uint8_t* my_ring = smem + static_cast<size_t>(warp) * kRing * kBatchBytes;
   const uint32_t ring_u32 = smem_addr(my_ring);
@@ -467,6 +479,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     if (!waited) {      // the first weight batches are on their way; everything below depends on the predecessor kernel
       pdl_wait();
       waited = true;
+      clear_arrays();
     }
     {
       float v[NTOK][8];
@@ -554,7 +567,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
         const float* src = red + ((parity * NTOK + k) * kMaxWarps * kBatch + i) * kRowsPerTile + row;
         float sum = src[0];
         for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile];
-        part[(static_cast<int64_t>(cur.grp) * n_tok_total + tok0 + k) * mpad + (cur.rt + i) * kRowsPerTile + row] = sum;
+        if (!(fabsf(sum) < kAccLimit)) atomicExch(status, 2);
+        atomicAdd(acc_out + static_cast<int64_t>(tok0 + k) * mpad + (cur.rt + i) * kRowsPerTile + row, acc_from(sum));
       }
     }
     parity ^= 1;
@@ -614,7 +628,7 @@ bool gemv_uses_tensor_cores() {
   return mma;
 }
 
-int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, float* part, int sm_count, cudaStream_t st) {
+int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, int sm_count, cudaStream_t st) {
   if (w.n_rt == 0 || w.n_sb == 0) return 0;
   if (w.n_rt * w.n_sb >= (int64_t(1) << 31)) return cuda_rc(cudaErrorInvalidValue);
   const int sg = gemv_group_size(w.n_sb);
@@ -623,11 +637,12 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, float* part, 
   in.ssq_out.width = w.cols;
   GemvParams P;
   P.w = w.data; P.n_rt = static_cast<int>(w.n_rt); P.n_sb = static_cast<int>(w.n_sb); P.sg = sg;
-  P.kind = in.kind; P.x = in.x; P.h_in = in.h_in; P.h_out = in.h_out; P.part_in = in.part_in; P.n_parts_in = in.n_parts_in;
+  P.kind = in.kind; P.x = in.x; P.h_in = in.h_in; P.h_out = in.h_out; P.acc_in = in.acc_in;
   P.mpad_in = in.mpad_in; P.gain = in.gain; P.ssq_out = in.ssq_out.data; P.ssq_in = in.ssq_in.data; P.n_ssq_in = in.ssq_in.n_groups;
   P.inv_width_in = in.ssq_in.width > 0 ? 1.0f / static_cast<float>(in.ssq_in.width) : 0.f;
   P.eps_in = in.ssq_in.eps;
-  P.n_tok_total = n_tok; P.part = part; P.mpad = w.mpad(); P.status = in.status;
+  P.n_tok_total = n_tok; P.acc = acc; P.mpad = w.mpad(); P.status = in.status;
+  P.zero0 = in.zero0; P.zero0_n = in.zero0_n; P.zero1 = in.zero1; P.zero1_n = in.zero1_n;
   int launches = 0;
   int tok = 0;
   while (tok < n_tok) {
@@ -640,6 +655,7 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, float* part, 
     P.tok0 = tok;
     const cudaError_t e = gemv_uses_tensor_cores() ? launch_n<true>(chunk, P, grid, st) : launch_n<false>(chunk, P, grid, st);
     if (e != cudaSuccess) return cuda_rc(e);
+    P.zero0_n = P.zero1_n = 0;   // cleared by the first pass
     ++launches;
     tok += chunk;
   }
