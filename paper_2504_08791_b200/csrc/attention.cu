@@ -64,7 +64,7 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
                     float2* __restrict__ ml_part) {
   pdl_trigger();
   extern __shared__ __align__(16) float dyn_smem[];
-  __shared__ float s_m[kWarps][16], s_l[kWarps][16];
+  __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
   __shared__ float s_inv[kMaxTok];
 
   const int group = n_q_heads / n_kv_heads;
@@ -319,28 +319,36 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
         s_l[warp][g + 8] = lsum[1];
       }
       __syncthreads();
-      // ---- combine the warps: each group of 128 threads takes every (kThreads/128)-th row of the
-      //      tile, thread d of the group owning head dim d
-      {
-        const int d = threadIdx.x % kHeadDim;
-        const int col = swz(d);
-        for (int r = threadIdx.x / kHeadDim; r < 16 && tile * 16 + r < n_rows; r += kThreads / kHeadDim) {
-          float big = -INFINITY;
+      // ---- combine the warps.  First the factors e^(m_w - M) of every (warp, row), one thread each;
+      //      then thread (row, group of 4 head dims) adds up its 16 bytes of the eight tiles.
+      const int live_rows = min(16, n_rows - tile * 16);
+      if (threadIdx.x < kWarps * 16) {
+        const int w = threadIdx.x >> 4, r = threadIdx.x & 15;
+        float big = -INFINITY;
 #pragma unroll
-          for (int w = 0; w < kWarps; ++w) big = fmaxf(big, s_m[w][r]);
-          float l = 0.f, accum = 0.f;
+        for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
+        const float mine = s_m[w][r];
+        s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
+        if (w == 0) s_big[r] = big;
+      }
+      __syncthreads();
+      for (int idx = threadIdx.x; idx < live_rows * (kHeadDim / 4); idx += kThreads) {
+        const int r = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
+        const int col = swz(d4);
+        float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l = 0.f;
 #pragma unroll
-          for (int w = 0; w < kWarps; ++w) {
-            const float f = s_m[w][r] > -INFINITY ? expf(s_m[w][r] - big) : 0.f;
-            l += f * s_l[w][r];
-            accum += f * s_o[(w * o_rows + r) * kRowPad + col];
-          }
-          const int rr = tile * 16 + r;
-          const int tok = rr / group, head = kv * group + rr % group;
-          const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * n_chunks + chunk;
-          o_part[slot * kHeadDim + d] = accum;
-          if (d == 0) ml_part[slot] = make_float2(big, l);
+        for (int w = 0; w < kWarps; ++w) {
+          const float f = s_f[w][r];
+          const float4 v = *reinterpret_cast<const float4*>(s_o + (w * o_rows + r) * kRowPad + col);
+          l += f * s_l[w][r];
+          accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
         }
+        const int rr = tile * 16 + r;
+        const int tok = rr / group, head = kv * group + rr % group;
+        const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * n_chunks + chunk;
+        *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
+        if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
       }
       __syncthreads();
     }
@@ -365,15 +373,16 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
 #pragma unroll
   for (int c = 0; c < kMergePre; ++c)
     if (c < n_chunks) pre[c] = __ldcg(op + static_cast<int64_t>(c) * kHeadDim);
-  float big = -INFINITY;
-  for (int c = d; c < n_chunks; c += kHeadDim) big = fmaxf(big, __ldcg(ml + c).x);
+  const float2 ml0 = d < n_chunks ? __ldcg(ml + d) : make_float2(-INFINITY, 0.f);      // this thread's first chunk
+  float big = ml0.x;
+  for (int c = d + kHeadDim; c < n_chunks; c += kHeadDim) big = fmaxf(big, __ldcg(ml + c).x);
 #pragma unroll
   for (int of = 16; of > 0; of >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, of));
   if ((d & 31) == 0) s_red[d >> 5] = big;
   __syncthreads();
   big = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
   for (int c = d; c < n_chunks; c += kHeadDim) {
-    const float2 v = __ldcg(ml + c);
+    const float2 v = c == d ? ml0 : __ldcg(ml + c);
     const float w = v.x > -INFINITY ? expf(v.x - big) : 0.f;
     s_w[c] = w;
     s_wl[c] = w * v.y;
@@ -381,6 +390,7 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
   __syncthreads();
   // every thread forms the same denominator in chunk order
   float denom = 0.f;
+#pragma unroll 8
   for (int c = 0; c < n_chunks; ++c) denom += s_wl[c];
   float accum = 0.f;
 #pragma unroll

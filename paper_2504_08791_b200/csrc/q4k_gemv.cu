@@ -408,8 +408,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   int p0 = 0, p1 = 0;
   const int per_group = gridDim.x / n_groups;
   if (per_group >= 1) {
-    const int grp = blockIdx.x / per_group, i = blockIdx.x - grp * per_group;
-    if (grp < n_groups) {
+    // CTAs of one group are spread evenly over the launch order (CTA b works for group b mod
+    // n_groups): CTAs that start later, or share an SM with an older CTA, run a little slower, and
+    // every group should get the same mix of them.
+    const int grp = blockIdx.x % n_groups, i = blockIdx.x / n_groups;
+    if (i < per_group) {
       p0 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * i / per_group);
       p1 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * (i + 1) / per_group);
     }
