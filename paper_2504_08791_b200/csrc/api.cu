@@ -413,16 +413,17 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
     in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status;
     in_o.zero0 = c->acc_qkv; in_o.zero0_n = static_cast<int64_t>(n_tok) * L.qkv.mpad();
     in_o.zero1 = c->acc_down; in_o.zero1_n = static_cast<int64_t>(n_tok) * mpad_e;
+    in_o.out_order = kOrderResidual;
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->acc_o, c->sm_count, st), "gemv(o)");
     GemvIn in_f;                                 // gate/up: h_b + O projection -> h_a
     in_f.kind = kResidual; in_f.h_in = c->h_b; in_f.h_out = c->h_a; in_f.acc_in = c->acc_o; in_f.mpad_in = L.o.mpad();
-    in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status;
+    in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status; in_f.out_order = kOrderSwiglu;
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->acc_gu, c->sm_count, st), "gemv(gate/up)");
     c->ssq_ffn = in_f.ssq_out;
     c->ssq_ffn.eps = g.rms_eps;
     GemvIn in_d;                                 // down: SwiGLU of the gate/up product
     in_d.kind = kSwiglu; in_d.acc_in = c->acc_gu; in_d.mpad_in = L.gu.mpad();
-    in_d.ssq_in = c->ssq_ffn; in_d.status = c->status;
+    in_d.ssq_in = c->ssq_ffn; in_d.status = c->status; in_d.out_order = kOrderResidual;
     in_d.zero0 = c->acc_o; in_d.zero0_n = static_cast<int64_t>(n_tok) * L.o.mpad();
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->acc_down, c->sm_count, st), "gemv(down)");
     h_in = c->h_a;

@@ -105,7 +105,18 @@ bool gemv_uses_tensor_cores();
 //             the previous (gate/up) product, inv from ssq_in
 // After its dependency wait the kernel also clears the accumulator arrays zero0 / zero1 (arrays
 // whose last reader was the predecessor kernel or an earlier one).
+//
+// Order of the accumulators inside a token's mpad words (GemvIn.out_order of the producer): a
+// consumer's lane owns 8 consecutive columns, and with the plain order its 16-byte loads would each
+// touch a different 128-byte line.  The producer therefore stores in the order in which the
+// consumer's warp reads, so that every load instruction of the warp covers 512 contiguous bytes:
+//   kOrderRows      element r at r (read by the attention and output finishers)
+//   kOrderResidual  for a kResidual consumer: inside every block of 256 rows, the pair of rows
+//                   (2p, 2p+1) sits at pair position 32 (p % 4) + p / 4
+//   kOrderSwiglu    for a kSwiglu consumer: inside every block of 512 fused rows (256 columns), the
+//                   (gate, up) pair of column w sits at pair position 32 (w % 8) + w / 8
 enum GemvKind { kPlain = 0, kResidual = 1, kSwiglu = 2 };
+enum AccOrder { kOrderRows = 0, kOrderResidual = 1, kOrderSwiglu = 2 };
 struct GemvIn {
   int kind = kPlain;
   const float* x = nullptr;        // kPlain: [n_tok][cols]
@@ -116,6 +127,7 @@ struct GemvIn {
   const float* gain = nullptr;     // kResidual: [cols]
   SumSq ssq_out;                   // kResidual: written (n_groups is set by the launcher)
   SumSq ssq_in;                    // kSwiglu: read
+  int out_order = kOrderRows;      // order of the accumulators this product leaves (padded rows a multiple of 256 / 512 for kOrderResidual / kOrderSwiglu)
   acc_t* zero0 = nullptr;          // accumulator arrays to clear, with their lengths
   int64_t zero0_n = 0;
   acc_t* zero1 = nullptr;
@@ -127,8 +139,8 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
 // y[t][r] = scale_t * value(acc[t * mpad + r]), scale_t = the RMSNorm factor from ssq when
 // ssq.data != nullptr, else 1; every accumulator is cleared after it has been read.
 int launch_finish_acc(acc_t* acc, int64_t mpad, int64_t rows, int n_tok, float* y, const SumSq& ssq, cudaStream_t st);
-// out[t][r] = h[t][r] + value(acc[t * mpad + r]) (the residual stream leaving a window); clears acc
-// behind the read and the array zero0.
+// out[t][r] = h[t][r] + value of row r's accumulator, stored in kOrderResidual (the residual stream
+// leaving a window); clears acc behind the read and the array zero0.
 int launch_finish_residual(acc_t* acc, int64_t mpad, int64_t rows, int n_tok, const float* h, float* out, acc_t* zero0, int64_t zero0_n,
                            cudaStream_t st);
 
@@ -173,6 +185,18 @@ inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? 0 : -static_cast<i
 // does before pdl_wait() (set-up, prefetching immutable weights) overlaps the predecessor's tail.
 #ifdef __CUDACC__
 __device__ __forceinline__ float acc_value(acc_t a) { return static_cast<float>(static_cast<long long>(a)) * kAccInvScale; }
+// Position of row r (fused row for kOrderSwiglu) inside a token's accumulators.
+__device__ __forceinline__ int64_t acc_position(int order, int64_t r) {
+  if (order == kOrderResidual) {
+    const int64_t p = (r & 255) >> 1;
+    return (r & ~int64_t(255)) + 2 * (32 * (p & 3) + (p >> 2)) + (r & 1);
+  }
+  if (order == kOrderSwiglu) {
+    const int64_t w = (r >> 1) & 255;
+    return (r & ~int64_t(511)) + 2 * (32 * (w & 7) + (w >> 3)) + (r & 1);
+  }
+  return r;
+}
 __device__ __forceinline__ acc_t acc_from(float v) { return static_cast<acc_t>(__float2ll_rn(v * kAccScale)); }
 
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

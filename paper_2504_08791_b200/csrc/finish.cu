@@ -59,8 +59,9 @@ __global__ void finish_residual_kernel(acc_t* __restrict__ acc, int64_t mpad, in
   pdl_wait();
   const int tok = blockIdx.y;
   for (int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; r < mpad; r += static_cast<int64_t>(gridDim.x) * kBlock) {
-    const acc_t a = __ldcg(acc + tok * mpad + r);
-    acc[tok * mpad + r] = 0;
+    const int64_t at = tok * mpad + acc_position(kOrderResidual, r);
+    const acc_t a = __ldcg(acc + at);
+    acc[at] = 0;
     if (r < rows) out[tok * rows + r] = h[tok * rows + r] + acc_value(a);
   }
   const int64_t stride = static_cast<int64_t>(gridDim.x) * gridDim.y * kBlock;

@@ -262,6 +262,7 @@ struct GemvParams {
   int64_t zero0_n;
   acc_t* zero1;
   int64_t zero1_n;
+  int out_order;
   int* status;
 };
 
@@ -292,10 +293,10 @@ __device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float (&v
       const float4 g0 = __ldg(reinterpret_cast<const float4*>(P.gain + k0)), g1 = __ldg(reinterpret_cast<const float4*>(P.gain + k0 + 4));
       float r[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
       if (P.acc_in) {
-        const acc_t* ain = P.acc_in + row * P.mpad_in + k0;
+        const acc_t* ain = P.acc_in + row * P.mpad_in + static_cast<int64_t>(s) * 256;   // kOrderResidual
         ulonglong2 a[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a[i] = ld_l2(ain + 2 * i);
+        for (int i = 0; i < 4; ++i) a[i] = ld_l2(ain + 2 * (32 * i + lane));
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           r[2 * i] += acc_value(a[i].x);
@@ -309,10 +310,10 @@ __device__ __forceinline__ void stage_warp(const GemvParams& P, int s, float (&v
 #pragma unroll
       for (int i = 0; i < 8; ++i) v[k][i] = r[i] * gg[i];
     } else {   // kSwiglu: the previous product's fused rows 2c (gate) and 2c+1 (up): 16 consecutive accumulators
-      const acc_t* ain = P.acc_in + row * P.mpad_in + 2 * k0;
+      const acc_t* ain = P.acc_in + row * P.mpad_in + static_cast<int64_t>(s) * 512;   // kOrderSwiglu
       ulonglong2 a[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) a[i] = ld_l2(ain + 2 * i);
+      for (int i = 0; i < 8; ++i) a[i] = ld_l2(ain + 2 * (32 * i + lane));
       float ssq = 0.f;
       const float* sp = P.ssq_in + (P.tok0 + k) * kMaxStatBlocks;
       for (int g0 = 0; g0 < P.n_ssq_in; g0 += 8) {     // groups added in ascending order
@@ -571,7 +572,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
         float sum = src[0];
         for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile];
         if (!(fabsf(sum) < kAccLimit)) atomicExch(status, 2);
-        atomicAdd(acc_out + static_cast<int64_t>(tok0 + k) * mpad + (cur.rt + i) * kRowsPerTile + row, acc_from(sum));
+        atomicAdd(acc_out + static_cast<int64_t>(tok0 + k) * mpad + acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row), acc_from(sum));
       }
     }
     parity ^= 1;
@@ -646,6 +647,8 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
   P.eps_in = in.ssq_in.eps;
   P.n_tok_total = n_tok; P.acc = acc; P.mpad = w.mpad(); P.status = in.status;
   P.zero0 = in.zero0; P.zero0_n = in.zero0_n; P.zero1 = in.zero1; P.zero1_n = in.zero1_n;
+  P.out_order = in.out_order;
+  if ((in.out_order == kOrderResidual && w.mpad() % 256 != 0) || (in.out_order == kOrderSwiglu && w.mpad() % 512 != 0)) return cuda_rc(cudaErrorInvalidValue);
   int launches = 0;
   int tok = 0;
   while (tok < n_tok) {
