@@ -6,7 +6,10 @@ the model, issued as contiguous layer windows (4 windows of 20 layers for the 70
 paper's ring schedule with window 20), then through the output layer.  Weights are synthetic
 random-init Q4_K tensors of the named shape; the KV cache is prefilled with N(0,1) fp16 entries.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 70b|32b|8b] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 70b|32b|8b] [--n-tok T] [--impl ours|reference]
+
+With --n-tok T > 1 a step is one verification pass of speculative decoding: T tokens at consecutive
+positions go through the model together (causal among themselves) and the time is reported per step.
 
 With N > 1 (launched by torch.distributed.run) every rank decodes its own request on its own
 GPU: the path does not shard, ranks are independent replicas and no collective is on the data
@@ -162,28 +165,30 @@ def run_ours(args, rank, world, local_rank):
     cfg = synth.model_config(shape)
     if args.layers:
         cfg["n_layers"] = args.layers
+    cfg["kv_capacity"] = max(cfg["kv_capacity"], n_ctx + 64 * args.n_tok)
     L = cfg["n_layers"]
     seed = SEEDS[args.workload] + 1000 * rank
     ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank)
     bpt = bytes_per_token(cfg, n_ctx)
     bounds = [L * i // n_windows for i in range(n_windows + 1)]
 
-    h0 = torch.from_numpy(synth.activations(seed, 1, cfg["hidden"])).cuda()
+    T = args.n_tok
+    h0 = torch.from_numpy(synth.activations(seed, T, cfg["hidden"])).cuda()
     hid = torch.empty_like(h0)
-    logits = torch.empty((1, cfg["vocab"]), dtype=torch.float32, device="cuda")
+    logits = torch.empty((T, cfg["vocab"]), dtype=torch.float32, device="cuda")
 
     def device_step(pos):
         hid.copy_(h0)
         for w in range(n_windows):
-            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, 1)
-        ctx.logits(hid, 1, logits)
+            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, T)
+        ctx.logits(hid, T, logits)
 
     def e2e_step(tok, pos):
-        ctx.embed([tok], hid)                      # host token id -> device (4 bytes)
+        ctx.embed([tok] * T, hid)                  # host token ids -> device (4 bytes each)
         for w in range(n_windows):
-            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, 1)
-        ctx.logits(hid, 1, logits)
-        return int(ctx.argmax(logits, 1)[0])       # device -> host (4 bytes), waits
+            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, T)
+        ctx.logits(hid, T, logits)
+        return int(ctx.argmax(logits, T)[T - 1])   # device -> host (4 bytes each), waits
 
     def barrier():
         torch.cuda.synchronize()
@@ -213,14 +218,14 @@ def run_ours(args, rank, world, local_rank):
     # end to end through the ABI: host token in, host token out, every step
     tok = 0
     for i in range(min(args.warmup, 3)):
-        tok = e2e_step(tok, n_ctx + i)
+        tok = e2e_step(tok, n_ctx + i * T)
     barrier()
-    e2e_steps = min(args.steps, cfg["kv_capacity"] - n_ctx - 3)
+    e2e_steps = min(args.steps, (cfg["kv_capacity"] - n_ctx - 3 * T) // T)
     ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.perf_counter()
     ev2.record()
     for i in range(e2e_steps):
-        tok = e2e_step(tok, n_ctx + 3 + i)
+        tok = e2e_step(tok, n_ctx + (3 + i) * T)
     ev3.record()
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - wall0) * 1e3
@@ -257,17 +262,18 @@ def run_ours(args, rank, world, local_rank):
         "dtype": "q4_k weights x int16 activations, int32/fp32 accumulate",
         "data": "synthetic",
         "tokens_per_s": job_value(ms_step, world)["tokens_per_s"],
-        "config": {"workload": desc, "layers": L, "windows": n_windows, "n_ctx": n_ctx, "n_tok": 1,
+        "config": {"workload": desc, "layers": L, "windows": n_windows, "n_ctx": n_ctx, "n_tok": T,
+                   "value_is": "ms per decoded token" if T == 1 else "ms per verification step of %d tokens" % T,
                    "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs larger than L2 (>= 4.9 GB per step)",
                    "bytes_per_token": bpt["total"]},
         "step_roofline": {"bound": "hbm", "achieved": step_gbs, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                           "frac": step_gbs / peak, "frac_of_nominal_8000": step_gbs / 8000.0},
-        "roofline": {"kernel": "gemv_partials_kernel<1>", "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
+        "roofline": {"kernel": "gemv_partials_kernel<%d>" % min(T, 4), "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
                      "unit": "GB/s", "frac": gemv_gbs / peak, "traffic": None,
                      "launches": g_n // prof_steps, "avg_launch_us": (g_ms * 1e3 / g_n) if g_n else None,
                      "timing": f"cuda events around each launch, separate pass of {prof_steps} steps"},
         "attention_kernel": {"achieved": attn_gbs, "unit": "GB/s", "frac": attn_gbs / peak, "launches": a_n // prof_steps},
-        "e2e": {"value": e2e_ms / world, "unit": "ms/token", "h2d_bytes_per_step": 4, "d2h_bytes_per_step": 4, "steps": e2e_steps},
+        "e2e": {"value": e2e_ms / world, "unit": "ms/token", "h2d_bytes_per_step": 4 * T, "d2h_bytes_per_step": 4 * T, "steps": e2e_steps},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -340,6 +346,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="70b", choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
+    ap.add_argument("--n-tok", type=int, default=1, help="tokens per step (speculative verification pass when > 1)")
     ap.add_argument("--ctx", type=int, default=0, help="override the KV context length (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
