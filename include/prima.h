@@ -117,7 +117,11 @@ int prima_load_q4k_weights(prima_ctx* ctx, int layer, int tensor_id, const void*
  * one step must be issued in ascending layer order; any split of the layer range into windows
  * gives bit-identical results.  Errors (no launch): a layer of the range is not fully loaded
  * (PRIMA_ERR_STATE); bad range, pos < 0, pos + n_tok > kv_capacity, n_tok outside 1..max_n_tok,
- * NULL pointers (PRIMA_ERR_ARG). */
+ * NULL pointers (PRIMA_ERR_ARG).
+ * Range: the products are summed in 64-bit fixed point with 32 fractional bits (order-independent,
+ * hence the bit-identical results); a partial sum of a projection beyond +-2^27 (1.3e8) raises the
+ * status word, which prima_sync reports as PRIMA_ERR_DEVICE (the outputs of that step are then
+ * invalid).  Contributions below 2^-33 in absolute value are rounded away. */
 int prima_forward_window(prima_ctx* ctx, int layer_begin, int layer_end, const float* hidden_in,
                          float* hidden_out, int pos, int n_tok);
 
@@ -138,7 +142,8 @@ int prima_argmax(prima_ctx* ctx, const float* logits, int n_tok, int32_t* tokens
 int prima_kv_load(prima_ctx* ctx, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v);
 int prima_kv_read(prima_ctx* ctx, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v);
 
-/* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word and
+/* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word (a
+ * partial sum outside the accumulator range, or a bounded wait inside a kernel that gave up) and
  * PRIMA_ERR_CUDA if the stream reports an error. */
 int prima_sync(prima_ctx* ctx);
 
@@ -172,6 +177,7 @@ int prima_dequant_q4k(const void* dev_blocks, int64_t n_superblocks, float* dev_
 /* y[c][r] = sum_k W[r][k] x[c][k] for c < n_cols (1..8).  dev_w: standard layout; dev_x: fp32
  * [n_cols x cols]; dev_y: fp32 [n_cols x rows].  Allocates and frees its own temporary buffers
  * (tiled copy of W and scratch) and waits for completion; meant for testing single projections.
+ * Returns PRIMA_ERR_DEVICE if a partial sum left the accumulator range (see prima_forward_window).
  * For timing, use prima_gemv_plan_* below. */
 int prima_gemv_q4k(const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols,
                    float* dev_y, void* stream);

@@ -543,7 +543,9 @@ int prima_sync(prima_ctx* c) {
   cudaError_t e = cudaMemcpyAsync(&status, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync");
-  if (status != 0) return fail(c, PRIMA_ERR_DEVICE, "a kernel raised the device status word: " + std::to_string(status));
+  if (status != 0)
+    return fail(c, PRIMA_ERR_DEVICE, status == 2 ? "a partial sum was outside the accumulator range (+-2^27); results of this step are invalid"
+                                                 : "a bounded wait inside a kernel gave up (status " + std::to_string(status) + ")");
   return PRIMA_OK;
 }
 
@@ -654,9 +656,14 @@ int prima_gemv_q4k(const void* dev_w, int64_t rows, int64_t cols, const float* d
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = prima_gemv_plan_run(p, dev_x, n_cols, dev_y, st);
   cudaError_t e = cudaStreamSynchronize(st);
+  int status = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&status, p->status, sizeof(int), cudaMemcpyDeviceToHost);
   prima_gemv_plan_destroy(p);
   if (rc != PRIMA_OK) return rc;
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "prima_gemv_q4k");
+  if (status != 0)
+    return fail(nullptr, PRIMA_ERR_DEVICE, status == 2 ? "prima_gemv_q4k: a partial sum is outside the accumulator range (+-2^27)"
+                                                       : "prima_gemv_q4k: a bounded wait inside the kernel gave up");
   return PRIMA_OK;
 }
 

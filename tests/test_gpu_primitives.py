@@ -119,6 +119,37 @@ def test_gemv_activation_scales_and_special_vectors(gpu):
     _check_rows(_gemv_gpu(gpu, w, rows, cols, x), want, s_abs)
 
 
+def test_gemv_several_tokens_with_outliers_and_mixed_scales(gpu):
+    # 5..8 columns go through the kernel that quantises a column's 256 activations with one step
+    rows, cols, n = 264, 2048, 6
+    w = synth.model_tensor(8, 0, synth.WQ, rows, cols)
+    x = synth.activations(8, n, cols)
+    x[1] *= 1e-4
+    x[2] *= 2e3
+    x[3, 5] = 700.0          # one large value in a block of small ones
+    x[4, 256:512] = 0.0      # an all-zero block
+    x[5] = np.abs(x[5])
+    want, s_abs = oracle.gemv_q4k(w, rows, cols, x)
+    got = _gemv_gpu(gpu, w, rows, cols, x)
+    _check_rows(got, want, s_abs)
+    # the same columns one by one (other kernel) agree within the same bound
+    for c in range(n):
+        one = _gemv_gpu(gpu, w, rows, cols, x[c:c + 1])
+        _check_rows(one, want[c:c + 1], s_abs[c:c + 1])
+
+
+def test_gemv_reports_sums_outside_the_accumulator_range(gpu):
+    torch, binding = gpu
+    w, x = synth.gemv_case(seed=3, rows=64, cols=2048)       # literal distribution: weights of mean +1.6
+    y = torch.zeros((1, 64), dtype=torch.float32, device="cuda")
+    binding.prima_gemv_q4k(_to_dev(torch, w), 64, 2048, _to_dev(torch, np.abs(x) * 1e3), 1, y)          # sums ~2.6e6: fine
+    with pytest.raises(binding.PrimaError) as err:
+        binding.prima_gemv_q4k(_to_dev(torch, w), 64, 2048, _to_dev(torch, np.abs(x) * 1e6), 1, y)      # sums ~2.6e9 > 2^27
+    assert err.value.code == binding.ERR_DEVICE
+    # the library stays usable
+    binding.prima_gemv_q4k(_to_dev(torch, w), 64, 2048, _to_dev(torch, x), 1, y)
+
+
 def test_gemv_run_to_run_bits_are_identical(gpu):
     w, x = synth.gemv_case(seed=2, rows=2048, cols=4096)
     a = _gemv_gpu(gpu, w, 2048, 4096, x)
