@@ -417,10 +417,15 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
   const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
   if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
   const int n_rows = n_tok * (n_q_heads / n_kv_heads);
-  cudaError_t e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(partial_smem_bytes(8 * kMaxTok, kMaxTok)));
-  if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-  if (e0 != cudaSuccess) return cuda_rc(e0);
+  static bool configured[kMaxDevices] = {};
+  int dev = -1;
+  if (first_launch_on_device(configured, &dev)) {
+    cudaError_t e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(partial_smem_bytes(8 * kMaxTok, kMaxTok)));
+    if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e0 != cudaSuccess) return cuda_rc(e0);
+    if (dev >= 0) configured[dev] = true;
+  }
   // Two CTAs fit on an SM: with more chunks than that, a CTA takes several (gridDim.x apart).
   const int per_head = std::max(1, 2 * sm_count / n_kv_heads);
   dim3 grid(std::min(n_chunks, per_head), n_kv_heads);

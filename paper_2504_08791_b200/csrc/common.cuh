@@ -177,6 +177,21 @@ constexpr int kArgmaxBlocks = 128;
 
 inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? 0 : -static_cast<int>(e); }
 
+// Function attributes (dynamic shared memory size, carve-out) are per device and do not change:
+// each launcher sets them the first time it runs on a device, not at every launch (a call costs the
+// host more than a microsecond, and with six launches per layer the host must stay ahead of the GPU).
+// `done` is the launcher's own table of kMaxDevices flags; returns true when the caller must set them.
+constexpr int kMaxDevices = 64;
+inline bool first_launch_on_device(bool (&done)[kMaxDevices], int* device_out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    *device_out = -1;
+    return true;
+  }
+  *device_out = dev;
+  return !done[dev];
+}
+
 // ---- programmatic dependent launch -------------------------------------------------------------
 // Every kernel of the forward pass is launched with programmatic stream serialisation: it may
 // start while its predecessor in the stream is still running.  A kernel calls pdl_trigger() first

@@ -933,8 +933,13 @@ size_t gemv_smem_bytes(int sg, int n_tok) {
 template <int NTOK, bool MMA>
 cudaError_t launch_one(const GemvParams& P, int64_t grid, cudaStream_t st) {
   auto kern = gemv_partials_kernel<NTOK, MMA>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_smem_bytes(kMaxWarps, NTOK)));
-  if (e != cudaSuccess) return e;
+  static bool configured[kMaxDevices] = {};
+  int dev = -1;
+  if (first_launch_on_device(configured, &dev)) {
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_smem_bytes(kMaxWarps, NTOK)));
+    if (e != cudaSuccess) return e;
+    if (dev >= 0) configured[dev] = true;
+  }
   return launch_pdl(kern, dim3(static_cast<unsigned>(grid)), dim3(P.sg * 32), gemv_smem_bytes(P.sg, NTOK), st, P);
 }
 
@@ -985,7 +990,13 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
     if (grid > n_pos) grid = n_pos;
     P.tok0 = 0;
     const size_t smem_bytes = gemv_tokens_smem_bytes(sg);
-    cudaError_t e = cudaFuncSetAttribute(gemv_tokens_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_tokens_smem_bytes(kMaxWarps)));
+    static bool configured[kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaSuccess;
+    if (first_launch_on_device(configured, &dev)) {
+      e = cudaFuncSetAttribute(gemv_tokens_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(gemv_tokens_smem_bytes(kMaxWarps)));
+      if (e == cudaSuccess && dev >= 0) configured[dev] = true;
+    }
     if (e == cudaSuccess) e = launch_pdl(gemv_tokens_kernel, dim3(static_cast<unsigned>(grid)), dim3(sg * 32), smem_bytes, st, P);
     if (e != cudaSuccess) return cuda_rc(e);
     return 1;
