@@ -603,17 +603,17 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
 // row tiles), B = the activations of that sub-block for 8 tokens, once with their high and once with
 // their low bytes.  The weights are read once for all tokens.  Same tiled matrix, same ring of bulk
 // copies and exact integer sums as the one-token kernel; what differs:
-//  * A lane owns (row g, sub-block t) and (row g, sub-block 4+t) of a tile, 16 bytes each, but the
-//    instruction wants from lane (g, t) bytes 4t..4t+3 of every sub-block of row g.  A 4x4 transpose
-//    of 32-bit words inside the lane quad (two exchanges) provides them; word t of a sub-block holds
-//    weights 8t..8t+7, whose even nibbles become k slots 4t..4t+3 and odd nibbles k slots 16+4t..+3.
+//  * A unit stores (row g, sub-block j) as one 16-byte piece, but the instruction wants from lane
+//    (g, t) bytes 4t..4t+3 of every sub-block of row g: exactly what a matrix load (ldmatrix) of the
+//    eight rows' pieces delivers.  Word t of a sub-block holds weights 8t..8t+7, whose even nibbles
+//    become k slots 4t..4t+3 and odd nibbles k slots 16+4t..+3.
 //  * Lane (g, t) supplies column g of B, i.e. token g: for each sub-block the four words (high/low
 //    bytes x even/odd weights) of its quarter t.  The quantised activations of a column go through
 //    shared memory once to reach the lanes in that arrangement.
 //  * The activations of a token are 16-bit integers with ONE step for the 256 values of the column,
 //    s = max|x| / 32639, so that the sums over the sub-blocks can stay in the integers:
 //        partial[row][tok] = s[tok] * (d * sum_j sc_j I_j  -  dmin * sum_j m_j sum(x_q)_j),
-//    I_j = 256 * high + low from the two instructions; sum_j sc_j I_j needs 64 bits.
+//    I_j = 256 * high + low from the two instructions (the high and low parts are summed apart).
 //  * The instruction leaves lane (g, t) the complete sums of rows g and g+8 for tokens 2t and 2t+1:
 //    no reduction over the quad.
 // Two CTAs of SG warps per SM, warp w on column group * SG + w as in the one-token kernel, ring of
@@ -623,17 +623,15 @@ constexpr int kRingTok = 2;
 constexpr int kTokCols = 8;   // columns of the instruction = tokens per pass
 static_assert(kTokCols * 32 * 16 + kTokCols * 8 * 4 + kTokCols * 4 <= kBatchBytes, "the activation buffer must fit a ring slot");
 
-// 4x4 transpose of 32-bit words over the lanes of a quad: lane t gives row t (q.x..q.w) and ends
-// with column t: word i = what lane i held in position t.
-__device__ __forceinline__ void quad_transpose(uint4& q, int t) {
-  const bool b0 = t & 1, b1 = t & 2;
-  uint32_t s0 = b0 ? q.x : q.y, s1 = b0 ? q.z : q.w;
-  uint32_t r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
-  if (b0) { q.x = r0; q.z = r1; } else { q.y = r0; q.w = r1; }
-  s0 = b1 ? q.x : q.z; s1 = b1 ? q.y : q.w;
-  r0 = __shfl_xor_sync(0xffffffffu, s0, 2); r1 = __shfl_xor_sync(0xffffffffu, s1, 2);
-  if (b1) { q.x = r0; q.y = r1; } else { q.z = r0; q.w = r1; }
+// Four 8x8 matrices of 16-bit elements from shared memory: lane l gives the address of row l % 8 of
+// matrix l / 8 (16 bytes each); lane (g, t) receives bytes 4t..4t+3 of row g of each matrix.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
 }
+
+// 256 * high + low as a float: the two 32-bit sums are each below 2^25 in magnitude, their combination
+// needs up to 33 bits, so it is formed in fp32 (relative error 2^-24, far below the other roundings).
+__device__ __forceinline__ float scaled_sum(int high, int low) { return fmaf(static_cast<float>(high), 256.0f, static_cast<float>(low)); }
 
 // The sixteen 6-bit fields of one header row: sc[j], m[j], j = 0..7 (see the unit layout).
 struct RowScales {
@@ -853,40 +851,41 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
         const uint8_t* u1 = u0 + kUnitBytes;
         const RowScales r0 = decode_row(*reinterpret_cast<const uint4*>(u0 + g * 16));
         const RowScales r1 = decode_row(*reinterpret_cast<const uint4*>(u1 + g * 16));
-        uint4 qa0 = *reinterpret_cast<const uint4*>(u0 + kUnitHdrBytes + lane * 16);
-        uint4 qa1 = *reinterpret_cast<const uint4*>(u1 + kUnitHdrBytes + lane * 16);
-        uint4 qb0 = *reinterpret_cast<const uint4*>(u0 + kUnitHdrBytes + 512 + lane * 16);
-        uint4 qb1 = *reinterpret_cast<const uint4*>(u1 + kUnitHdrBytes + 512 + lane * 16);
-        quad_transpose(qa0, t);
-        quad_transpose(qa1, t);
-        quad_transpose(qb0, t);
-        quad_transpose(qb1, t);
-        const uint32_t w0[8] = {qa0.x, qa0.y, qa0.z, qa0.w, qb0.x, qb0.y, qb0.z, qb0.w};   // tile 2 pr, sub-blocks 0..7
-        const uint32_t w1[8] = {qa1.x, qa1.y, qa1.z, qa1.w, qb1.x, qb1.y, qb1.z, qb1.w};   // tile 2 pr + 1
-        long long accT[4] = {0, 0, 0, 0};   // sum_j sc_j I_j        [row g / g+8][token 2t / 2t+1]
-        int accM[4] = {0, 0, 0, 0};         // sum_j m_j sum(x_q)_j
+        // word t of (row g, sub-block j), j = 0..7, for both tiles: four matrix loads, each of which
+        // reads the 16-byte pieces of rows 0..7 for four sub-blocks and hands lane (g, t) bytes 4t..4t+3
+        const uint32_t piece = static_cast<uint32_t>(kUnitHdrBytes + ((lane & 7) * 4 + (lane >> 3)) * 16);
+        const uint32_t a_u0 = smem_addr(u0) + piece, a_u1 = smem_addr(u1) + piece;
+        int accH[4] = {0, 0, 0, 0}, accL[4] = {0, 0, 0, 0};   // sum_j sc_j * (high, low sums)   [row g / g+8][token 2t / 2t+1]
+        int accM[4] = {0, 0, 0, 0};                           // sum_j m_j sum(x_q)_j
+        uint32_t w0[4], w1[4];   // sub-blocks 4 (j / 4) .. + 3 of tile 2 pr / 2 pr + 1
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
+          if ((j & 3) == 0) {
+            ldmatrix_x4(w0[0], w0[1], w0[2], w0[3], a_u0 + 512 * (j >> 2));
+            ldmatrix_x4(w1[0], w1[1], w1[2], w1[3], a_u1 + 512 * (j >> 2));
+          }
           int dh[4] = {0, 0, 0, 0}, dl[4] = {0, 0, 0, 0};
-          const uint32_t a0 = w0[j] & E, a1 = w1[j] & E, a2 = (w0[j] >> 4) & E, a3 = (w1[j] >> 4) & E;
+          const uint32_t a0 = w0[j & 3] & E, a1 = w1[j & 3] & E, a2 = (w0[j & 3] >> 4) & E, a3 = (w1[j & 3] >> 4) & E;
           mma_u8s8(dh, a0, a1, a2, a3, x_he[j], x_ho[j]);
           mma_u8s8(dl, a0, a1, a2, a3, x_le[j], x_lo[j]);
           const int sc0 = r0.sc(j), sc1 = r1.sc(j), m0 = r0.m(j), m1 = r1.m(j);
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
-            accT[c] += static_cast<long long>(sc0) * (dh[c] * 256 + dl[c]);
-            accT[2 + c] += static_cast<long long>(sc1) * (dh[2 + c] * 256 + dl[2 + c]);
+            accH[c] += sc0 * dh[c];
+            accL[c] += sc0 * dl[c];
+            accH[2 + c] += sc1 * dh[2 + c];
+            accL[2 + c] += sc1 * dl[2 + c];
             accM[c] += m0 * sumx[c][j];
             accM[2 + c] += m1 * sumx[c][j];
           }
         }
         // rows g of tiles 2 pr and 2 pr + 1, tokens 2t and 2t+1
         *reinterpret_cast<float2*>(red_w + ((2 * pr) * kRowsPerTile + g) * kTokCols + 2 * t) =
-            make_float2(step[0] * (r0.d * static_cast<float>(accT[0]) - r0.dmin * static_cast<float>(accM[0])),
-                        step[1] * (r0.d * static_cast<float>(accT[1]) - r0.dmin * static_cast<float>(accM[1])));
+            make_float2(step[0] * (r0.d * scaled_sum(accH[0], accL[0]) - r0.dmin * static_cast<float>(accM[0])),
+                        step[1] * (r0.d * scaled_sum(accH[1], accL[1]) - r0.dmin * static_cast<float>(accM[1])));
         *reinterpret_cast<float2*>(red_w + ((2 * pr + 1) * kRowsPerTile + g) * kTokCols + 2 * t) =
-            make_float2(step[0] * (r1.d * static_cast<float>(accT[2]) - r1.dmin * static_cast<float>(accM[2])),
-                        step[1] * (r1.d * static_cast<float>(accT[3]) - r1.dmin * static_cast<float>(accM[3])));
+            make_float2(step[0] * (r1.d * scaled_sum(accH[2], accL[2]) - r1.dmin * static_cast<float>(accM[2])),
+                        step[1] * (r1.d * scaled_sum(accH[3], accL[3]) - r1.dmin * static_cast<float>(accM[3])));
       }
       // the whole warp has consumed the slot: hand it back and request the next batch
       __syncwarp();
