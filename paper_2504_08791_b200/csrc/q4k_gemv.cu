@@ -275,46 +275,72 @@ __device__ __forceinline__ ulonglong2 ld_l2(const acc_t* p) { return __ldcg(rein
 // lane's share of the sum of squares (kResidual).  This step sits on the critical path between two
 // products and a round trip to L2 takes about a microsecond, so every load of a token is issued
 // before any is used.
-template <int NTOK>
-__device__ __forceinline__ void stage_warp(const GemvParams& P, int s, int tok_first, float (&v)[NTOK][8], float (&ss)[NTOK]) {
+template <int NTOK, int K0, int N>
+__device__ __forceinline__ void stage_tokens(const GemvParams& P, int s, int tok_first, float (&v)[NTOK][8], float (&ss)[NTOK]) {
   const int lane = threadIdx.x & 31;
   const int64_t cols = static_cast<int64_t>(P.n_sb) * 256;
   const int64_t k0 = static_cast<int64_t>(s) * 256 + 8 * lane;
+  // Tokens K0 .. K0 + N - 1 of the pass: their loads come first (one round trip), then the arithmetic.
+  if (P.kind == kPlain) {
+    float4 a[NTOK], b[NTOK];
 #pragma unroll
-  for (int k = 0; k < NTOK; ++k) {
-    const int64_t row = static_cast<int64_t>(tok_first + k);
-    ss[k] = 0.f;
-    if (P.kind == kPlain) {
-      const float4 a = ld_l2(P.x + row * cols + k0), b = ld_l2(P.x + row * cols + k0 + 4);
-      v[k][0] = a.x; v[k][1] = a.y; v[k][2] = a.z; v[k][3] = a.w;
-      v[k][4] = b.x; v[k][5] = b.y; v[k][6] = b.z; v[k][7] = b.w;
-    } else if (P.kind == kResidual) {
-      const float4 h0 = ld_l2(P.h_in + row * cols + k0), h1 = ld_l2(P.h_in + row * cols + k0 + 4);
-      const float4 g0 = __ldg(reinterpret_cast<const float4*>(P.gain + k0)), g1 = __ldg(reinterpret_cast<const float4*>(P.gain + k0 + 4));
-      float r[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-      if (P.acc_in) {
+    for (int k = K0; k < K0 + N; ++k) {
+      const float* x = P.x + static_cast<int64_t>(tok_first + k) * cols + k0;
+      a[k] = ld_l2(x);
+      b[k] = ld_l2(x + 4);
+    }
+#pragma unroll
+    for (int k = K0; k < K0 + N; ++k) {
+      ss[k] = 0.f;
+      v[k][0] = a[k].x; v[k][1] = a[k].y; v[k][2] = a[k].z; v[k][3] = a[k].w;
+      v[k][4] = b[k].x; v[k][5] = b[k].y; v[k][6] = b[k].z; v[k][7] = b[k].w;
+    }
+  } else if (P.kind == kResidual) {
+    float4 h0[NTOK], h1[NTOK];
+    ulonglong2 a[NTOK][4];
+    const bool has_acc = P.acc_in != nullptr;
+#pragma unroll
+    for (int k = K0; k < K0 + N; ++k) {
+      const int64_t row = static_cast<int64_t>(tok_first + k);
+      h0[k] = ld_l2(P.h_in + row * cols + k0);
+      h1[k] = ld_l2(P.h_in + row * cols + k0 + 4);
+      if (has_acc) {
         const acc_t* ain = P.acc_in + row * P.mpad_in + static_cast<int64_t>(s) * 256;   // kOrderResidual
-        ulonglong2 a[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a[i] = ld_l2(ain + 2 * (32 * i + lane));
+        for (int i = 0; i < 4; ++i) a[k][i] = ld_l2(ain + 2 * (32 * i + lane));
+      }
+    }
+    const float4 g0 = __ldg(reinterpret_cast<const float4*>(P.gain + k0)), g1 = __ldg(reinterpret_cast<const float4*>(P.gain + k0 + 4));
+    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+    for (int k = K0; k < K0 + N; ++k) {
+      const int64_t row = static_cast<int64_t>(tok_first + k);
+      float r[8] = {h0[k].x, h0[k].y, h0[k].z, h0[k].w, h1[k].x, h1[k].y, h1[k].z, h1[k].w};
+      if (has_acc) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          r[2 * i] += acc_value(a[i].x);
-          r[2 * i + 1] += acc_value(a[i].y);
+          r[2 * i] += acc_value(a[k][i].x);
+          r[2 * i + 1] += acc_value(a[k][i].y);
         }
       }
       *reinterpret_cast<float4*>(P.h_out + row * cols + k0) = make_float4(r[0], r[1], r[2], r[3]);
       *reinterpret_cast<float4*>(P.h_out + row * cols + k0 + 4) = make_float4(r[4], r[5], r[6], r[7]);
       ss[k] = ((r[0] * r[0] + r[1] * r[1]) + (r[2] * r[2] + r[3] * r[3])) + ((r[4] * r[4] + r[5] * r[5]) + (r[6] * r[6] + r[7] * r[7]));
-      const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
       for (int i = 0; i < 8; ++i) v[k][i] = r[i] * gg[i];
-    } else {   // kSwiglu: the previous product's fused rows 2c (gate) and 2c+1 (up): 16 consecutive accumulators
-      const acc_t* ain = P.acc_in + row * P.mpad_in + static_cast<int64_t>(s) * 512;   // kOrderSwiglu
-      ulonglong2 a[8];
+    }
+  } else {   // kSwiglu: the previous product's fused rows 2c (gate) and 2c+1 (up): 16 consecutive accumulators
+    ulonglong2 a[NTOK][8];
+    float ssq[NTOK];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) a[i] = ld_l2(ain + 2 * (32 * i + lane));
-      float ssq = 0.f;
+    for (int k = K0; k < K0 + N; ++k) {
+      const acc_t* ain = P.acc_in + static_cast<int64_t>(tok_first + k) * P.mpad_in + static_cast<int64_t>(s) * 512;   // kOrderSwiglu
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[k][i] = ld_l2(ain + 2 * (32 * i + lane));
+    }
+#pragma unroll
+    for (int k = K0; k < K0 + N; ++k) {
+      ssq[k] = 0.f;
       const float* sp = P.ssq_in + (tok_first + k) * kMaxStatBlocks;
       for (int g0 = 0; g0 < P.n_ssq_in; g0 += 8) {     // groups added in ascending order
         float sq[8];
@@ -323,15 +349,34 @@ __device__ __forceinline__ void stage_warp(const GemvParams& P, int s, int tok_f
           if (g0 + i < P.n_ssq_in) sq[i] = __ldcg(sp + g0 + i);
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          if (g0 + i < P.n_ssq_in) ssq += sq[i];
+          if (g0 + i < P.n_ssq_in) ssq[k] += sq[i];
       }
-      const float inv = 1.0f / sqrtf(ssq * P.inv_width_in + P.eps_in);
+    }
+#pragma unroll
+    for (int k = K0; k < K0 + N; ++k) {
+      ss[k] = 0.f;
+      const float inv = 1.0f / sqrtf(ssq[k] * P.inv_width_in + P.eps_in);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const float gt = acc_value(a[i].x) * inv, up = acc_value(a[i].y) * inv;
+        const float gt = acc_value(a[k][i].x) * inv, up = acc_value(a[k][i].y) * inv;
         v[k][i] = gt / (1.0f + expf(-gt)) * up;
       }
     }
+  }
+}
+
+// One or two tokens: one round trip.  Three or four tokens are staged one at a time: with their
+// activation registers (20 per token) there is no room for more loads in flight without spills.
+template <int NTOK>
+__device__ __forceinline__ void stage_warp(const GemvParams& P, int s, int tok_first, float (&v)[NTOK][8], float (&ss)[NTOK]) {
+  static_assert(NTOK <= 4, "at most four tokens per pass of this kernel");
+  if constexpr (NTOK <= 2) {
+    stage_tokens<NTOK, 0, NTOK>(P, s, tok_first, v, ss);
+  } else {
+    stage_tokens<NTOK, 0, 1>(P, s, tok_first, v, ss);
+    stage_tokens<NTOK, 1, 1>(P, s, tok_first, v, ss);
+    stage_tokens<NTOK, 2, 1>(P, s, tok_first, v, ss);
+    if constexpr (NTOK == 4) stage_tokens<NTOK, 3, 1>(P, s, tok_first, v, ss);
   }
 }
 
@@ -790,26 +835,38 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
       uint4* xs_q = reinterpret_cast<uint4*>(my_ring + rslot * kBatchBytes);
       int* xs_sum = reinterpret_cast<int*>(xs_q + kTokCols * 32);
       float* xs_step = reinterpret_cast<float*>(xs_sum + kTokCols * 8);
-      for (int k = 0; k < kTokCols; ++k) {
-        LaneQuant lq;
-        lq.q = make_uint4(0, 0, 0, 0);
-        lq.step = 0.f;
-        lq.sum = 0;
-        if (k < n_tok) {
-          float v[1][8];
-          float ss1[1];
-          stage_warp<1>(P, cur.grp * sg + warp, k, v, ss1);
-          lq = quantise_lane_column(v[0]);
-          if (P.kind == kResidual) {
-            float a = ss1[0];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-            if (lane == 0) s_red[warp * kTokCols + k] = a;
-          }
-        }
+      auto publish = [&](int k, const LaneQuant& lq, float ssv, bool live) {
         xs_q[k * 32 + lane] = lq.q;
         if (t == 0) xs_sum[k * 8 + g] = lq.sum;
         if (lane == 0) xs_step[k] = lq.step;
+        if (P.kind == kResidual && live) {
+          float a = ssv;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+          if (lane == 0) s_red[warp * kTokCols + k] = a;
+        }
+      };
+      LaneQuant zero;
+      zero.q = make_uint4(0, 0, 0, 0);
+      zero.step = 0.f;
+      zero.sum = 0;
+      for (int k = 0; k < kTokCols; k += 2) {      // two tokens per round trip
+        if (k + 1 < n_tok) {
+          float v[2][8];
+          float ss2[2];
+          stage_warp<2>(P, cur.grp * sg + warp, k, v, ss2);
+          publish(k, quantise_lane_column(v[0]), ss2[0], true);
+          publish(k + 1, quantise_lane_column(v[1]), ss2[1], true);
+        } else if (k < n_tok) {
+          float v[1][8];
+          float ss1[1];
+          stage_warp<1>(P, cur.grp * sg + warp, k, v, ss1);
+          publish(k, quantise_lane_column(v[0]), ss1[0], true);
+          publish(k + 1, zero, 0.f, false);
+        } else {
+          publish(k, zero, 0.f, false);
+          publish(k + 1, zero, 0.f, false);
+        }
       }
       __syncwarp();
 #pragma unroll
