@@ -79,6 +79,18 @@ class SpeculativeDecoder:
         self.draft = _Stepper(draft)
         self.n_draft = n_draft
         self.draft_filter = draft_filter
+        self.capacity = min(target.cfg["kv_capacity"], draft.cfg["kv_capacity"])
+
+    @classmethod
+    def from_steppers(cls, target_step, draft_step, n_draft: int, capacity: int, max_n_tok: int = 8):
+        """A decoder over two objects with ``step(tokens, pos) -> next tokens`` (how the accept/reject
+        logic is exercised without a GPU)."""
+        if not 1 <= n_draft < max_n_tok:
+            raise ValueError("n_draft + 1 tokens must fit one step of the target")
+        self = cls.__new__(cls)
+        self.target, self.draft = target_step, draft_step
+        self.n_draft, self.draft_filter, self.capacity = n_draft, None, capacity
+        return self
 
     def generate(self, first_token: int, pos: int, n_new: int):
         """Continue from ``first_token`` (not yet in either cache) at position ``pos``; returns the
@@ -88,7 +100,7 @@ class SpeculativeDecoder:
         history = {pos: int(first_token)}      # token at each position from `pos` on
         last_pos = pos                         # position of the newest token, present in no cache yet
         draft_valid = pos                      # the draft cache holds positions < draft_valid
-        capacity = min(self.target.ctx.cfg["kv_capacity"], self.draft.ctx.cfg["kv_capacity"])
+        capacity = self.capacity
         while len(out) < n_new:
             n_draft = min(self.n_draft, capacity - last_pos - 1)
             if n_draft < 1:
