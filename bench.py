@@ -42,6 +42,9 @@ WORKLOADS = {
     "8b": ("8b", 1024, 1, "Llama-3-8B-shaped random-init Q4_K, 32 layers, fp16 KV context 1024, batch 1"),
 }
 SEEDS = {"70b": 3, "32b": 2, "8b": 1}
+# dram__bytes_read.sum + dram__bytes_write.sum over the four 70B-shaped layer matrices / their Q4_K bytes
+# (one ncu capture of gemv_partials_kernel<1>, profiles/gemv_partials_70b_matrices.md)
+NCU_TRAFFIC_RATIO = 489.9 / 481.3
 
 
 def log(*a):
@@ -268,8 +271,11 @@ def run_ours(args, rank, world, local_rank):
                    "bytes_per_token": bpt["total"]},
         "step_roofline": {"bound": "hbm", "achieved": step_gbs, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                           "frac": step_gbs / peak, "frac_of_nominal_8000": step_gbs / 8000.0},
-        "roofline": {"kernel": "gemv_partials_kernel<%d>" % min(T, 4), "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
-                     "unit": "GB/s", "frac": gemv_gbs / peak, "traffic": None,
+        "roofline": {"kernel": "gemv_partials_kernel<%d>" % T if T <= 4 else "gemv_tokens_kernel", "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
+                     "unit": "GB/s", "frac": gemv_gbs / peak,
+                     "traffic": (NCU_TRAFFIC_RATIO * g_bytes / g_n) if (g_n and T == 1) else None,
+                     "traffic_note": "bytes per launch: algorithmic bytes x 1.018, the DRAM read+write / Q4_K bytes ratio of the ncu "
+                                     "capture of the four layer matrices (profiles/gemv_partials_70b_matrices.md)",
                      "launches": g_n // prof_steps, "avg_launch_us": (g_ms * 1e3 / g_n) if g_n else None,
                      "timing": f"cuda events around each launch, separate pass of {prof_steps} steps"},
         "attention_kernel": {"achieved": attn_gbs, "unit": "GB/s", "frac": attn_gbs / peak, "launches": a_n // prof_steps},
