@@ -51,6 +51,11 @@ def log(*a):
     print(*a, file=sys.stderr, flush=True)
 
 
+def L_kv_bytes(cfg: dict, n_ctx: int) -> int:
+    """K and V bytes of one request's attended positions over all layers."""
+    return cfg["n_layers"] * 2 * (cfg["n_kv_heads"] * cfg["head_dim"] * 2) * n_ctx
+
+
 def bytes_per_token(cfg: dict, n_ctx: int, n_layers: int | None = None, with_head: bool = True) -> dict:
     """Algorithmic bytes one decoded token must move: Q4_K weight bytes touched + K and V bytes of
     the attended positions (the paper's device-loading model: b + 2(h_k e_k + h_v e_v) n_kv per
@@ -134,7 +139,7 @@ def job_value(ms_per_step_max: float, world: int) -> dict:
 
 
 # ------------------------------------------------------------------------------------ the GPU arm
-def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None):
+def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None, n_requests=1):
     import torch
     t0 = time.time()
     ctx = binding.Context(cfg, device=device)
@@ -144,7 +149,8 @@ def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None):
     t1 = time.time()
     for l in layers:
         k, v = synth.kv_prefill(seed, l, n_ctx, cfg["n_kv_heads"], cfg["head_dim"])
-        ctx.kv_load(l, 0, k, v)
+        for r in range(n_requests):               # every request gets a cache of its own (same synthetic content)
+            ctx.kv_load(l, 0, k, v, seq=r)
     torch.cuda.synchronize()
     log(f"[bench] model resident: weights {t1 - t0:.1f}s, kv prefill {time.time() - t1:.1f}s")
     return ctx
@@ -171,25 +177,35 @@ def run_ours(args, rank, world, local_rank):
     cfg["kv_capacity"] = max(cfg["kv_capacity"], n_ctx + 64 * args.n_tok)
     L = cfg["n_layers"]
     seed = SEEDS[args.workload] + 1000 * rank
-    ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank)
+    R = args.requests
+    if R > 1 and args.n_tok > 1:
+        raise SystemExit("--requests and --n-tok are alternatives")
+    ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank, n_requests=R)
     bpt = bytes_per_token(cfg, n_ctx)
+    if R > 1:                                     # the weights are read once per step, every request's cache once
+        bpt = dict(bpt, total=bpt["total"] + (R - 1) * L_kv_bytes(cfg, n_ctx))
     bounds = [L * i // n_windows for i in range(n_windows + 1)]
 
-    T = args.n_tok
+    T = args.n_tok if R == 1 else R
     h0 = torch.from_numpy(synth.activations(seed, T, cfg["hidden"])).cuda()
     hid = torch.empty_like(h0)
     logits = torch.empty((T, cfg["vocab"]), dtype=torch.float32, device="cuda")
 
+    def windows(pos):
+        for w in range(n_windows):
+            if R > 1:                              # one token of each of R requests, all at the same depth of their caches
+                ctx.forward_window_seqs(bounds[w], bounds[w + 1], hid, hid, list(range(R)), [pos] * R)
+            else:
+                ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, T)
+
     def device_step(pos):
         hid.copy_(h0)
-        for w in range(n_windows):
-            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, T)
+        windows(pos)
         ctx.logits(hid, T, logits)
 
     def e2e_step(tok, pos):
         ctx.embed([tok] * T, hid)                  # host token ids -> device (4 bytes each)
-        for w in range(n_windows):
-            ctx.forward_window(bounds[w], bounds[w + 1], hid, hid, pos, T)
+        windows(pos)
         ctx.logits(hid, T, logits)
         return int(ctx.argmax(logits, T)[T - 1])   # device -> host (4 bytes each), waits
 
@@ -219,16 +235,17 @@ def run_ours(args, rank, world, local_rank):
     ms_step = ms_total / args.steps
 
     # end to end through the ABI: host token in, host token out, every step
+    adv = 1 if R > 1 else T                        # positions a step advances a cache by
     tok = 0
     for i in range(min(args.warmup, 3)):
-        tok = e2e_step(tok, n_ctx + i * T)
+        tok = e2e_step(tok, n_ctx + i * adv)
     barrier()
-    e2e_steps = min(args.steps, (cfg["kv_capacity"] - n_ctx - 3 * T) // T)
+    e2e_steps = min(args.steps, (cfg["kv_capacity"] - n_ctx - 3 * adv) // adv)
     ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.perf_counter()
     ev2.record()
     for i in range(e2e_steps):
-        tok = e2e_step(tok, n_ctx + (3 + i) * T)
+        tok = e2e_step(tok, n_ctx + (3 + i) * adv)
     ev3.record()
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - wall0) * 1e3
@@ -264,9 +281,10 @@ def run_ours(args, rank, world, local_rank):
         "vs_baseline": None,
         "dtype": "q4_k weights x int16 activations, int32/fp32 accumulate",
         "data": "synthetic",
-        "tokens_per_s": job_value(ms_step, world)["tokens_per_s"],
+        "tokens_per_s": job_value(ms_step, world)["tokens_per_s"] * (R if R > 1 else 1),
         "config": {"workload": desc, "layers": L, "windows": n_windows, "n_ctx": n_ctx, "n_tok": T,
-                   "value_is": "ms per decoded token" if T == 1 else "ms per verification step of %d tokens" % T,
+                   "value_is": ("ms per decoded token" if T == 1 else "ms per verification step of %d tokens" % T) if R == 1
+                   else "ms per step of %d concurrent requests (one token each)" % R, "requests": R,
                    "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs larger than L2 (>= 4.9 GB per step)",
                    "bytes_per_token": bpt["total"]},
         "step_roofline": {"bound": "hbm", "achieved": step_gbs, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
@@ -382,6 +400,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     ap.add_argument("--n-tok", type=int, default=1, help="tokens per step (speculative verification pass when > 1)")
     ap.add_argument("--ctx", type=int, default=0, help="override the KV context length (profiling captures)")
+    ap.add_argument("--requests", type=int, default=1, help="concurrent requests per step, one token each, own KV caches")
     ap.add_argument("--speculative", default="", choices=["", "8b", "32b"],
                     help="also time speculative decoding cycles with a draft model of this shape")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -125,6 +125,19 @@ int prima_load_q4k_weights(prima_ctx* ctx, int layer, int tensor_id, const void*
 int prima_forward_window(prima_ctx* ctx, int layer_begin, int layer_end, const float* hidden_in,
                          float* hidden_out, int pos, int n_tok);
 
+/* One step of several independent requests (the paper's serving mode: Appendix A.11 "Concurrent
+ * requests" / A.12, requests merged per token step, each with its own KV cache).  Token t belongs to
+ * sequence seq[t] (0..63, each at most once per step) and sits at position pos[t] of that sequence's
+ * cache; the projections run over all n_seq tokens together (the weights are read once), attention
+ * runs per token over its own sequence's cache, to which the token's K and V are appended.
+ * Sequence 0 is the cache that prima_forward_window and prima_kv_load use; the cache of another
+ * sequence is allocated (zero-filled) the first time it is named.  seq, pos: host int32[n_seq];
+ * hidden_in / hidden_out: dev fp32 [n_seq x hidden].  Errors as prima_forward_window, plus
+ * PRIMA_ERR_ARG for a sequence id out of range or named twice and PRIMA_ERR_NOMEM if a cache cannot
+ * be allocated. */
+int prima_forward_window_seqs(prima_ctx* ctx, int layer_begin, int layer_end, const float* hidden_in,
+                              float* hidden_out, const int32_t* seq, const int32_t* pos, int n_seq);
+
 /* Output layer: logits[t][v] = W_head . RMSNorm(hidden[t]; out_norm).  hidden: dev fp32
  * [n_tok x hidden]; logits: dev fp32 [n_tok x vocab]. */
 int prima_logits(prima_ctx* ctx, const float* hidden, int n_tok, float* logits);
@@ -141,6 +154,9 @@ int prima_argmax(prima_ctx* ctx, const float* logits, int n_tok, int32_t* tokens
  * binary16 bit patterns.  Both calls synchronise.  Used to prefill a context and by tests. */
 int prima_kv_load(prima_ctx* ctx, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v);
 int prima_kv_read(prima_ctx* ctx, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v);
+/* The same for the cache of sequence `seq` (0..63; sequence 0 is the cache of the calls above). */
+int prima_kv_load_seq(prima_ctx* ctx, int seq, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v);
+int prima_kv_read_seq(prima_ctx* ctx, int seq, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v);
 
 /* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word (a
  * partial sum outside the accumulator range, or a bounded wait inside a kernel that gave up) and

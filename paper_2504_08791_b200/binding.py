@@ -24,6 +24,7 @@ EXPORTS = [
     "prima_embed", "prima_argmax", "prima_kv_load", "prima_kv_read", "prima_sync", "prima_last_error",
     "prima_launch_count", "prima_profile_enable", "prima_profile_read", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
     "prima_gemv_plan_destroy", "prima_gemv_q4k_noalloc", "prima_gemv_q4k_noalloc_error",
+    "prima_forward_window_seqs", "prima_kv_load_seq", "prima_kv_read_seq",
 ]
 
 
@@ -60,6 +61,9 @@ def lib():
         L.prima_argmax.argtypes = [vp, vp, i32, vp]
         L.prima_kv_load.argtypes = [vp, i32, i32, i32, vp, vp]
         L.prima_kv_read.argtypes = [vp, i32, i32, i32, vp, vp]
+        L.prima_forward_window_seqs.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32]
+        L.prima_kv_load_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.prima_kv_read_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.prima_sync.argtypes = [vp]
         L.prima_last_error.argtypes = [vp]
         L.prima_last_error.restype = C.c_char_p
@@ -195,16 +199,25 @@ class Context:
         _check(lib().prima_argmax(self._h, _dev_ptr(logits), n_tok, _host_ptr(out)), self._h)
         return out
 
-    def kv_load(self, layer: int, pos_begin: int, k_bits: np.ndarray, v_bits: np.ndarray):
+    def kv_load(self, layer: int, pos_begin: int, k_bits: np.ndarray, v_bits: np.ndarray, seq: int = 0):
         k_bits = np.ascontiguousarray(k_bits, dtype=np.uint16)
         v_bits = np.ascontiguousarray(v_bits, dtype=np.uint16)
-        _check(lib().prima_kv_load(self._h, layer, pos_begin, k_bits.shape[0], _host_ptr(k_bits), _host_ptr(v_bits)), self._h)
+        _check(lib().prima_kv_load_seq(self._h, seq, layer, pos_begin, k_bits.shape[0], _host_ptr(k_bits), _host_ptr(v_bits)), self._h)
 
-    def kv_read(self, layer: int, pos_begin: int, n_pos: int):
+    def kv_read(self, layer: int, pos_begin: int, n_pos: int, seq: int = 0):
         shape = (n_pos, self.cfg["n_kv_heads"], self.cfg["head_dim"])
         k, v = np.empty(shape, np.uint16), np.empty(shape, np.uint16)
-        _check(lib().prima_kv_read(self._h, layer, pos_begin, n_pos, _host_ptr(k), _host_ptr(v)), self._h)
+        _check(lib().prima_kv_read_seq(self._h, seq, layer, pos_begin, n_pos, _host_ptr(k), _host_ptr(v)), self._h)
         return k, v
+
+    def forward_window_seqs(self, layer_begin: int, layer_end: int, hidden_in, hidden_out, seqs, positions):
+        """prima_forward_window_seqs: one token of each of several independent requests."""
+        seqs = np.ascontiguousarray(seqs, dtype=np.int32).reshape(-1)
+        positions = np.ascontiguousarray(positions, dtype=np.int32).reshape(-1)
+        if seqs.size != positions.size:
+            raise ValueError("one position per sequence")
+        _check(lib().prima_forward_window_seqs(self._h, layer_begin, layer_end, _dev_ptr(hidden_in), _dev_ptr(hidden_out),
+                                               _host_ptr(seqs), _host_ptr(positions), seqs.size), self._h)
 
     def sync(self):
         _check(lib().prima_sync(self._h), self._h)

@@ -33,8 +33,9 @@ struct Layer {
   float* g_ffn = nullptr;
   float gmax_attn = 1.f, gmax_ffn = 1.f;
   uint32_t have = 0;   // bit per tensor id
-  __half* k = nullptr;
+  __half* k = nullptr;        // cache of sequence 0 (the only one that prima_forward_window uses)
   __half* v = nullptr;
+  std::vector<__half*> k_seq, v_seq;   // caches of sequences 1.. (index seq - 1), allocated on first use
 };
 
 constexpr uint32_t kLayerMask = (1u << 9) - 1;
@@ -146,6 +147,33 @@ int ensure_kv(prima_ctx* c, int layer) {
   int rc = dev_alloc(c, &L.k, n, true);
   if (rc != PRIMA_OK) return rc;
   return dev_alloc(c, &L.v, n, true);
+}
+
+constexpr int kMaxSeqs = 64;
+
+// Cache pointers of (layer, sequence); allocates the sequence's cache on first use.
+int ensure_kv_seq(prima_ctx* c, int layer, int seq, __half** k, __half** v) {
+  int rc = ensure_kv(c, layer);
+  if (rc != PRIMA_OK) return rc;
+  Layer& L = c->layers[layer];
+  if (seq == 0) {
+    *k = L.k;
+    *v = L.v;
+    return PRIMA_OK;
+  }
+  if (static_cast<int>(L.k_seq.size()) < seq) {
+    L.k_seq.resize(seq, nullptr);
+    L.v_seq.resize(seq, nullptr);
+  }
+  if (!L.k_seq[seq - 1]) {
+    const size_t n = static_cast<size_t>(c->cfg.n_kv_heads) * c->cfg.kv_capacity * kHeadDim;
+    rc = dev_alloc(c, &L.k_seq[seq - 1], n, true);
+    if (rc == PRIMA_OK) rc = dev_alloc(c, &L.v_seq[seq - 1], n, true);
+    if (rc != PRIMA_OK) return rc;
+  }
+  *k = L.k_seq[seq - 1];
+  *v = L.v_seq[seq - 1];
+  return PRIMA_OK;
 }
 
 // Copy a standard-layout matrix (host or device) through the staging buffer and re-tile it.
@@ -366,16 +394,12 @@ int prima_load_q4k_weights(prima_ctx* c, int layer, int tensor_id, const void* d
   return rc;
 }
 
-int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos,
-                         int n_tok) {
-  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_forward_window: null context");
+// One step over layers [layer_begin, layer_end).  seq == nullptr: n_tok tokens of sequence 0 at positions
+// pos0 .. pos0 + n_tok - 1, causal among themselves.  Otherwise token t belongs to sequence seq[t] and sits at
+// position pos[t] of that sequence's own cache: the products run over all tokens together, attention per token.
+static int forward_window_impl(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos0,
+                               int n_tok, const int32_t* seq, const int32_t* pos) {
   const prima_model_config& g = c->cfg;
-  if (!hidden_in || !hidden_out) return fail(c, PRIMA_ERR_ARG, "prima_forward_window: null hidden pointer");
-  if (layer_begin < 0 || layer_end > g.n_layers || layer_begin > layer_end) return fail(c, PRIMA_ERR_ARG, "bad layer range");
-  if (n_tok < 1 || n_tok > g.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
-  if (pos < 0 || static_cast<int64_t>(pos) + n_tok > g.kv_capacity) return fail(c, PRIMA_ERR_ARG, "pos + n_tok exceeds kv_capacity");
-  for (int l = layer_begin; l < layer_end; ++l)
-    if ((c->layers[l].have & kLayerMask) != kLayerMask) return fail(c, PRIMA_ERR_STATE, "a layer of the window is not fully loaded");
   DeviceGuard guard(g.device);
   cudaStream_t st = c->stream;
   const int64_t e_ = g.hidden;
@@ -388,7 +412,12 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
     }
     return PRIMA_OK;
   }
-  LAUNCH(c, launch_rope_table(c->rope_tab, pos, n_tok, g.rope_theta, st), "rope_table");
+  if (!seq) {
+    LAUNCH(c, launch_rope_table(c->rope_tab, pos0, n_tok, g.rope_theta, st), "rope_table");
+  } else {
+    for (int t = 0; t < n_tok; ++t)
+      LAUNCH(c, launch_rope_table(c->rope_tab + t * (kHeadDim / 2), pos[t], 1, g.rope_theta, st), "rope_table");
+  }
   const int64_t mpad_e = (e_ + 7) / 8 * 8;
   // The residual stream entering a layer is h_in plus the value of the previous down projection's
   // accumulators (nothing for the first layer of the call); each product's CTAs finish what they
@@ -406,9 +435,23 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(qkv)");
     c->ssq_attn = in.ssq_out;
     c->ssq_attn.eps = g.rms_eps;
-    LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos + n_tok),
-             launch_attention(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k, L.v, g.kv_capacity, H, G, pos, n_tok,
-                              c->attn, c->obuf, c->sm_count, st), "attention");
+    if (!seq) {
+      LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos0 + n_tok),
+               launch_attention(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k, L.v, g.kv_capacity, H, G, pos0, n_tok,
+                                c->attn, c->obuf, c->sm_count, st), "attention");
+    } else {
+      for (int t = 0; t < n_tok; ++t) {          // one request per token: its own cache, its own position
+        __half *kc = nullptr, *vc = nullptr;
+        const int rc = ensure_kv_seq(c, l, seq[t], &kc, &vc);
+        if (rc != PRIMA_OK) return rc;
+        SumSq ssq_t = c->ssq_attn;
+        ssq_t.data += t * kMaxStatBlocks;
+        LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos[t] + 1),
+                 launch_attention(c->acc_qkv + t * L.qkv.mpad(), L.qkv.mpad(), ssq_t, c->rope_tab + t * (kHeadDim / 2), g.rope_mode, kc, vc,
+                                  g.kv_capacity, H, G, pos[t], 1, c->attn, c->obuf + static_cast<int64_t>(t) * H * kHeadDim, c->sm_count, st),
+                 "attention");
+      }
+    }
     GemvIn in_o;                                 // O: plain attention output
     in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status;
     in_o.zero0 = c->acc_qkv; in_o.zero0_n = static_cast<int64_t>(n_tok) * L.qkv.mpad();
@@ -432,6 +475,40 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
   LAUNCH(c, launch_finish_residual(c->acc_down, mpad_e, e_, n_tok, c->h_a, hidden_out, c->acc_gu,
                                    static_cast<int64_t>(n_tok) * c->layers[layer_end - 1].gu.mpad(), st), "finish_residual");
   return PRIMA_OK;
+}
+
+static int window_args_ok(prima_ctx* c, const char* who, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int n_tok) {
+  const prima_model_config& g = c->cfg;
+  if (!hidden_in || !hidden_out) return fail(c, PRIMA_ERR_ARG, std::string(who) + ": null hidden pointer");
+  if (layer_begin < 0 || layer_end > g.n_layers || layer_begin > layer_end) return fail(c, PRIMA_ERR_ARG, "bad layer range");
+  if (n_tok < 1 || n_tok > g.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
+  for (int l = layer_begin; l < layer_end; ++l)
+    if ((c->layers[l].have & kLayerMask) != kLayerMask) return fail(c, PRIMA_ERR_STATE, "a layer of the window is not fully loaded");
+  return PRIMA_OK;
+}
+
+int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos,
+                         int n_tok) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_forward_window: null context");
+  int rc = window_args_ok(c, "prima_forward_window", layer_begin, layer_end, hidden_in, hidden_out, n_tok);
+  if (rc != PRIMA_OK) return rc;
+  if (pos < 0 || static_cast<int64_t>(pos) + n_tok > c->cfg.kv_capacity) return fail(c, PRIMA_ERR_ARG, "pos + n_tok exceeds kv_capacity");
+  return forward_window_impl(c, layer_begin, layer_end, hidden_in, hidden_out, pos, n_tok, nullptr, nullptr);
+}
+
+int prima_forward_window_seqs(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out,
+                              const int32_t* seq, const int32_t* pos, int n_seq) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_forward_window_seqs: null context");
+  int rc = window_args_ok(c, "prima_forward_window_seqs", layer_begin, layer_end, hidden_in, hidden_out, n_seq);
+  if (rc != PRIMA_OK) return rc;
+  if (!seq || !pos) return fail(c, PRIMA_ERR_ARG, "prima_forward_window_seqs: null seq or pos");
+  for (int t = 0; t < n_seq; ++t) {
+    if (seq[t] < 0 || seq[t] >= kMaxSeqs) return fail(c, PRIMA_ERR_ARG, "sequence id outside 0..63");
+    if (pos[t] < 0 || pos[t] >= c->cfg.kv_capacity) return fail(c, PRIMA_ERR_ARG, "position outside the cache");
+    for (int u = 0; u < t; ++u)
+      if (seq[u] == seq[t]) return fail(c, PRIMA_ERR_ARG, "a sequence may appear once per step");
+  }
+  return forward_window_impl(c, layer_begin, layer_end, hidden_in, hidden_out, 0, n_seq, seq, pos);
 }
 
 int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
@@ -487,14 +564,23 @@ static int kv_args_ok(prima_ctx* c, int layer, int pos_begin, int n_pos, const v
 
 // Host layout [n_pos][G][128]; device layout [G][capacity][128]: one strided 2-D copy per KV head.
 int prima_kv_load(prima_ctx* c, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v) {
+  return prima_kv_load_seq(c, 0, layer, pos_begin, n_pos, k, v);
+}
+
+int prima_kv_read(prima_ctx* c, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v) {
+  return prima_kv_read_seq(c, 0, layer, pos_begin, n_pos, k, v);
+}
+
+int prima_kv_load_seq(prima_ctx* c, int seq, int layer, int pos_begin, int n_pos, const uint16_t* k, const uint16_t* v) {
   if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_kv_load: null context");
   int rc = kv_args_ok(c, layer, pos_begin, n_pos, k, v);
   if (rc != PRIMA_OK) return rc;
+  if (seq < 0 || seq >= kMaxSeqs) return fail(c, PRIMA_ERR_ARG, "sequence id outside 0..63");
   DeviceGuard guard(c->cfg.device);
-  rc = ensure_kv(c, layer);
+  struct { __half* k; __half* v; } L;
+  rc = ensure_kv_seq(c, layer, seq, &L.k, &L.v);
   if (rc != PRIMA_OK) return rc;
   if (n_pos == 0) return PRIMA_OK;
-  Layer& L = c->layers[layer];
   const int G = c->cfg.n_kv_heads;
   const size_t row = kHeadDim * 2;
   for (int gk = 0; gk < G; ++gk) {
@@ -510,15 +596,16 @@ int prima_kv_load(prima_ctx* c, int layer, int pos_begin, int n_pos, const uint1
   return PRIMA_OK;
 }
 
-int prima_kv_read(prima_ctx* c, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v) {
+int prima_kv_read_seq(prima_ctx* c, int seq, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v) {
   if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_kv_read: null context");
   int rc = kv_args_ok(c, layer, pos_begin, n_pos, k, v);
   if (rc != PRIMA_OK) return rc;
+  if (seq < 0 || seq >= kMaxSeqs) return fail(c, PRIMA_ERR_ARG, "sequence id outside 0..63");
   DeviceGuard guard(c->cfg.device);
-  rc = ensure_kv(c, layer);
+  struct { __half* k; __half* v; } L;
+  rc = ensure_kv_seq(c, layer, seq, &L.k, &L.v);
   if (rc != PRIMA_OK) return rc;
   if (n_pos == 0) return PRIMA_OK;
-  Layer& L = c->layers[layer];
   const int G = c->cfg.n_kv_heads;
   const size_t row = kHeadDim * 2;
   for (int gk = 0; gk < G; ++gk) {
