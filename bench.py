@@ -33,7 +33,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2504_08791_b200 import synth  # noqa: E402
+from paper_2504_08791_b200 import schedule, synth  # noqa: E402
 
 WORKLOADS = {
     # name: (shape, context length, number of windows, description)
@@ -184,7 +184,10 @@ def run_ours(args, rank, world, local_rank):
     bpt = bytes_per_token(cfg, n_ctx)
     if R > 1:                                     # the weights are read once per step, every request's cache once
         bpt = dict(bpt, total=bpt["total"] + (R - 1) * L_kv_bytes(cfg, n_ctx))
-    bounds = [L * i // n_windows for i in range(n_windows + 1)]
+    # the ring schedule with equal windows and one round: n_windows "devices" of L / n_windows layers each
+    ring = schedule.windows(L, [-(-L // n_windows)] * n_windows)
+    bounds = [w.layer_begin for w in ring] + [L]
+    n_windows = len(ring)
 
     T = args.n_tok if R == 1 else R
     h0 = torch.from_numpy(synth.activations(seed, T, cfg["hidden"])).cuda()

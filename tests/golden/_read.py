@@ -37,3 +37,23 @@ def handbuilt_blocks():
             w={int(t.split(":")[0]): float(t.split(":")[1]) for t in f["w"].split()},
         )
     return blocks
+
+
+def prp_schedules():
+    """Parse prp_schedule.txt -> {name: dict(layers, window_sizes, rounds, w=[(round, device, first, last)], ...)}."""
+    out, cur = {}, None
+    for line in open(os.path.join(HERE, "prp_schedule.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("["):
+            cur = line.strip("[]")
+            out[cur] = {"w": []}
+            continue
+        key, val = [t.strip() for t in line.split(":", 1)]
+        nums = [int(t) for t in val.split()]
+        if key == "w":
+            out[cur]["w"].append(tuple(nums))
+        else:
+            out[cur][key] = nums if key == "window_sizes" else nums[0]
+    return out

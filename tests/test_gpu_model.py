@@ -114,6 +114,27 @@ def test_window_splits_are_bit_identical_on_the_gpu(gpu, splits, n_tok):
     part.close()
 
 
+@pytest.mark.parametrize("sizes", [[1, 2], [2, 1], [1, 1, 1]])
+def test_ring_schedule_with_uneven_windows_is_bit_identical_to_one_pass(gpu, sizes):
+    """The paper's ring schedule (devices take w_m layers per turn, several rounds) executed window by
+    window gives the bits of a single full-depth pass."""
+    from paper_2504_08791_b200 import schedule
+    torch, binding = gpu
+    cfg = synth.model_config("small")
+    L = cfg["n_layers"]
+    p = Pair(gpu, cfg, seed=29, n_prefill=50)
+    h0 = synth.activations(29, 2, cfg["hidden"])
+    one = p.gpu_window(0, L, h0, 50)
+    ws = schedule.windows(L, sizes)
+    assert schedule.rounds(L, sizes) >= 2
+    hin = torch.from_numpy(h0).cuda()
+    hout = torch.empty_like(hin)
+    schedule.run_schedule(p.ctx, ws, hin, hout, 50, 2)
+    p.ctx.sync()
+    assert np.array_equal(hout.cpu().numpy().view(np.uint32), one.view(np.uint32))
+    p.close()
+
+
 def test_five_token_step_agrees_with_five_single_steps_on_the_gpu(gpu):
     cfg = synth.model_config("small")
     pos = 77
