@@ -1,0 +1,361 @@
+// Q4_K product for five to eight tokens per step: the tokens are the columns of the tensor-core product.
+#include "gemv_device.cuh"
+
+namespace prima {
+namespace {
+using namespace gemv_detail;
+
+// ---- several tokens per step: the tokens are the columns of the tensor-core product ----------------
+//
+// With 2..8 tokens (verification of draft tokens) the product is a small dense contraction and the
+// int8 instruction m16n8k32 is used as one: A = the 32 weights of ONE sub-block for 16 rows (two
+// row tiles), B = the activations of that sub-block for 8 tokens, once with their high and once with
+// their low bytes.  The weights are read once for all tokens.  Same tiled matrix, same ring of bulk
+// copies and exact integer sums as the one-token kernel; what differs:
+//  * A unit stores (row g, sub-block j) as one 16-byte piece, but the instruction wants from lane
+//    (g, t) bytes 4t..4t+3 of every sub-block of row g: exactly what a matrix load (ldmatrix) of the
+//    eight rows' pieces delivers.  Word t of a sub-block holds weights 8t..8t+7, whose even nibbles
+//    become k slots 4t..4t+3 and odd nibbles k slots 16+4t..+3.
+//  * Lane (g, t) supplies column g of B, i.e. token g: for each sub-block the four words (high/low
+//    bytes x even/odd weights) of its quarter t.  The quantised activations of a column go through
+//    shared memory once to reach the lanes in that arrangement.
+//  * The activations of a token are 16-bit integers with ONE step for the 256 values of the column,
+//    s = max|x| / 32639, so that the sums over the sub-blocks can stay in the integers:
+//        partial[row][tok] = s[tok] * (d * sum_j sc_j I_j  -  dmin * sum_j m_j sum(x_q)_j),
+//    I_j = 256 * high + low from the two instructions (the high and low parts are summed apart).
+//  * The instruction leaves lane (g, t) the complete sums of rows g and g+8 for tokens 2t and 2t+1:
+//    no reduction over the quad.
+// Two CTAs of SG warps per SM, warp w on column group * SG + w as in the one-token kernel, ring of
+// kRingTok batches per warp; the second ring slot doubles as the buffer through which the warp's
+// quantised activations are rearranged, before its first copy is requested.
+constexpr int kRingTok = 2;
+constexpr int kTokCols = 8;   // columns of the instruction = tokens per pass
+static_assert(kTokCols * 32 * 16 + kTokCols * 8 * 4 + kTokCols * 4 <= kBatchBytes, "the activation buffer must fit a ring slot");
+
+// Four 8x8 matrices of 16-bit elements from shared memory: lane l gives the address of row l % 8 of
+// matrix l / 8 (16 bytes each); lane (g, t) receives bytes 4t..4t+3 of row g of each matrix.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+
+// 256 * high + low as a float: the two 32-bit sums are each below 2^25 in magnitude, their combination
+// needs up to 33 bits, so it is formed in fp32 (relative error 2^-24, far below the other roundings).
+__device__ __forceinline__ float scaled_sum(int high, int low) { return fmaf(static_cast<float>(high), 256.0f, static_cast<float>(low)); }
+
+// The sixteen 6-bit fields of one header row: sc[j], m[j], j = 0..7 (see the unit layout).
+struct RowScales {
+  float d, dmin;
+  uint32_t f[4];   // f[t] = sc_t | sc_{t+4} << 6 | m_t << 12 | m_{t+4} << 18
+  __device__ __forceinline__ int sc(int j) const { return (f[j & 3] >> (j < 4 ? 0 : 6)) & 63u; }
+  __device__ __forceinline__ int m(int j) const { return (f[j & 3] >> (j < 4 ? 12 : 18)) & 63u; }
+};
+__device__ __forceinline__ RowScales decode_row(const uint4& h) {
+  RowScales r;
+  const float2 df = __half22float2(*reinterpret_cast<const __half2*>(&h.x));
+  r.d = df.x;
+  r.dmin = df.y;
+  r.f[0] = h.y & 0xffffffu;
+  r.f[1] = h.z & 0xffffffu;
+  r.f[2] = h.w & 0xffffffu;
+  r.f[3] = (h.y >> 24) | ((h.z >> 24) << 8) | ((h.w >> 24) << 16);
+  return r;
+}
+
+// Quantise the warp's 256 staged activations of one token with one step for all of them; lane l
+// holds quarter l % 4 of sub-block l / 4 as in quantise_lane; `sum` is the sub-block's sum of x_q.
+__device__ __forceinline__ LaneQuant quantise_lane_column(const float (&v)[8]) {
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  const bool ok = amax > 0.f && amax < 3.0e38f;
+  const float inv_step = ok ? 32639.0f / amax : 0.f;
+  int sum = 0;
+  uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    int xq = __float2int_rn(v[i] * inv_step);
+    xq = max(-32639, min(32639, xq));
+    sum += xq;
+    const int l = ((xq + 128) & 255) - 128;      // signed low byte
+    const int h = (xq - l) >> 8;                 // signed high byte, |h| <= 127
+    hi[i & 1] |= (static_cast<uint32_t>(h) & 0xffu) << (8 * (i >> 1));
+    lo[i & 1] |= (static_cast<uint32_t>(l) & 0xffu) << (8 * (i >> 1));
+  }
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+  LaneQuant r;
+  r.q = make_uint4(hi[0], hi[1], lo[0], lo[1]);
+  r.step = ok ? amax / 32639.0f : 0.f;
+  r.sum = sum;
+  return r;
+}
+
+size_t gemv_tokens_smem_bytes(int sg) {
+  return static_cast<size_t>(sg) * kRingTok * kBatchBytes + static_cast<size_t>((sg * kRingTok + 15) & ~15) * 8 +   // ring, mbarriers
+         static_cast<size_t>(2) * kMaxWarps * kBatch * kRowsPerTile * kTokCols * sizeof(float) +                    // reduction buffer
+         static_cast<size_t>(kMaxWarps) * kTokCols * sizeof(float);                                                  // sums of squares
+}
+
+__global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const GemvParams P) {
+  pdl_trigger();
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int n_warps = blockDim.x >> 5;
+  const uint8_t* __restrict__ w = P.w;
+  const int n_rt = P.n_rt, n_sb = P.n_sb, sg = P.sg, n_tok = P.n_tok_total;
+  acc_t* __restrict__ acc_out = P.acc;
+  const int64_t mpad = P.mpad;
+  int* __restrict__ status = P.status;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + static_cast<size_t>(n_warps) * kRingTok * kBatchBytes);
+  float* red = reinterpret_cast<float*>(bars + ((n_warps * kRingTok + 15) & ~15));       // [2][warps][kBatch][8 rows][8 tokens]
+  float* s_red = red + 2 * kMaxWarps * kBatch * kRowsPerTile * kTokCols;                 // [warps][8 tokens]
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+
+  // fixed, even shares as in the one-token kernel
+  const int n_groups = n_sb / sg;
+  const int n_pos = n_groups * n_rt;
+  int p0 = 0, p1 = 0;
+  const int per_group = gridDim.x / n_groups;
+  if (per_group >= 1) {
+    const int grp = blockIdx.x % n_groups, i = blockIdx.x / n_groups;
+    if (i < per_group) {
+      p0 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * i / per_group);
+      p1 = grp * n_rt + static_cast<int>(static_cast<int64_t>(n_rt) * (i + 1) / per_group);
+    }
+  } else {
+    p0 = static_cast<int>(static_cast<int64_t>(n_pos) * blockIdx.x / gridDim.x);
+    p1 = static_cast<int>(static_cast<int64_t>(n_pos) * (blockIdx.x + 1) / gridDim.x);
+  }
+  auto clear_arrays = [&]() {
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < P.zero0_n; i += stride) P.zero0[i] = 0;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < P.zero1_n; i += stride) P.zero1[i] = 0;
+  };
+  if (p0 >= p1) {
+    pdl_wait();
+    clear_arrays();
+    return;
+  }
+
+  uint8_t* my_ring = smem + static_cast<size_t>(warp) * kRingTok * kBatchBytes;
+  const uint32_t ring_u32 = smem_addr(my_ring);
+  const uint32_t bar_u32 = smem_addr(bars + warp * kRingTok);
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < kRingTok; ++i) mbar_init(bar_u32 + 8 * i, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  Walk pf, cur;
+  cur.init(p0, p1, n_rt);
+  int n_in_flight = 0;
+  int rslot = 0;
+  auto request = [&]() {
+    const int nb = pf.batch();
+    if (lane == 0) {
+      const uint8_t* src = w + (static_cast<int64_t>(pf.grp * sg + warp) * n_rt + pf.rt) * kUnitBytes;
+      mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
+      bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot, stream_once_policy());
+    }
+    pf.next(nb);
+    ++n_in_flight;
+    if (++rslot == kRingTok) rslot = 0;
+  };
+
+  // B operands of the lane: token g, sub-block j: high or low bytes of the even or odd weights of
+  // quarter t.  For the lane's output tokens 2t and 2t+1: the sums of x_q per sub-block and the step.
+  uint32_t x_he[8], x_ho[8], x_le[8], x_lo[8];
+  int sumx[2][8];
+  float step[2];
+  int parity = 0;
+  bool alive = true;
+  bool waited = false;
+  int slot = 0;
+  uint32_t phase = 0;
+  constexpr uint32_t E = 0x0f0f0f0fu;
+
+  while (!cur.done()) {
+    // ---- a segment.  The ring is empty: all slots but the one that follows (in ring order) the last
+    //      requested one are requested now; that one serves as the activation buffer first.
+    const int seg_end = min(p1, (cur.grp + 1) * n_rt);
+    pf.init(cur.pos, seg_end, n_rt);
+#pragma unroll
+    for (int i = 0; i < kRingTok - 1; ++i)
+      if (!pf.done()) request();
+    if (!waited) {
+      pdl_wait();
+      waited = true;
+      clear_arrays();
+    }
+    {
+      // the slot that the next request will fill: [token][lane] 16 bytes (hi even, hi odd, lo even,
+      // lo odd of a quarter sub-block), [token][sub-block] sums of x_q, [token] steps
+      uint4* xs_q = reinterpret_cast<uint4*>(my_ring + rslot * kBatchBytes);
+      int* xs_sum = reinterpret_cast<int*>(xs_q + kTokCols * 32);
+      float* xs_step = reinterpret_cast<float*>(xs_sum + kTokCols * 8);
+      auto publish = [&](int k, const LaneQuant& lq, float ssv, bool live) {
+        xs_q[k * 32 + lane] = lq.q;
+        if (t == 0) xs_sum[k * 8 + g] = lq.sum;
+        if (lane == 0) xs_step[k] = lq.step;
+        if (P.kind == kResidual && live) {
+          float a = ssv;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+          if (lane == 0) s_red[warp * kTokCols + k] = a;
+        }
+      };
+      LaneQuant zero;
+      zero.q = make_uint4(0, 0, 0, 0);
+      zero.step = 0.f;
+      zero.sum = 0;
+      for (int k = 0; k < kTokCols; k += 2) {      // two tokens per round trip
+        if (k + 1 < n_tok) {
+          float v[2][8];
+          float ss2[2];
+          stage_warp<2>(P, cur.grp * sg + warp, k, v, ss2);
+          publish(k, quantise_lane_column(v[0]), ss2[0], true);
+          publish(k + 1, quantise_lane_column(v[1]), ss2[1], true);
+        } else if (k < n_tok) {
+          float v[1][8];
+          float ss1[1];
+          stage_warp<1>(P, cur.grp * sg + warp, k, v, ss1);
+          publish(k, quantise_lane_column(v[0]), ss1[0], true);
+          publish(k + 1, zero, 0.f, false);
+        } else {
+          publish(k, zero, 0.f, false);
+          publish(k + 1, zero, 0.f, false);
+        }
+      }
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint4 q = xs_q[g * 32 + 4 * j + t];
+        x_he[j] = q.x; x_ho[j] = q.y; x_le[j] = q.z; x_lo[j] = q.w;
+        sumx[0][j] = xs_sum[(2 * t) * 8 + j];
+        sumx[1][j] = xs_sum[(2 * t + 1) * 8 + j];
+      }
+      step[0] = xs_step[2 * t];
+      step[1] = xs_step[2 * t + 1];
+      __syncwarp();
+      // the generic-proxy reads of the buffer are done; order them before the copy that overwrites it
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (!pf.done()) request();
+    }
+    if (P.kind == kResidual) {
+      __syncthreads();
+      if (threadIdx.x < n_tok) {
+        float a = 0.f;
+        for (int ww = 0; ww < n_warps; ++ww) a += s_red[ww * kTokCols + threadIdx.x];
+        P.ssq_out[threadIdx.x * kMaxStatBlocks + cur.grp] = a;
+      }
+      __syncthreads();
+    }
+    while (cur.pos < seg_end) {
+      const int nb = cur.batch();
+      if (alive && !mbar_wait(bar_u32 + 8 * slot, phase)) {
+        alive = false;
+        if (lane == 0) atomicExch(status, 1);
+      }
+      --n_in_flight;
+      const uint8_t* base = my_ring + slot * kBatchBytes;
+      float* red_w = red + ((parity * kMaxWarps + warp) * kBatch) * kRowsPerTile * kTokCols;
+#pragma unroll 1
+      for (int pr = 0; pr < kBatch / 2; ++pr) {
+        if (2 * pr >= nb) break;
+        const uint8_t* u0 = base + (2 * pr) * kUnitBytes;
+        const uint8_t* u1 = u0 + kUnitBytes;
+        const RowScales r0 = decode_row(*reinterpret_cast<const uint4*>(u0 + g * 16));
+        const RowScales r1 = decode_row(*reinterpret_cast<const uint4*>(u1 + g * 16));
+        // word t of (row g, sub-block j), j = 0..7, for both tiles: four matrix loads, each of which
+        // reads the 16-byte pieces of rows 0..7 for four sub-blocks and hands lane (g, t) bytes 4t..4t+3
+        const uint32_t piece = static_cast<uint32_t>(kUnitHdrBytes + ((lane & 7) * 4 + (lane >> 3)) * 16);
+        const uint32_t a_u0 = smem_addr(u0) + piece, a_u1 = smem_addr(u1) + piece;
+        int accH[4] = {0, 0, 0, 0}, accL[4] = {0, 0, 0, 0};   // sum_j sc_j * (high, low sums)   [row g / g+8][token 2t / 2t+1]
+        int accM[4] = {0, 0, 0, 0};                           // sum_j m_j sum(x_q)_j
+        uint32_t w0[4], w1[4];   // sub-blocks 4 (j / 4) .. + 3 of tile 2 pr / 2 pr + 1
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if ((j & 3) == 0) {
+            ldmatrix_x4(w0[0], w0[1], w0[2], w0[3], a_u0 + 512 * (j >> 2));
+            ldmatrix_x4(w1[0], w1[1], w1[2], w1[3], a_u1 + 512 * (j >> 2));
+          }
+          int dh[4] = {0, 0, 0, 0}, dl[4] = {0, 0, 0, 0};
+          const uint32_t a0 = w0[j & 3] & E, a1 = w1[j & 3] & E, a2 = (w0[j & 3] >> 4) & E, a3 = (w1[j & 3] >> 4) & E;
+          mma_u8s8(dh, a0, a1, a2, a3, x_he[j], x_ho[j]);
+          mma_u8s8(dl, a0, a1, a2, a3, x_le[j], x_lo[j]);
+          const int sc0 = r0.sc(j), sc1 = r1.sc(j), m0 = r0.m(j), m1 = r1.m(j);
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            accH[c] += sc0 * dh[c];
+            accL[c] += sc0 * dl[c];
+            accH[2 + c] += sc1 * dh[2 + c];
+            accL[2 + c] += sc1 * dl[2 + c];
+            accM[c] += m0 * sumx[c][j];
+            accM[2 + c] += m1 * sumx[c][j];
+          }
+        }
+        // rows g of tiles 2 pr and 2 pr + 1, tokens 2t and 2t+1
+        *reinterpret_cast<float2*>(red_w + ((2 * pr) * kRowsPerTile + g) * kTokCols + 2 * t) =
+            make_float2(step[0] * (r0.d * scaled_sum(accH[0], accL[0]) - r0.dmin * static_cast<float>(accM[0])),
+                        step[1] * (r0.d * scaled_sum(accH[1], accL[1]) - r0.dmin * static_cast<float>(accM[1])));
+        *reinterpret_cast<float2*>(red_w + ((2 * pr + 1) * kRowsPerTile + g) * kTokCols + 2 * t) =
+            make_float2(step[0] * (r1.d * scaled_sum(accH[2], accL[2]) - r1.dmin * static_cast<float>(accM[2])),
+                        step[1] * (r1.d * scaled_sum(accH[3], accL[3]) - r1.dmin * static_cast<float>(accM[3])));
+      }
+      // the whole warp has consumed the slot: hand it back and request the next batch
+      __syncwarp();
+      if (alive && !pf.done()) request();
+      __syncthreads();
+      // warp-ordered sum of the SG warps' partials: thread = (tile of the batch, row, token)
+      for (int idx = threadIdx.x; idx < kBatch * kRowsPerTile * kTokCols; idx += blockDim.x) {
+        const int i = idx / (kRowsPerTile * kTokCols);
+        const int row = (idx / kTokCols) % kRowsPerTile;
+        const int tok = idx % kTokCols;
+        if (i < nb && tok < n_tok) {
+          const float* src = red + (parity * kMaxWarps * kBatch) * kRowsPerTile * kTokCols + idx;
+          float sum = src[0];
+          for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile * kTokCols];
+          if (!(fabsf(sum) < kAccLimit)) atomicExch(status, 2);
+          atomicAdd(acc_out + static_cast<int64_t>(tok) * mpad + acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row), acc_from(sum));
+        }
+      }
+      parity ^= 1;
+      if (++slot == kRingTok) {
+        slot = 0;
+        phase ^= 1u;
+      }
+      cur.next(nb);
+    }
+  }
+  if (!alive) {
+    for (int i = 0; i < n_in_flight && i < kRingTok; ++i) {
+      mbar_wait(bar_u32 + 8 * slot, phase);
+      if (++slot == kRingTok) {
+        slot = 0;
+        phase ^= 1u;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gemv_tokens(const gemv_detail::GemvParams& P, int64_t grid, cudaStream_t st) {
+  static bool configured[kMaxDevices] = {};
+  int dev = -1;
+  if (first_launch_on_device(configured, &dev)) {
+    const cudaError_t e = cudaFuncSetAttribute(gemv_tokens_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(gemv_tokens_smem_bytes(kMaxWarps)));
+    if (e != cudaSuccess) return e;
+    if (dev >= 0) configured[dev] = true;
+  }
+  return launch_pdl(gemv_tokens_kernel, dim3(static_cast<unsigned>(grid)), dim3(P.sg * 32), gemv_tokens_smem_bytes(P.sg), st, P);
+}
+
+}  // namespace prima
