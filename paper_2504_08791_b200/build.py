@@ -46,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.returncode != 0:
             raise RuntimeError("nvcc failed on %s:\n%s" % (src, out))
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.run([_nvcc(), "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
+    subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
     os.replace(tmp, LIB)
     with open(os.path.join(HERE, "_build", "ptxas.log"), "w") as f:
         f.write("\n".join(log))
