@@ -440,17 +440,18 @@ static int forward_window_impl(prima_ctx* c, int layer_begin, int layer_end, con
                launch_attention(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k, L.v, g.kv_capacity, H, G, pos0, n_tok,
                                 c->attn, c->obuf, c->sm_count, st), "attention");
     } else {
-      for (int t = 0; t < n_tok; ++t) {          // one request per token: its own cache, its own position
-        __half *kc = nullptr, *vc = nullptr;
-        const int rc = ensure_kv_seq(c, l, seq[t], &kc, &vc);
+      AttnSeqs as;                               // one request per token: its own cache, its own position
+      as.n = n_tok;
+      int64_t kv_bytes = 0;
+      for (int t = 0; t < n_tok; ++t) {
+        const int rc = ensure_kv_seq(c, l, seq[t], &as.k[t], &as.v[t]);
         if (rc != PRIMA_OK) return rc;
-        SumSq ssq_t = c->ssq_attn;
-        ssq_t.data += t * kMaxStatBlocks;
-        LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos[t] + 1),
-                 launch_attention(c->acc_qkv + t * L.qkv.mpad(), L.qkv.mpad(), ssq_t, c->rope_tab + t * (kHeadDim / 2), g.rope_mode, kc, vc,
-                                  g.kv_capacity, H, G, pos[t], 1, c->attn, c->obuf + static_cast<int64_t>(t) * H * kHeadDim, c->sm_count, st),
-                 "attention");
+        as.pos[t] = pos[t];
+        kv_bytes += static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos[t] + 1);
       }
+      LAUNCH_P(c, PRIMA_PROF_ATTENTION, kv_bytes,
+               launch_attention_seqs(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, as, g.kv_capacity, H, G, c->attn, c->obuf,
+                                     c->sm_count, st), "attention");
     }
     GemvIn in_o;                                 // O: plain attention output
     in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status;

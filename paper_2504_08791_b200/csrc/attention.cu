@@ -60,9 +60,23 @@ __device__ __forceinline__ int swz(int dim) { return dim ^ (((dim >> 5) & 1) << 
 __global__ void __launch_bounds__(kThreads, 2)
 attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
                     const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
-                    int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks, float* __restrict__ o_part,
-                    float2* __restrict__ ml_part) {
+                    int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks, int chunk_stride,
+                    float* __restrict__ o_part, float2* __restrict__ ml_part, const AttnSeqs seqs) {
   pdl_trigger();
+  int row_base = 0;                 // first output row (token * heads) of this CTA's token(s)
+  if (seqs.n > 0) {                 // one request per blockIdx.z: its own cache and position, one token
+    const int tq = blockIdx.z;
+    k_cache = seqs.k[tq];
+    v_cache = seqs.v[tq];
+    pos = seqs.pos[tq];
+    n_tok = 1;
+    n_chunks = (pos + kChunk) / kChunk;
+    if (static_cast<int>(blockIdx.x) >= n_chunks) return;
+    acc += tq * mpad;
+    ssq += tq * kMaxStatBlocks;
+    rope_tab += tq * (kHeadDim / 2);
+    row_base = tq * n_q_heads;
+  }
   extern __shared__ __align__(16) float dyn_smem[];
   __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
   __shared__ float s_inv[kMaxTok];
@@ -346,7 +360,7 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
         }
         const int rr = tile * 16 + r;
         const int tok = rr / group, head = kv * group + rr % group;
-        const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * n_chunks + chunk;
+        const int64_t slot = (static_cast<int64_t>(row_base) + static_cast<int64_t>(tok) * n_q_heads + head) * chunk_stride + chunk;
         *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
         if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
       }
@@ -359,16 +373,18 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
 // head dim d.  The partial outputs of the first kMergePre chunks are requested before anything
 // else, together with the (max, sum) pairs, so that the kernel costs one round trip to L2.
 __global__ void __launch_bounds__(kHeadDim)
-attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks, float* __restrict__ o) {
+attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks, int chunk_stride, int n_q_heads,
+                  float* __restrict__ o, const AttnSeqs seqs) {
   pdl_trigger();
   pdl_wait();
+  if (seqs.n > 0) n_chunks = (seqs.pos[blockIdx.x / n_q_heads] + kChunk) / kChunk;      // the row's own request
   extern __shared__ float s_w[];         // [n_chunks] weights e^(m_c - M), then [n_chunks] weights times l_c
   float* s_wl = s_w + n_chunks;
   __shared__ float s_red[4];
   const int row = blockIdx.x;            // tok * H + head
   const int d = threadIdx.x;
-  const float2* ml = ml_part + static_cast<int64_t>(row) * n_chunks;
-  const float* op = o_part + static_cast<int64_t>(row) * n_chunks * kHeadDim + d;
+  const float2* ml = ml_part + static_cast<int64_t>(row) * chunk_stride;
+  const float* op = o_part + static_cast<int64_t>(row) * chunk_stride * kHeadDim + d;
   float pre[kMergePre];
 #pragma unroll
   for (int c = 0; c < kMergePre; ++c)
@@ -410,13 +426,7 @@ size_t partial_smem_bytes(int n_rows, int n_tok) {
 
 int attention_chunk_len() { return kChunk; }
 
-int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, __half* k_cache,
-                     __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, const AttnScratch& scr, float* o,
-                     int sm_count, cudaStream_t st) {
-  const int n_ctx = pos + n_tok;
-  const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
-  if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
-  const int n_rows = n_tok * (n_q_heads / n_kv_heads);
+static int configure_partial_kernel() {
   static bool configured[kMaxDevices] = {};
   int dev = -1;
   if (first_launch_on_device(configured, &dev)) {
@@ -426,16 +436,51 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
     if (e0 != cudaSuccess) return cuda_rc(e0);
     if (dev >= 0) configured[dev] = true;
   }
+  return 0;
+}
+
+int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, __half* k_cache,
+                     __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, const AttnScratch& scr, float* o,
+                     int sm_count, cudaStream_t st) {
+  const int n_ctx = pos + n_tok;
+  const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
+  if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
+  const int n_rows = n_tok * (n_q_heads / n_kv_heads);
+  const int rc = configure_partial_kernel();
+  if (rc != 0) return rc;
   // Two CTAs fit on an SM: with more chunks than that, a CTA takes several (gridDim.x apart).
   const int per_head = std::max(1, 2 * sm_count / n_kv_heads);
   dim3 grid(std::min(n_chunks, per_head), n_kv_heads);
+  const AttnSeqs none{};
   cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), partial_smem_bytes(n_rows, n_tok), st, acc_qkv, mpad,
                              static_cast<const float*>(ssq.data), ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f,
                              ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok, n_chunks,
-                             scr.o_part, scr.ml_part);
+                             n_chunks, scr.o_part, scr.ml_part, none);
   if (e != cudaSuccess) return cuda_rc(e);
   e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * n_chunks) * sizeof(float), st,
-                 scr.o_part, scr.ml_part, n_chunks, o);
+                 scr.o_part, scr.ml_part, n_chunks, n_chunks, n_q_heads, o, none);
+  if (e != cudaSuccess) return cuda_rc(e);
+  return 2;
+}
+
+int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, const AttnSeqs& seqs,
+                          int kv_capacity, int n_q_heads, int n_kv_heads, const AttnScratch& scr, float* o, int sm_count, cudaStream_t st) {
+  if (seqs.n < 1 || seqs.n > kMaxTok) return cuda_rc(cudaErrorInvalidValue);
+  int max_chunks = 1;
+  for (int t = 0; t < seqs.n; ++t) max_chunks = std::max(max_chunks, (seqs.pos[t] + kChunk) / kChunk);
+  if (max_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
+  const int rc = configure_partial_kernel();
+  if (rc != 0) return rc;
+  const int group = n_q_heads / n_kv_heads;
+  const int per_head = std::max(1, 2 * sm_count / n_kv_heads);
+  dim3 grid(std::min(max_chunks, per_head), n_kv_heads, seqs.n);      // CTAs beyond a request's own chunks leave at once
+  cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), partial_smem_bytes(group, 1), st, acc_qkv, mpad,
+                             static_cast<const float*>(ssq.data), ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f,
+                             ssq.eps, rope_tab, rope_mode, static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads,
+                             n_kv_heads, 0, 1, max_chunks, max_chunks, scr.o_part, scr.ml_part, seqs);
+  if (e != cudaSuccess) return cuda_rc(e);
+  e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * max_chunks) * sizeof(float), st,
+                 scr.o_part, scr.ml_part, max_chunks, max_chunks, n_q_heads, o, seqs);
   if (e != cudaSuccess) return cuda_rc(e);
   return 2;
 }

@@ -163,6 +163,17 @@ struct AttnScratch {
   float2* ml_part;  // [n_tok*H][n_chunks]  (running max, running sum)
   int max_chunks;
 };
+// Several independent requests in one launch: token t of the step belongs to a request with its own
+// cache (k[t], v[t]) and position pos[t]; rows, statistics, rotary table and outputs of token t are
+// the t-th slices of the arrays that launch_attention takes.
+struct AttnSeqs {
+  __half* k[kMaxTok];
+  __half* v[kMaxTok];
+  int pos[kMaxTok];
+  int n = 0;
+};
+int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, const AttnSeqs& seqs,
+                          int kv_capacity, int n_q_heads, int n_kv_heads, const AttnScratch& scr, float* o, int sm_count, cudaStream_t st);
 int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode,
                      __half* k_cache, __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok,
                      const AttnScratch& scr, float* o, int sm_count, cudaStream_t st);
