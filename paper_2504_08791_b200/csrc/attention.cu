@@ -20,6 +20,9 @@
 // the cache and keeps a copy in shared memory, from which its warps take them (the cache is never
 // read back inside the kernel).
 //
+// With several independent requests per step (one token each) the grid gets a third dimension: CTA
+// (chunk, KV head, request) works on that request's own cache and position, all in one launch.
+//
 // Latency matters more than bandwidth here (the whole cache of a layer is a few microseconds of
 // HBM time): every warp requests the old entries of its positions before it waits for the
 // predecessor kernel, all loads of the finishing step are issued together, and the shared-memory
