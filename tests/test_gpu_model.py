@@ -114,6 +114,26 @@ def test_window_splits_are_bit_identical_on_the_gpu(gpu, splits, n_tok):
     part.close()
 
 
+@pytest.mark.parametrize("over,pos,n_tok", [
+    (dict(rope_mode=1), 70, 1),                                             # interleaved rotation pairs
+    (dict(rope_mode=1), 129, 6),                                            # ... on the multi-token kernels
+    (dict(n_q_heads=2, n_kv_heads=2, hidden=256), 33, 1),                   # no grouping, one super-block column
+    (dict(n_q_heads=8, n_kv_heads=1, hidden=1024), 200, 3),                 # one KV head for eight query heads
+    (dict(n_q_heads=10, n_kv_heads=2, hidden=1280, ffn=1280), 127, 1),      # five query heads per KV head, column groups of 5
+    (dict(n_q_heads=10, n_kv_heads=2, hidden=1280, ffn=1280), 128, 7),
+    (dict(n_q_heads=4, n_kv_heads=4, hidden=512, ffn=3328, vocab=1000), 0, 2),   # 13 super-block columns (prime), vocab not a multiple of 8
+])
+def test_unusual_shapes_match_checker(gpu, over, pos, n_tok):
+    cfg = synth.model_config("small", **over)
+    p = Pair(gpu, cfg, seed=37, n_prefill=pos)
+    h0 = synth.activations(37, n_tok, cfg["hidden"])
+    want = p.ref.forward_window(0, cfg["n_layers"], h0, pos)
+    got = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    _hidden_close(got, want)
+    assert np.abs(p.gpu_logits(got).astype(np.float64) - p.ref.logits(want)).max() <= LOGIT_TOL
+    p.close()
+
+
 @pytest.mark.parametrize("sizes", [[1, 2], [2, 1], [1, 1, 1]])
 def test_ring_schedule_with_uneven_windows_is_bit_identical_to_one_pass(gpu, sizes):
     """The paper's ring schedule (devices take w_m layers per turn, several rounds) executed window by
