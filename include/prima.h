@@ -160,7 +160,8 @@ int prima_kv_read_seq(prima_ctx* ctx, int seq, int layer, int pos_begin, int n_p
 
 /* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word (a
  * partial sum outside the accumulator range, or a bounded wait inside a kernel that gave up) and
- * PRIMA_ERR_CUDA if the stream reports an error. */
+ * PRIMA_ERR_CUDA if the stream reports an error.  A raised status word is reported once and
+ * cleared: the context can go on with the next step. */
 int prima_sync(prima_ctx* ctx);
 
 /* Text of the most recent error of this context (never NULL; "" if none).  With ctx == NULL,

@@ -631,6 +631,7 @@ int prima_sync(prima_ctx* c) {
   cudaError_t e = cudaMemcpyAsync(&status, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync");
+  if (status != 0) cudaMemsetAsync(c->status, 0, sizeof(int), c->stream);      // reported once; the context stays usable
   if (status != 0)
     return fail(c, PRIMA_ERR_DEVICE, status == 2 ? "a partial sum was outside the accumulator range (+-2^27); results of this step are invalid"
                                                  : "a bounded wait inside a kernel gave up (status " + std::to_string(status) + ")");

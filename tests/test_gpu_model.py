@@ -234,3 +234,21 @@ def test_errors_leave_the_context_usable(gpu):
     ctx.sync()
     assert ctx.launch_count() > 0
     ctx.close()
+
+
+def test_sums_outside_the_accumulator_range_are_reported_once(gpu):
+    torch, binding = gpu
+    cfg = synth.model_config("tiny")
+    p = Pair(gpu, cfg, seed=41, n_prefill=10)
+    h0 = synth.activations(41, 1, cfg["hidden"])
+    good = p.gpu_window(0, cfg["n_layers"], h0, 10)
+    hin = torch.from_numpy(h0 * 1e12).cuda()            # products of the first projection far beyond 2^27
+    hout = torch.empty_like(hin)
+    p.ctx.forward_window(0, cfg["n_layers"], hin, hout, 10, 1)
+    with pytest.raises(binding.PrimaError) as err:
+        p.ctx.sync()
+    assert err.value.code == binding.ERR_DEVICE
+    p.ctx.sync()                                        # reported once
+    again = p.gpu_window(0, cfg["n_layers"], h0, 10)    # and the context computes the same bits as before
+    assert np.array_equal(again.view(np.uint32), good.view(np.uint32))
+    p.close()
