@@ -252,3 +252,17 @@ def test_sums_outside_the_accumulator_range_are_reported_once(gpu):
     again = p.gpu_window(0, cfg["n_layers"], h0, 10)    # and the context computes the same bits as before
     assert np.array_equal(again.view(np.uint32), good.view(np.uint32))
     p.close()
+
+
+@pytest.mark.parametrize("n_tok", [1, 3])
+def test_long_context_with_more_chunks_than_resident_ctas(gpu, n_tok):
+    """19,100 cached positions on a model with two KV heads: 150 chunks per head, more than the 148 CTAs per
+    head that the grid gets, so CTAs take a second chunk, and the merge sees more chunks than it has threads."""
+    cfg = synth.model_config("tiny", kv_capacity=19200)
+    pos = 19100
+    p = Pair(gpu, cfg, seed=43, n_prefill=pos)
+    h0 = synth.activations(43, n_tok, cfg["hidden"])
+    want = p.ref.forward_window(0, cfg["n_layers"], h0, pos)
+    got = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    _hidden_close(got, want)
+    p.close()
