@@ -20,6 +20,9 @@
 // the cache and keeps a copy in shared memory, from which its warps take them (the cache is never
 // read back inside the kernel).
 //
+// With at most eight query rows (one token) a CTA that takes several chunks carries its running state
+// from chunk to chunk and leaves one partial result (see the first branch of the chunk loop).
+//
 // With several independent requests per step (one token each) the grid gets a third dimension: CTA
 // (chunk, KV head, request) works on that request's own cache and position, all in one launch.
 //
@@ -221,6 +224,134 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   __syncthreads();
 
   const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
+  if (n_rows <= 8) {
+    // ---- At most eight query rows (one token): one tile, and a CTA that takes several chunks carries
+    //      its running (max, sum, output) from chunk to chunk instead of leaving one partial result per
+    //      chunk.  A warp keeps the un-normalised output of its positions in its own tile in shared memory
+    //      (every lane re-reads and re-writes only its own 32 floats, so the chunk loop has no barrier and
+    //      the warps' loads and arithmetic overlap freely); the warps are combined once, at the end, and
+    //      the CTA leaves ONE partial result, numbered by blockIdx.x.
+    const bool live = g < n_rows;
+    const int my_tok = live ? g / group : -1;
+    const float* qrow = q_s + (live ? g : 0) * kRowPad;
+    float* so = s_o + (warp * o_rows + g) * kRowPad;
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) *reinterpret_cast<float4*>(so + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+    float m_run = -INFINITY, l_run = 0.f;      // of row g, the same in the four lanes of a quad
+    for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
+      const int wbase = chunk * kChunk + warp * 16;
+      if (!first) load_old(wbase);
+      patch_new(wbase);
+      float sc[2][4];
+#pragma unroll
+      for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (live) {
+          a = *reinterpret_cast<const float4*>(qrow + swz(32 * j + 8 * t));
+          b = *reinterpret_cast<const float4*>(qrow + swz(32 * j + 8 * t) + 4);
+        }
+        const uint32_t qa0 = pack_h2(a.x * scale, a.y * scale), qa2 = pack_h2(a.z * scale, a.w * scale);
+        const uint32_t qb0 = pack_h2(b.x * scale, b.y * scale), qb2 = pack_h2(b.z * scale, b.w * scale);
+#pragma unroll
+        for (int pb = 0; pb < 2; ++pb) {      // rows 8..15 of the tile do not exist: zero operands
+          mma_f16(sc[pb], qa0, 0u, qa2, 0u, kreg[pb][j].x, kreg[pb][j].y);
+          mma_f16(sc[pb], qb0, 0u, qb2, 0u, kreg[pb][j].z, kreg[pb][j].w);
+        }
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int pb = 0; pb < 2; ++pb)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int p = wbase + 8 * pb + 2 * t + e;
+          const bool ok = live && p <= pos + my_tok;
+          sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
+          mx = fmaxf(mx, sc[pb][e]);
+        }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m_run, mx);
+      const float alpha = m_run > -INFINITY ? expf(m_run - m_new) : 1.0f;      // nothing accumulated yet: the tile is zero
+      float lsum = 0.f;
+      uint32_t pa[2];
+#pragma unroll
+      for (int pb = 0; pb < 2; ++pb) {
+        const float p0 = m_new > -INFINITY ? expf(sc[pb][0] - m_new) : 0.f;
+        const float p1 = m_new > -INFINITY ? expf(sc[pb][1] - m_new) : 0.f;
+        lsum += p0 + p1;
+        pa[pb] = pack_h2(p0, p1);
+      }
+      lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+      lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+      l_run = l_run * alpha + lsum;
+      m_run = m_new;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+        for (int bh = 0; bh < 2; ++bh) {
+          float oc[4][4];
+#pragma unroll
+          for (int bb = 0; bb < 4; ++bb) {
+            const int b = 4 * bh + bb, j = b >> 1;
+            const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
+            const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
+            const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
+            const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
+            const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
+            const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
+            const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
+            oc[bb][0] = oc[bb][1] = oc[bb][2] = oc[bb][3] = 0.f;
+            mma_f16(oc[bb], pa[0], 0u, pa[1], 0u, b0, b1);
+          }
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            float4* dst = reinterpret_cast<float4*>(so + swz(64 * hf + 16 * t + 8 * e + 4 * bh));
+            const float4 old = *dst;
+            *dst = make_float4(fmaf(old.x, alpha, oc[0][e]), fmaf(old.y, alpha, oc[1][e]), fmaf(old.z, alpha, oc[2][e]), fmaf(old.w, alpha, oc[3][e]));
+          }
+        }
+      }
+    }
+    if (t == 0) {
+      s_m[warp][g] = m_run;
+      s_l[warp][g] = l_run;
+      s_m[warp][g + 8] = -INFINITY;
+      s_l[warp][g + 8] = 0.f;
+    }
+    __syncthreads();
+    if (threadIdx.x < kWarps * 16) {
+      const int w = threadIdx.x >> 4, r = threadIdx.x & 15;
+      float big = -INFINITY;
+#pragma unroll
+      for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
+      const float mine = s_m[w][r];
+      s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
+      if (w == 0) s_big[r] = big;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < n_rows * (kHeadDim / 4); idx += kThreads) {
+      const int r = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
+      const int col = swz(d4);
+      float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
+      float l = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const float f = s_f[w][r];
+        const float4 v = *reinterpret_cast<const float4*>(s_o + (w * o_rows + r) * kRowPad + col);
+        l += f * s_l[w][r];
+        accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
+      }
+      const int tok = r / group, head = kv * group + r % group;
+      const int64_t slot = (static_cast<int64_t>(row_base) + static_cast<int64_t>(tok) * n_q_heads + head) * chunk_stride + blockIdx.x;
+      *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
+      if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
+    }
+    return;
+  }
   for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
     const int wbase = chunk * kChunk + warp * 16;      // first position of this warp
     if (!first) load_old(wbase);
@@ -380,7 +511,7 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
                   float* __restrict__ o, const AttnSeqs seqs) {
   pdl_trigger();
   pdl_wait();
-  if (seqs.n > 0) n_chunks = (seqs.pos[blockIdx.x / n_q_heads] + kChunk) / kChunk;      // the row's own request
+  if (seqs.n > 0) n_chunks = min(n_chunks, (seqs.pos[blockIdx.x / n_q_heads] + kChunk) / kChunk);      // the row's own request
   extern __shared__ float s_w[];         // [n_chunks] weights e^(m_c - M), then [n_chunks] weights times l_c
   float* s_wl = s_w + n_chunks;
   __shared__ float s_red[4];
@@ -460,8 +591,10 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
                              ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok, n_chunks,
                              n_chunks, scr.o_part, scr.ml_part, none);
   if (e != cudaSuccess) return cuda_rc(e);
-  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * n_chunks) * sizeof(float), st,
-                 scr.o_part, scr.ml_part, n_chunks, n_chunks, n_q_heads, o, none);
+  // with at most eight query rows a CTA leaves one partial result, however many chunks it took
+  const int n_parts = n_rows <= 8 ? static_cast<int>(grid.x) : n_chunks;
+  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * n_parts) * sizeof(float), st,
+                 scr.o_part, scr.ml_part, n_parts, n_chunks, n_q_heads, o, none);
   if (e != cudaSuccess) return cuda_rc(e);
   return 2;
 }
@@ -483,7 +616,7 @@ int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, 
                              n_kv_heads, 0, 1, max_chunks, max_chunks, scr.o_part, scr.ml_part, seqs);
   if (e != cudaSuccess) return cuda_rc(e);
   e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * max_chunks) * sizeof(float), st,
-                 scr.o_part, scr.ml_part, max_chunks, max_chunks, n_q_heads, o, seqs);
+                 scr.o_part, scr.ml_part, static_cast<int>(grid.x), max_chunks, n_q_heads, o, seqs);
   if (e != cudaSuccess) return cuda_rc(e);
   return 2;
 }

@@ -256,10 +256,11 @@ def test_sums_outside_the_accumulator_range_are_reported_once(gpu):
 
 @pytest.mark.parametrize("n_tok", [1, 3])
 def test_long_context_with_more_chunks_than_resident_ctas(gpu, n_tok):
-    """19,100 cached positions on a model with two KV heads: 150 chunks per head, more than the 148 CTAs per
-    head that the grid gets, so CTAs take a second chunk, and the merge sees more chunks than it has threads."""
-    cfg = synth.model_config("tiny", kv_capacity=19200)
-    pos = 19100
+    """19,100 / 39,000 cached positions on a model with two KV heads: 150 / 305 chunks per head, more than the 148
+    CTAs per head that the grid gets, so CTAs take further chunks, and the merge sees more partial results than it
+    has threads."""
+    cfg = synth.model_config("tiny", kv_capacity=40000)
+    pos = 39000 if n_tok == 1 else 19100               # 305 chunks: three per CTA, carried from chunk to chunk
     p = Pair(gpu, cfg, seed=43, n_prefill=pos)
     h0 = synth.activations(43, n_tok, cfg["hidden"])
     want = p.ref.forward_window(0, cfg["n_layers"], h0, pos)
