@@ -3,8 +3,8 @@
 // Work decomposition.  The matrix is a grid of units (row tile of 8 rows  x  super-block column of
 // 256 weights, 1152 bytes each, see common.cuh) stored column-major.  The n_sb columns are taken in
 // groups of SG adjacent columns (SG = the largest divisor of n_sb that is <= 8); a CTA has SG warps,
-// warp w always works on column  group*SG + w.  The n_groups * n_rt (group, row tile) positions are
-// ordered group-major and cut into one contiguous range per CTA of a persistent grid, so all CTAs
+// warp w always works on column  group*SG + w.  CTA b of a persistent grid (2 CTAs per SM) works for
+// group b mod n_groups and takes an even, contiguous share of that group's row tiles, so all CTAs
 // get the same number of tiles to within one.  A CTA walks its range in batches of up to 4
 // consecutive row tiles of one group (a batch never crosses a group boundary), so each warp's part
 // of a batch is one contiguous piece of HBM of up to 4608 bytes, and the warp keeps its column's
