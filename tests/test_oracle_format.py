@@ -228,3 +228,28 @@ def test_generator_distributions():
     # deterministic, and different tensors differ
     assert np.array_equal(wm, synth.model_tensor(1, 0, synth.WQ, 128, 1024))
     assert not np.array_equal(wm, synth.model_tensor(1, 1, synth.WQ, 128, 1024))
+
+
+def test_dequant_agrees_with_the_gguf_package_decoder_on_random_blocks():
+    """An extra, not a pin: the gguf Python package (when it is installed) decodes the same bytes to the
+    same values, which shows that the layout defined here is the public Q4_K arrangement."""
+    gguf = pytest.importorskip("gguf")
+    from gguf import quants
+    rng = np.random.default_rng(77)
+    n = 300
+    blocks = rng.integers(0, 256, (n, oracle.BLOCK_BYTES), dtype=np.uint8)
+    # keep d and dmin finite: clear the top exponent bit of both halves
+    blocks[:, 1] &= 0xBF
+    blocks[:, 3] &= 0xBF
+    want = quants.dequantize(blocks.reshape(-1), gguf.GGMLQuantizationType.Q4_K).reshape(-1).astype(np.float64)
+    got32 = oracle.q4k_dequant(blocks, np.float32).astype(np.float64)
+    got64 = oracle.q4k_dequant(blocks, np.float64)
+    # the package computes in fp32 with a rounding per operation; this checker rounds the exact value once:
+    # allow 3 units of fp32 rounding on the two terms' magnitudes (they may cancel)
+    mag = np.empty((n, 256))
+    for i in range(n):
+        d, dmin, sc, m = oracle.q4k_fields(blocks[i])
+        mag[i] = (abs(d) * np.repeat(sc, 32) * 15.0 + abs(dmin) * np.repeat(m, 32))
+    tol = 3 * 2.0 ** -24 * mag.reshape(-1) + 1e-40
+    assert np.all(np.abs(want - got64) <= tol)
+    assert np.all(np.abs(want - got32) <= tol)

@@ -56,6 +56,45 @@ def test_rope_unit_vectors_give_cos_and_sin_at_the_paired_index():
         assert abs(out[0] + np.sin(pos)) < 1e-12 and abs(out[D // 2] - np.cos(pos)) < 1e-12
 
 
+def test_rope_interleaved_mode_uses_pair_index_not_element_index_for_the_frequency():
+    """Mode 1 pairs (2i, 2i+1); pair i turns at theta^(-2i/D).  Pair D/4 (elements D/2, D/2+1) at
+    theta = 1e4 turns at exactly 0.01 rad per position, pair 1 (elements 2, 3) at 1e4^(-1/64)."""
+    D, theta = 128, 1e4
+    for pos in (1, 17, 4095):
+        e = np.zeros((2, D))
+        e[0, D // 2] = 1.0           # first element of pair D/4
+        e[1, D // 2 + 1] = 1.0       # its partner
+        out = oracle.rope(e, pos, theta, 1)
+        assert abs(out[0, D // 2] - np.cos(0.01 * pos)) < 1e-12 and abs(out[0, D // 2 + 1] - np.sin(0.01 * pos)) < 1e-12
+        assert abs(out[1, D // 2] + np.sin(0.01 * pos)) < 1e-12 and abs(out[1, D // 2 + 1] - np.cos(0.01 * pos)) < 1e-12
+        assert np.count_nonzero(np.abs(out) > 1e-15) <= 4
+        f1 = theta ** (-2.0 / D)
+        e = np.zeros((1, D))
+        e[0, 2] = 1.0
+        out = oracle.rope(e, pos, theta, 1)[0]
+        assert abs(out[2] - np.cos(f1 * pos)) < 1e-12 and abs(out[3] - np.sin(f1 * pos)) < 1e-12
+        # the last pair is the slowest one
+        fl = theta ** (-2.0 * (D // 2 - 1) / D)
+        e = np.zeros((1, D))
+        e[0, D - 2] = 1.0
+        out = oracle.rope(e, pos, theta, 1)[0]
+        assert abs(out[D - 2] - np.cos(fl * pos)) < 1e-12 and abs(out[D - 1] - np.sin(fl * pos)) < 1e-12
+
+
+def test_rope_modes_are_the_same_rotation_up_to_the_fixed_permutation_of_elements():
+    rng = np.random.default_rng(5)
+    D, theta = 128, 5e5
+    x = rng.normal(0, 1, (4, D))
+    perm = np.empty(D, np.int64)            # element of the interleaved layout that holds split-layout element k
+    perm[:D // 2] = 2 * np.arange(D // 2)
+    perm[D // 2:] = 2 * np.arange(D // 2) + 1
+    y = np.empty_like(x)
+    y[:, perm] = x                           # y in interleaved layout = x in split layout
+    a = oracle.rope(x, 321, theta, 0)
+    b = oracle.rope(y, 321, theta, 1)
+    np.testing.assert_allclose(b[:, perm], a, rtol=0, atol=1e-13)
+
+
 def test_rope_is_identity_at_zero_preserves_norms_and_is_relative():
     rng = np.random.default_rng(1)
     D, theta = 128, 5e5
@@ -168,12 +207,18 @@ def _np_rms(h, g, eps):
     return h / np.sqrt(np.mean(h * h) + eps) * g
 
 
-def _np_rope(x, pos, theta):          # x: [heads, D], pairs (i, i + D/2)
+def _np_rope(x, pos, theta, mode=0):  # x: [heads, D]; mode 0 pairs (i, i + D/2), mode 1 pairs (2i, 2i + 1)
     D = x.shape[1]
     ang = pos * theta ** (-2.0 * np.arange(D // 2) / D)
     c, s = np.cos(ang), np.sin(ang)
-    a, b = x[:, :D // 2], x[:, D // 2:]
-    return np.concatenate([a * c - b * s, b * c + a * s], axis=1)
+    if mode == 0:
+        a, b = x[:, :D // 2], x[:, D // 2:]
+        return np.concatenate([a * c - b * s, b * c + a * s], axis=1)
+    a, b = x[:, 0::2], x[:, 1::2]
+    out = np.empty_like(x)
+    out[:, 0::2] = a * c - b * s
+    out[:, 1::2] = b * c + a * s
+    return out
 
 
 def _np_forward(cfg, dense, h, pos, kv):
@@ -183,8 +228,8 @@ def _np_forward(cfg, dense, h, pos, kv):
     for l in range(cfg["n_layers"]):
         hd = h.astype(np.float64)
         a = _np_rms(hd, dense[(l, synth.ATTN_NORM)], cfg["rms_eps"])
-        q = _np_rope((dense[(l, synth.WQ)] @ a).reshape(H, D), pos, cfg["rope_theta"])
-        k = _np_rope((dense[(l, synth.WK)] @ a).reshape(G, D), pos, cfg["rope_theta"])
+        q = _np_rope((dense[(l, synth.WQ)] @ a).reshape(H, D), pos, cfg["rope_theta"], cfg.get("rope_mode", 0))
+        k = _np_rope((dense[(l, synth.WK)] @ a).reshape(G, D), pos, cfg["rope_theta"], cfg.get("rope_mode", 0))
         v = (dense[(l, synth.WV)] @ a).reshape(G, D)
         K, V = kv[l]
         K[pos] = k.astype(np.float16).astype(np.float64)
@@ -207,8 +252,9 @@ def _np_forward(cfg, dense, h, pos, kv):
 TINY = synth.model_config("tiny")
 
 
-def test_tiny_model_matches_dense_numpy_forward_over_several_tokens():
-    cfg = TINY
+@pytest.mark.parametrize("rope_mode", [0, 1])
+def test_tiny_model_matches_dense_numpy_forward_over_several_tokens(rope_mode):
+    cfg = dict(TINY, rope_mode=rope_mode)
     mdl, dense = _build_explicit_model(cfg, seed=21)
     kv = [({}, {}) for _ in range(cfg["n_layers"])]
     tokens = [3, 700, 41, 5]
