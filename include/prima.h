@@ -125,8 +125,8 @@ int prima_load_q4k_weights(prima_ctx* ctx, int layer, int tensor_id, const void*
 int prima_forward_window(prima_ctx* ctx, int layer_begin, int layer_end, const float* hidden_in,
                          float* hidden_out, int pos, int n_tok);
 
-/* One step of several independent requests (the paper's serving mode: Appendix A.11 "Concurrent
- * requests" / A.12, requests merged per token step, each with its own KV cache).  Token t belongs to
+/* One step of several independent requests (the paper's serving mode: Appendix A.11 "Ablation
+ * Study on Multi-Request Workloads" / A.12, requests merged per token step, each with its own KV cache).  Token t belongs to
  * sequence seq[t] (0..63, each at most once per step) and sits at position pos[t] of that sequence's
  * cache; the projections run over all n_seq tokens together (the weights are read once), attention
  * runs per token over its own sequence's cache, to which the token's K and V are appended.
@@ -160,9 +160,33 @@ int prima_kv_read_seq(prima_ctx* ctx, int seq, int layer, int pos_begin, int n_p
 
 /* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word (a
  * partial sum outside the accumulator range, or a bounded wait inside a kernel that gave up) and
- * PRIMA_ERR_CUDA if the stream reports an error.  A raised status word is reported once and
- * cleared: the context can go on with the next step. */
+ * PRIMA_ERR_CUDA if the stream reports an error.  A raised status word is reported once; the
+ * outputs of the steps queued since the previous prima_sync are then invalid, and before it returns
+ * prima_sync clears the status word and the library's internal accumulators, so the context can go
+ * on with the next step (the KV cache keeps whatever the failed step appended: re-run the step
+ * at the same positions, which overwrites those entries). */
 int prima_sync(prima_ctx* ctx);
+
+/* Failures of prima_forward_window / prima_forward_window_seqs / prima_logits:
+ *   - argument and state errors are found before anything is queued or allocated;
+ *   - PRIMA_ERR_NOMEM of prima_forward_window_seqs (a sequence's cache could not be allocated) is
+ *     also returned before anything is queued: the caches of every (layer, sequence) pair of the
+ *     window are allocated first, the launches follow;
+ *   - PRIMA_ERR_CUDA from a launch in the middle of a window: the kernels queued before it still
+ *     run, hidden_out is not valid, and the library queues the clearing of its accumulators behind
+ *     them, so a later call computes from a clean state. */
+
+/* Options of a context.  PRIMA_OPT_FIRST_WAIT_POLLS (for tests of the failure path): how many
+ * times the first wait of every warp of the streaming kernels polls for its first batch of weights
+ * before it gives up (0: gives up at once); -1 restores the ordinary limit of 2^24 polls.  A wait
+ * that gives up raises the status word (see prima_sync); the kernel still waits, with the
+ * ordinary limit, for every copy it requested before it returns.
+ * PRIMA_OPT_FAIL_AFTER_LAUNCHES (for tests of the failure path, host side only): after `value` more
+ * launch steps of this context the next one is refused with PRIMA_ERR_CUDA as if the runtime had
+ * rejected it (nothing is sent to the GPU for it), once; -1 switches the injection off. */
+#define PRIMA_OPT_FIRST_WAIT_POLLS 1
+#define PRIMA_OPT_FAIL_AFTER_LAUNCHES 2
+int prima_ctx_set_option(prima_ctx* ctx, int option, int64_t value);
 
 /* Text of the most recent error of this context (never NULL; "" if none).  With ctx == NULL,
  * the most recent error of a context-free call on this thread. */
@@ -216,8 +240,11 @@ int prima_gemv_plan_destroy(prima_gemv_plan* plan);
  * Nothing is allocated or freed, here or in anything it calls: the partial sums live in a 16 MiB
  * array built into the library (each GPU that loads the library holds it until exit).  Limit:
  * rows * (cols/256) * n_cols <= 4,194,304; larger products return PRIMA_ERR_ARG with a message
- * that says so.  The first call on a device looks up the array's device address; make that
- * first call before any stream capture begins.  The call queues its kernels on `stream` and
+ * that says so.  The first call on a device looks up the array's device address and remembers it
+ * for that device ordinal; make that first call before any stream capture begins, and with the
+ * CUDA context current that all later calls will use: the address belongs to that context (the
+ * runtime's primary context, normally), so after cudaDeviceReset, or under a different driver-API
+ * context on the same device, the remembered address is stale and this call must not be used.  The call queues its kernels on `stream` and
  * returns without waiting.  All calls on a device share the array: calls whose kernels may
  * overlap on the GPU (different streams without ordering) corrupt each other; calls ordered on a
  * stream, or by events, are safe, and nothing has to be cleared between them.

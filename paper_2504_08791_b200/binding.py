@@ -18,13 +18,15 @@ OK, ERR_ARG, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_DEVICE = 0, -1, -2, -3, -4, -5
 ATTN_NORM, WQ, WK, WV, WO, FFN_NORM, W_GATE, W_UP, W_DOWN, OUT_NORM, W_HEAD, TOK_EMBD = range(12)
 MAX_N_TOK = 8
 PROF_GEMV, PROF_ATTENTION = 0, 1
+OPT_FIRST_WAIT_POLLS = 1
+OPT_FAIL_AFTER_LAUNCHES = 2
 
 EXPORTS = [
     "prima_ctx_create", "prima_ctx_destroy", "prima_load_q4k_weights", "prima_forward_window", "prima_logits",
     "prima_embed", "prima_argmax", "prima_kv_load", "prima_kv_read", "prima_sync", "prima_last_error",
     "prima_launch_count", "prima_profile_enable", "prima_profile_read", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
     "prima_gemv_plan_destroy", "prima_gemv_q4k_noalloc", "prima_gemv_q4k_noalloc_error",
-    "prima_forward_window_seqs", "prima_kv_load_seq", "prima_kv_read_seq",
+    "prima_forward_window_seqs", "prima_kv_load_seq", "prima_kv_read_seq", "prima_ctx_set_option",
 ]
 
 
@@ -65,6 +67,7 @@ def lib():
         L.prima_kv_load_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.prima_kv_read_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.prima_sync.argtypes = [vp]
+        L.prima_ctx_set_option.argtypes = [vp, i32, i64]
         L.prima_last_error.argtypes = [vp]
         L.prima_last_error.restype = C.c_char_p
         L.prima_launch_count.argtypes = [vp]
@@ -221,6 +224,9 @@ class Context:
 
     def sync(self):
         _check(lib().prima_sync(self._h), self._h)
+
+    def set_option(self, option: int, value: int):
+        _check(lib().prima_ctx_set_option(self._h, option, value), self._h)
 
     def profile_enable(self, on: bool):
         _check(lib().prima_profile_enable(self._h, 1 if on else 0), self._h)

@@ -76,6 +76,8 @@ struct prima_ctx {
   std::vector<void*> allocs;
   std::string err;
   int64_t launches = 0;
+  uint32_t first_wait_polls = 0;   // PRIMA_OPT_FIRST_WAIT_POLLS (0: the ordinary limit)
+  int64_t fail_after = -1;         // PRIMA_OPT_FAIL_AFTER_LAUNCHES: launch steps still allowed before an injected failure (-1: off)
 
   // optional per-class device timing (prima_profile_*)
   bool profiling = false;
@@ -208,8 +210,20 @@ int load_norm(prima_ctx* c, float** dst, float* gmax, const void* data, int64_t 
   return PRIMA_OK;
 }
 
+// Host-side fault injection (PRIMA_OPT_FAIL_AFTER_LAUNCHES): stands in for a launch that the runtime refuses.
+inline bool injected_failure(prima_ctx* c) {
+  if (c->fail_after < 0) return false;
+  if (c->fail_after == 0) {
+    c->fail_after = -1;
+    return true;
+  }
+  --c->fail_after;
+  return false;
+}
+
 #define LAUNCH(c, expr, what)                                                       \
   do {                                                                              \
+    if (injected_failure(c)) return fail((c), PRIMA_ERR_CUDA, std::string(what) + ": injected launch failure"); \
     int k_ = (expr);                                                                \
     if (k_ < 0) return cuda_fail((c), static_cast<cudaError_t>(-k_), what);         \
     (c)->launches += k_;                                                            \
@@ -219,6 +233,7 @@ int load_norm(prima_ctx* c, float** dst, float* gmax, const void* data, int64_t 
 #define LAUNCH_P(c, klass_, bytes_, expr, what)                                     \
   do {                                                                              \
     prima_ctx::Span sp_{nullptr, nullptr, (klass_), (bytes_), 0};                   \
+    if (injected_failure(c)) return fail((c), PRIMA_ERR_CUDA, std::string(what) + ": injected launch failure"); \
     if ((c)->profiling) {                                                           \
       cudaEventCreate(&sp_.a);                                                      \
       cudaEventCreate(&sp_.b);                                                      \
@@ -235,6 +250,16 @@ int load_norm(prima_ctx* c, float** dst, float* gmax, const void* data, int64_t 
   } while (0)
 
 int64_t q4k_bytes(const TiledMat& t) { return t.rows * t.n_sb * kBlockBytes; }
+
+// Queue the clearing of the four accumulator arrays and of the status word: restores the "all zero
+// between calls" state after a step that failed half-way or whose kernels reported a failed self-check.
+void queue_reset(prima_ctx* c) {
+  cudaMemsetAsync(c->acc_qkv, 0, static_cast<size_t>(c->n_acc_qkv) * sizeof(acc_t), c->stream);
+  cudaMemsetAsync(c->acc_o, 0, static_cast<size_t>(c->n_acc_o) * sizeof(acc_t), c->stream);
+  cudaMemsetAsync(c->acc_gu, 0, static_cast<size_t>(c->n_acc_gu) * sizeof(acc_t), c->stream);
+  cudaMemsetAsync(c->acc_down, 0, static_cast<size_t>(c->n_acc_down) * sizeof(acc_t), c->stream);
+  cudaMemsetAsync(c->status, 0, sizeof(int), c->stream);
+}
 
 }  // namespace
 
@@ -397,10 +422,33 @@ int prima_load_q4k_weights(prima_ctx* c, int layer, int tensor_id, const void* d
 // One step over layers [layer_begin, layer_end).  seq == nullptr: n_tok tokens of sequence 0 at positions
 // pos0 .. pos0 + n_tok - 1, causal among themselves.  Otherwise token t belongs to sequence seq[t] and sits at
 // position pos[t] of that sequence's own cache: the products run over all tokens together, attention per token.
+static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos0,
+                                 int n_tok, const int32_t* seq, const int32_t* pos);
+
 static int forward_window_impl(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos0,
                                int n_tok, const int32_t* seq, const int32_t* pos) {
+  DeviceGuard guard(c->cfg.device);
+  // Everything that can fail without a launch comes first: the caches of the window's (layer, sequence)
+  // pairs are allocated here, so that an allocation failure means that nothing was queued.
+  if (seq) {
+    for (int l = layer_begin; l < layer_end; ++l)
+      for (int t = 0; t < n_tok; ++t) {
+        __half *k = nullptr, *v = nullptr;
+        const int rc = ensure_kv_seq(c, l, seq[t], &k, &v);
+        if (rc != PRIMA_OK) return rc;
+      }
+  }
+  const int64_t before = c->launches;
+  const int rc = forward_window_launch(c, layer_begin, layer_end, hidden_in, hidden_out, pos0, n_tok, seq, pos);
+  // A launch that failed after earlier kernels of the window were queued leaves accumulators that are
+  // not zero: clear them behind the queued work, so that the next call starts from the usual state.
+  if (rc != PRIMA_OK && c->launches != before) queue_reset(c);
+  return rc;
+}
+
+static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos0,
+                                 int n_tok, const int32_t* seq, const int32_t* pos) {
   const prima_model_config& g = c->cfg;
-  DeviceGuard guard(g.device);
   cudaStream_t st = c->stream;
   const int64_t e_ = g.hidden;
   const int H = g.n_q_heads, G = g.n_kv_heads;
@@ -430,7 +478,7 @@ static int forward_window_impl(prima_ctx* c, int layer_begin, int layer_end, con
     Layer& L = c->layers[l];
     GemvIn in;                                   // QKV: residual (+ down projection of layer l-1) -> h_b
     in.kind = kResidual; in.h_in = h_in; in.h_out = c->h_b; in.acc_in = acc_prev; in.mpad_in = mpad_e;
-    in.gain = L.g_attn; in.ssq_out = c->ssq_attn; in.status = c->status;
+    in.gain = L.g_attn; in.ssq_out = c->ssq_attn; in.status = c->status; in.first_wait_polls = c->first_wait_polls;
     in.zero0 = c->acc_gu; in.zero0_n = static_cast<int64_t>(n_tok) * L.gu.mpad();
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(qkv)");
     c->ssq_attn = in.ssq_out;
@@ -454,20 +502,20 @@ static int forward_window_impl(prima_ctx* c, int layer_begin, int layer_end, con
                                      c->sm_count, st), "attention");
     }
     GemvIn in_o;                                 // O: plain attention output
-    in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status;
+    in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status; in_o.first_wait_polls = c->first_wait_polls;
     in_o.zero0 = c->acc_qkv; in_o.zero0_n = static_cast<int64_t>(n_tok) * L.qkv.mpad();
     in_o.zero1 = c->acc_down; in_o.zero1_n = static_cast<int64_t>(n_tok) * mpad_e;
     in_o.out_order = kOrderResidual;
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->acc_o, c->sm_count, st), "gemv(o)");
     GemvIn in_f;                                 // gate/up: h_b + O projection -> h_a
     in_f.kind = kResidual; in_f.h_in = c->h_b; in_f.h_out = c->h_a; in_f.acc_in = c->acc_o; in_f.mpad_in = L.o.mpad();
-    in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status; in_f.out_order = kOrderSwiglu;
+    in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status; in_f.out_order = kOrderSwiglu; in_f.first_wait_polls = c->first_wait_polls;
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->acc_gu, c->sm_count, st), "gemv(gate/up)");
     c->ssq_ffn = in_f.ssq_out;
     c->ssq_ffn.eps = g.rms_eps;
     GemvIn in_d;                                 // down: SwiGLU of the gate/up product
     in_d.kind = kSwiglu; in_d.acc_in = c->acc_gu; in_d.mpad_in = L.gu.mpad();
-    in_d.ssq_in = c->ssq_ffn; in_d.status = c->status; in_d.out_order = kOrderResidual;
+    in_d.ssq_in = c->ssq_ffn; in_d.status = c->status; in_d.out_order = kOrderResidual; in_d.first_wait_polls = c->first_wait_polls;
     in_d.zero0 = c->acc_o; in_d.zero0_n = static_cast<int64_t>(n_tok) * L.o.mpad();
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->acc_down, c->sm_count, st), "gemv(down)");
     h_in = c->h_a;
@@ -521,7 +569,7 @@ int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
   cudaStream_t st = c->stream;
   GemvIn in;        // the head stages hidden itself (no partial sums to add) and leaves its sums of squares
   in.kind = kResidual; in.h_in = hidden; in.h_out = c->h_b; in.acc_in = nullptr;
-  in.mpad_in = (c->cfg.hidden + 7) / 8 * 8; in.gain = c->g_out; in.ssq_out = c->ssq_out; in.status = c->status;
+  in.mpad_in = (c->cfg.hidden + 7) / 8 * 8; in.gain = c->g_out; in.ssq_out = c->ssq_out; in.status = c->status; in.first_wait_polls = c->first_wait_polls;
   LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(head)");
   c->ssq_out = in.ssq_out;
   c->ssq_out.eps = c->cfg.rms_eps;
@@ -631,11 +679,31 @@ int prima_sync(prima_ctx* c) {
   cudaError_t e = cudaMemcpyAsync(&status, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync");
-  if (status != 0) cudaMemsetAsync(c->status, 0, sizeof(int), c->stream);      // reported once; the context stays usable
+  if (status != 0) {      // reported once; whatever the failed step left in the accumulators is cleared, so the context stays usable
+    queue_reset(c);
+    e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync(reset)");
+  }
   if (status != 0)
-    return fail(c, PRIMA_ERR_DEVICE, status == 2 ? "a partial sum was outside the accumulator range (+-2^27); results of this step are invalid"
+    return fail(c, PRIMA_ERR_DEVICE, !(status & 1) ? "a partial sum was outside the accumulator range (+-2^27); results of this step are invalid"
                                                  : "a bounded wait inside a kernel gave up (status " + std::to_string(status) + ")");
   return PRIMA_OK;
+}
+
+int prima_ctx_set_option(prima_ctx* c, int option, int64_t value) {
+  if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_ctx_set_option: null context");
+  switch (option) {
+    case PRIMA_OPT_FIRST_WAIT_POLLS:
+      if (value < -1 || value > (int64_t(1) << 30)) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_FIRST_WAIT_POLLS: value outside -1 .. 2^30");
+      c->first_wait_polls = value < 0 ? 0u : static_cast<uint32_t>(value) + 1u;
+      return PRIMA_OK;
+    case PRIMA_OPT_FAIL_AFTER_LAUNCHES:
+      if (value < -1) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_FAIL_AFTER_LAUNCHES: value below -1");
+      c->fail_after = value;
+      return PRIMA_OK;
+    default:
+      return fail(c, PRIMA_ERR_ARG, "prima_ctx_set_option: unknown option");
+  }
 }
 
 int prima_profile_enable(prima_ctx* c, int on) {
@@ -751,7 +819,7 @@ int prima_gemv_q4k(const void* dev_w, int64_t rows, int64_t cols, const float* d
   if (rc != PRIMA_OK) return rc;
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "prima_gemv_q4k");
   if (status != 0)
-    return fail(nullptr, PRIMA_ERR_DEVICE, status == 2 ? "prima_gemv_q4k: a partial sum is outside the accumulator range (+-2^27)"
+    return fail(nullptr, PRIMA_ERR_DEVICE, !(status & 1) ? "prima_gemv_q4k: a partial sum is outside the accumulator range (+-2^27)"
                                                        : "prima_gemv_q4k: a bounded wait inside the kernel gave up");
   return PRIMA_OK;
 }

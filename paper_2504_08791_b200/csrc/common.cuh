@@ -132,7 +132,8 @@ struct GemvIn {
   int64_t zero0_n = 0;
   acc_t* zero1 = nullptr;
   int64_t zero1_n = 0;
-  int* status = nullptr;           // device word raised if a bounded wait gives up (1) or a partial sum is out of range (2)
+  int* status = nullptr;           // device word: bit 0 set if a bounded wait gave up, bit 1 if a partial sum was out of range
+  uint32_t first_wait_polls = 0;   // 0: the ordinary limit; otherwise the poll limit of every warp's first wait + 1 (test hook)
 };
 int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, int sm_count, cudaStream_t st);
 

@@ -47,12 +47,38 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i)
+// Bounded wait: false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = kWaitLimit) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+
+// Book-keeping of a warp's ring for the case that a wait gives up.  Requests and waits go round the
+// ring in step, so the copies still on their way when a wait fails are those of the failing slot and
+// of the slots requested after it.  The warp issues no further requests, goes through the rest of
+// its loop without touching the ring (it must keep taking part in the CTA's barriers), and before
+// the CTA exits -- which releases the shared memory the copies are heading for -- gives every one of
+// those slots one more bounded wait.
+struct RingDrain {
+  int slot = 0, n = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void note(int failing_slot, uint32_t failing_phase, int outstanding) {
+    slot = failing_slot;
+    phase = failing_phase;
+    n = outstanding;
+  }
+  __device__ __forceinline__ void drain(uint32_t bar0, int ring) {
+    for (int i = 0; i < n; ++i) {
+      mbar_wait(bar0 + 8 * slot, phase);
+      if (++slot == ring) {
+        slot = 0;
+        phase ^= 1u;
+      }
+    }
+    n = 0;
+  }
+};
 
 // D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col)
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -94,6 +120,7 @@ struct GemvParams {
   int64_t zero1_n;
   int out_order;
   int* status;
+  uint32_t first_wait_polls;   // poll limit of a warp's first wait (kWaitLimit in normal use; a test lowers it to exercise the give-up path)
 };
 
 // Loads of what another kernel wrote go to L2 directly.

@@ -18,6 +18,12 @@
 // written by that same call, so nothing needs clearing between calls; but two calls whose kernels
 // overlap on the GPU (different streams, no ordering between them) overwrite each other's partial
 // sums and give wrong results.  Keep calls on one device ordered.
+//
+// Contexts.  The array's device address is looked up once per device ordinal, on the first call, and
+// remembered.  That address belongs to the CUDA context that was current on the device at that
+// moment (normally the runtime's primary context).  A caller that later resets the device
+// (cudaDeviceReset) or makes a different driver-API context current on the same device must not
+// use this entry point afterwards: the remembered address would be stale.
 #include <cstdio>
 #include <mutex>
 
@@ -92,10 +98,11 @@ int prima_gemv_q4k_noalloc(const void* dev_w, int64_t rows, int64_t cols, const 
   if (rows < 1 || cols < 256 || cols % 256 != 0 || n_cols < 1 || n_cols > PRIMA_MAX_N_TOK)
     return noalloc_fail(PRIMA_ERR_ARG, "prima_gemv_q4k_noalloc: rows >= 1, cols a positive multiple of 256 and 1 <= n_cols <= 8 are required");
   const int64_t n_sb = cols / 256;
-  if (rows > kScratchFloats || rows * n_sb > kScratchFloats || rows * n_sb * n_cols > kScratchFloats) {
+  // every factor is bounded before it enters a product, so that nothing wraps around for absurd sizes
+  if (n_sb > kScratchFloats || rows > kScratchFloats / n_sb || rows * n_sb > kScratchFloats / n_cols) {
     snprintf(g_noalloc_error, sizeof(g_noalloc_error),
-             "prima_gemv_q4k_noalloc: rows * (cols/256) * n_cols = %lld exceeds the built-in scratch of %lld floats",
-             static_cast<long long>(rows) * n_sb * n_cols, static_cast<long long>(kScratchFloats));
+             "prima_gemv_q4k_noalloc: rows * (cols/256) * n_cols = %.0f exceeds the built-in scratch of %lld floats",
+             static_cast<double>(rows) * static_cast<double>(n_sb) * n_cols, static_cast<long long>(kScratchFloats));
     return PRIMA_ERR_ARG;
   }
   int dev = -1;

@@ -176,6 +176,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
   int parity = 0;
   bool alive = true;
   bool waited = false;
+  bool first_wait = true;
+  RingDrain drain;
   int slot = 0;
   uint32_t phase = 0;
   constexpr uint32_t E = 0x0f0f0f0fu;
@@ -187,7 +189,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
     pf.init(cur.pos, seg_end, n_rt);
 #pragma unroll
     for (int i = 0; i < kRingTok - 1; ++i)
-      if (!pf.done()) request();
+      if (alive && !pf.done()) request();
     if (!waited) {
       pdl_wait();
       waited = true;
@@ -245,7 +247,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
       __syncwarp();
       // the generic-proxy reads of the buffer are done; order them before the copy that overwrites it
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      if (!pf.done()) request();
+      if (alive && !pf.done()) request();
     }
     if (P.kind == kResidual) {
       __syncthreads();
@@ -258,9 +260,14 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
     }
     while (cur.pos < seg_end) {
       const int nb = cur.batch();
-      if (alive && !mbar_wait(bar_u32 + 8 * slot, phase)) {
-        alive = false;
-        if (lane == 0) atomicExch(status, 1);
+      if (alive) {
+        const bool ok = mbar_wait(bar_u32 + 8 * slot, phase, first_wait ? P.first_wait_polls : kWaitLimit);
+        first_wait = false;
+        if (!__all_sync(0xffffffffu, ok)) {
+          alive = false;
+          drain.note(slot, phase, n_in_flight);
+          if (lane == 0) atomicOr(status, 1);
+        }
       }
       --n_in_flight;
       const uint8_t* base = my_ring + slot * kBatchBytes;
@@ -321,7 +328,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
           const float* src = red + (parity * kMaxWarps * kBatch) * kRowsPerTile * kTokCols + idx;
           float sum = src[0];
           for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile * kTokCols];
-          if (!(fabsf(sum) < kAccLimit)) atomicExch(status, 2);
+          if (!(fabsf(sum) < kAccLimit)) atomicOr(status, 2);
           atomicAdd(acc_out + static_cast<int64_t>(tok) * mpad + acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row), acc_from(sum));
         }
       }
@@ -333,15 +340,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
       cur.next(nb);
     }
   }
-  if (!alive) {
-    for (int i = 0; i < n_in_flight && i < kRingTok; ++i) {
-      mbar_wait(bar_u32 + 8 * slot, phase);
-      if (++slot == kRingTok) {
-        slot = 0;
-        phase ^= 1u;
-      }
-    }
-  }
+  if (!alive) drain.drain(bar_u32, kRingTok);
 }
 
 }  // namespace

@@ -294,6 +294,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   int parity = 0;
   bool alive = true;
   bool waited = false;
+  bool first_wait = true;
+  RingDrain drain;
   int slot = 0;                  // ring slot of the next wait
   uint32_t phase = 0;
 
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     pf.init(cur.pos, seg_end, n_rt);
 #pragma unroll
     for (int i = 0; i < kRing; ++i)
-      if (!pf.done()) request();
+      if (alive && !pf.done()) request();
     if (!waited) {      // the first weight batches are on their way; everything below depends on the predecessor kernel
       pdl_wait();
       waited = true;
@@ -341,9 +343,14 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     }
     while (cur.pos < seg_end) {
     const int nb = cur.batch();
-    if (alive && !mbar_wait(bar_u32 + 8 * slot, phase)) {
-      alive = false;
-      if (lane == 0) atomicExch(status, 1);
+    if (alive) {
+      const bool ok = mbar_wait(bar_u32 + 8 * slot, phase, first_wait ? P.first_wait_polls : kWaitLimit);
+      first_wait = false;
+      if (!__all_sync(0xffffffffu, ok)) {      // the same verdict in every lane
+        alive = false;
+        drain.note(slot, phase, n_in_flight);
+        if (lane == 0) atomicOr(status, 1);
+      }
     }
     --n_in_flight;
     const uint8_t* base = my_ring + slot * kBatchBytes;
@@ -396,7 +403,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
         const float* src = red + ((parity * NTOK + k) * kMaxWarps * kBatch + i) * kRowsPerTile + row;
         float sum = src[0];
         for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile];
-        if (!(fabsf(sum) < kAccLimit)) atomicExch(status, 2);
+        if (!(fabsf(sum) < kAccLimit)) atomicOr(status, 2);
         atomicAdd(acc_out + static_cast<int64_t>(tok0 + k) * mpad + acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row), acc_from(sum));
       }
     }
@@ -408,17 +415,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     cur.next(nb);
     }
   }
-  // A wait gave up: copies may still be in flight towards this CTA's shared memory.  Give each
-  // outstanding slot one more bounded wait before the memory is released.
-  if (!alive) {
-    for (int i = 0; i < n_in_flight && i < kRing; ++i) {
-      mbar_wait(bar_u32 + 8 * slot, phase);
-      if (++slot == kRing) {
-        slot = 0;
-        phase ^= 1u;
-      }
-    }
-  }
+  // A wait gave up: copies may still be on their way to this CTA's shared memory.
+  if (!alive) drain.drain(bar_u32, kRing);
 }
 
 size_t gemv_smem_bytes(int sg, int n_tok) {
@@ -478,6 +476,7 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
   P.n_tok_total = n_tok; P.acc = acc; P.mpad = w.mpad(); P.status = in.status;
   P.zero0 = in.zero0; P.zero0_n = in.zero0_n; P.zero1 = in.zero1; P.zero1_n = in.zero1_n;
   P.out_order = in.out_order;
+  P.first_wait_polls = in.first_wait_polls ? in.first_wait_polls - 1 : kWaitLimit;
   if ((in.out_order == kOrderResidual && w.mpad() % 256 != 0) || (in.out_order == kOrderSwiglu && w.mpad() % 512 != 0)) return cuda_rc(cudaErrorInvalidValue);
   int launches = 0;
   if (n_tok > 4 && gemv_uses_tensor_cores()) {

@@ -5,6 +5,14 @@
 * 70B shape, 5-token verification step at 8192 cached positions (first 3 layers; the checker's cost
   is 5x per layer), causal inside the step.
 * 32B shape (hidden 5120: column groups of 4, 27 groups in the down projection), first 3 layers + head.
+* 32B shape at full depth (64 layers, 4096 cached positions): four greedy tokens, logits and token of every step.
+* 32B widths, 2 layers + the full-vocabulary head: the 64-step greedy loop.
+
+Hidden-state tolerance after L layers: the per-layer errors (fp16 rounding of Q and P in attention,
+16-bit activation steps in the four products) are independent and zero-mean, so they add like a
+random walk while the residual stream's RMS also grows; 2e-3 of the RMS covers a window of 20
+layers with a margin of about 4, and the allowance grows with the square root of the depth:
+tol(L) = 2e-3 * sqrt(max(L, 20) / 20), i.e. 4e-3 after 80 layers.
 """
 import numpy as np
 import pytest
@@ -14,6 +22,10 @@ from paper_2504_08791_b200 import synth
 from tests.test_gpu_model import HIDDEN_TOL, LOGIT_TOL, MARGIN, Pair, _hidden_close, gpu  # noqa: F401
 
 pytestmark = pytest.mark.gpu
+
+
+def hidden_tol(n_layers_so_far: int) -> float:
+    return HIDDEN_TOL * float(np.sqrt(max(n_layers_so_far, 20) / 20.0))
 
 
 def test_70b_shape_80_layers_as_4_windows(gpu):
@@ -26,11 +38,11 @@ def test_70b_shape_80_layers_as_4_windows(gpu):
     for w in range(4):
         h_ref = p.ref.forward_window(20 * w, 20 * w + 20, h_ref, n_ctx)
         h_gpu = p.gpu_window(20 * w, 20 * w + 20, h_gpu, n_ctx)
-        worst = max(worst, _hidden_close(h_gpu, h_ref, tol=2 * HIDDEN_TOL))
+        worst = max(worst, _hidden_close(h_gpu, h_ref, tol=hidden_tol(20 * w + 20)) / hidden_tol(20 * w + 20))
     l_ref = p.ref.logits(h_ref)[0]
     l_gpu = p.gpu_logits(h_gpu)[0]
     err = float(np.abs(l_gpu.astype(np.float64) - l_ref).max())
-    print(f"70B shape: worst hidden error {worst:.2e} of RMS, logits max abs error {err:.2e}")
+    print(f"70B shape: worst hidden error {worst:.2f} of its allowance, logits max abs error {err:.2e}")
     assert err <= LOGIT_TOL
     tok, margin = oracle.argmax(l_ref)
     if margin > MARGIN:
@@ -59,4 +71,52 @@ def test_32b_shape_three_layers_and_head(gpu):
     got = p.gpu_window(0, 3, h0, n_ctx)
     _hidden_close(got, want)
     assert np.abs(p.gpu_logits(got).astype(np.float64) - p.ref.logits(want)).max() <= LOGIT_TOL
+    p.close()
+
+
+def _greedy(p, cfg, n_ctx, steps, torch):
+    """Greedy decoding through the ABI against the checker; both continue from the checker's token."""
+    hid = torch.empty((1, cfg["hidden"]), dtype=torch.float32, device="cuda")
+    logits = torch.empty((1, cfg["vocab"]), dtype=torch.float32, device="cuda")
+    tok, low_margin, worst = 0, 0, 0.0
+    for step in range(steps):
+        pos = n_ctx + step
+        l_ref = p.ref.logits(p.ref.forward_window(0, cfg["n_layers"], p.ref.embed([tok]), pos))[0]
+        want_tok, margin = oracle.argmax(l_ref)
+        p.ctx.embed([tok], hid)
+        p.ctx.forward_window(0, cfg["n_layers"], hid, hid, pos, 1)
+        p.ctx.logits(hid, 1, logits)
+        got_tok = int(p.ctx.argmax(logits, 1)[0])
+        l_gpu = logits.cpu().numpy()[0]
+        err = float(np.abs(l_gpu.astype(np.float64) - l_ref).max())
+        worst = max(worst, err)
+        assert err <= LOGIT_TOL, f"step {step}: logits differ by {err:.2e}"
+        assert got_tok == int(np.argmax(l_gpu))
+        if margin > MARGIN:
+            assert got_tok == want_tok, f"step {step}: margin {margin}"
+        else:
+            low_margin += 1
+        tok = want_tok
+    return low_margin, worst
+
+
+def test_32b_shape_full_depth_four_greedy_tokens(gpu):
+    torch, _ = gpu
+    cfg = synth.model_config("32b")
+    n_ctx, seed, steps = 4096, 2, 4
+    p = Pair(gpu, cfg, seed=seed, n_prefill=n_ctx)
+    low, worst = _greedy(p, cfg, n_ctx, steps, torch)
+    print(f"32B shape, 64 layers: {steps} greedy tokens, worst logit error {worst:.2e}, {low} step(s) with a top-2 gap below {MARGIN}")
+    assert low <= 1
+    p.close()
+
+
+def test_32b_widths_two_layers_64_greedy_tokens(gpu):
+    torch, _ = gpu
+    cfg = synth.model_config("32b", n_layers=2)
+    n_ctx, seed, steps = 4096 - 64, 2, 64
+    p = Pair(gpu, cfg, seed=seed, n_prefill=n_ctx)
+    low, worst = _greedy(p, cfg, n_ctx, steps, torch)
+    print(f"32B widths, 2 layers + head: {steps} greedy tokens, worst logit error {worst:.2e}, {low} step(s) with a top-2 gap below {MARGIN}")
+    assert low <= 8
     p.close()

@@ -267,3 +267,55 @@ def test_long_context_with_more_chunks_than_resident_ctas(gpu, n_tok):
     got = p.gpu_window(0, cfg["n_layers"], h0, pos)
     _hidden_close(got, want)
     p.close()
+
+
+@pytest.mark.parametrize("n_tok", [1, 6])
+def test_a_wait_that_gives_up_is_reported_once_and_the_next_step_is_clean(gpu, n_tok):
+    """The bounded waits of the streaming kernels: with the poll limit of every warp's first wait set to 0 the wait
+    runs out at once; the kernels must still wait (with the ordinary limit) for every copy they requested, return
+    normally and raise the status word.  prima_sync reports it once and clears the accumulators, after which the
+    context gives exactly the bits of a context that never failed."""
+    torch, binding = gpu
+    cfg = synth.model_config("small")
+    pos = 90
+    h0 = synth.activations(47, n_tok, cfg["hidden"])
+    p = Pair(gpu, cfg, seed=47, n_prefill=pos)
+    good = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    good_logits = p.gpu_logits(good)
+    p.ctx.set_option(binding.OPT_FIRST_WAIT_POLLS, 0)
+    hin = torch.from_numpy(h0).cuda()
+    hout = torch.empty_like(hin)
+    p.ctx.forward_window(0, cfg["n_layers"], hin, hout, pos, n_tok)
+    with pytest.raises(binding.PrimaError) as err:
+        p.ctx.sync()
+    assert err.value.code == binding.ERR_DEVICE and "wait" in str(err.value)
+    p.ctx.sync()                                         # reported once
+    p.ctx.set_option(binding.OPT_FIRST_WAIT_POLLS, -1)   # the ordinary limit again
+    again = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    assert np.array_equal(again.view(np.uint32), good.view(np.uint32))
+    assert np.array_equal(p.gpu_logits(again).view(np.uint32), good_logits.view(np.uint32))
+    with pytest.raises(binding.PrimaError):
+        p.ctx.set_option(99, 0)
+    p.close()
+
+
+@pytest.mark.parametrize("after", [2, 5, 9])
+def test_a_launch_refused_in_mid_window_leaves_the_next_call_clean(gpu, after):
+    """A launch in the middle of a window fails (injected on the host: the library is told to refuse it, nothing
+    faulty reaches the GPU).  The call returns an error; the call after it gives the bits of an undisturbed context."""
+    torch, binding = gpu
+    cfg = synth.model_config("small")
+    pos, n_tok = 60, 2
+    h0 = synth.activations(53, n_tok, cfg["hidden"])
+    p = Pair(gpu, cfg, seed=53, n_prefill=pos, with_globals=False)
+    good = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    hin = torch.from_numpy(h0).cuda()
+    hout = torch.empty_like(hin)
+    p.ctx.set_option(binding.OPT_FAIL_AFTER_LAUNCHES, after)
+    with pytest.raises(binding.PrimaError) as err:
+        p.ctx.forward_window(0, cfg["n_layers"], hin, hout, pos, n_tok)
+    assert err.value.code == binding.ERR_CUDA and "injected" in str(err.value)
+    p.ctx.sync()
+    again = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    assert np.array_equal(again.view(np.uint32), good.view(np.uint32))
+    p.close()

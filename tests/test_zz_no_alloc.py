@@ -46,5 +46,8 @@ def test_sizes_beyond_the_built_in_scratch_are_refused_with_a_clear_message():
     with pytest.raises(binding.PrimaError) as e:
         binding.prima_gemv_q4k_noalloc(d, 1 << 20, 2048, f, 1, f)      # 2^20 * 8 partials > 4 Mi: refused before any launch
     assert "exceeds the built-in scratch" in str(e.value)
+    with pytest.raises(binding.PrimaError) as e:
+        binding.prima_gemv_q4k_noalloc(d, 1 << 22, 256 << 42, f, 1, f)   # rows * (cols/256) wraps to 0 in 64 bits: still refused by size
+    assert e.value.code == binding.ERR_ARG and "exceeds the built-in scratch" in str(e.value)
     with pytest.raises(binding.PrimaError):
         binding.prima_gemv_q4k_noalloc(d, 8, 200, f, 1, f)             # cols not a multiple of 256
