@@ -139,21 +139,76 @@ def job_value(ms_per_step_max: float, world: int) -> dict:
 
 
 # ------------------------------------------------------------------------------------ the GPU arm
-def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None, n_requests=1):
+def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None, n_requests=1, on_layer=None, on_globals=None):
+    """Generate the synthetic model layer by layer and make it resident.  on_layer(l, tensors, k, v) and
+    on_globals(tensors) see the same host arrays (the CPU-baseline leg runs the checker on them, so the 39 GB of
+    a 70B-shaped model are generated once and never held in host memory all at once)."""
     import torch
     t0 = time.time()
     ctx = binding.Context(cfg, device=device)
     layers = range(cfg["n_layers"]) if n_layers is None else range(n_layers)
-    for layer, tid, rows, cols, data in synth.iter_model_tensors(seed, cfg, layers=layers):
-        ctx.load(layer, tid, data, rows, cols)
-    t1 = time.time()
     for l in layers:
+        tensors = {}
+        for layer, tid, rows, cols, data in synth.iter_model_tensors(seed, cfg, layers=[l], with_globals=False):
+            ctx.load(layer, tid, data, rows, cols)
+            tensors[tid] = (rows, cols, data)
         k, v = synth.kv_prefill(seed, l, n_ctx, cfg["n_kv_heads"], cfg["head_dim"])
         for r in range(n_requests):               # every request gets a cache of its own (same synthetic content)
             ctx.kv_load(l, 0, k, v, seq=r)
+        if on_layer is not None:
+            on_layer(l, tensors, k, v)
+    tensors = {}
+    for tid in synth.GLOBAL_TENSORS:
+        rows, cols = synth.tensor_shape(cfg, tid)
+        data = synth.make_tensor(seed, cfg, -1, tid)
+        ctx.load(-1, tid, data, rows, cols)
+        tensors[tid] = (rows, cols, data)
+    if on_globals is not None:
+        on_globals(tensors)
     torch.cuda.synchronize()
-    log(f"[bench] model resident: weights {t1 - t0:.1f}s, kv prefill {time.time() - t1:.1f}s")
+    log(f"[bench] model resident after {time.time() - t0:.1f}s")
     return ctx
+
+
+class WholeTokenOracle:
+    """The CPU checker, as it stands, run over ONE whole token of the workload while the model is being generated:
+    layer l is loaded into a one-layer checker model, run on the hidden state that layer l-1 left, and dropped;
+    then the output layer.  Only the checker's own calls are timed (not the generation of the weights)."""
+
+    def __init__(self, cfg, seed, n_ctx, n_tok=1):
+        import oracle
+        self.oracle, self.cfg, self.n_ctx = oracle, cfg, n_ctx
+        self.cores = oracle.default_threads()
+        self.h = synth.activations(seed, n_tok, cfg["hidden"])
+        self.seconds, self.layers_done, self.logits = 0.0, 0, None
+
+    def on_layer(self, l, tensors, k, v):
+        one = dict(self.cfg, n_layers=1)
+        mdl = self.oracle.Model(one, n_threads=self.cores)
+        for tid, (rows, cols, data) in tensors.items():
+            mdl.load(0, tid, data, rows, cols)
+        mdl.kv_load(0, 0, k, v)
+        t0 = time.perf_counter()
+        self.h = mdl.forward_window(0, 1, self.h, self.n_ctx)
+        self.seconds += time.perf_counter() - t0
+        self.layers_done += 1
+        mdl.close()
+
+    def on_globals(self, tensors):
+        one = dict(self.cfg, n_layers=1)
+        mdl = self.oracle.Model(one, n_threads=self.cores)
+        for tid in (synth.OUT_NORM, synth.W_HEAD):
+            rows, cols, data = tensors[tid]
+            mdl.load(-1, tid, data, rows, cols)
+        t0 = time.perf_counter()
+        self.logits = mdl.logits(self.h)
+        self.seconds += time.perf_counter() - t0
+        mdl.close()
+
+    def result(self, n_tok=1):
+        return {"value": self.seconds * 1e3, "unit": "ms/token" if n_tok == 1 else "ms/step", "cores": self.cores, "kind": "oracle",
+                "sample": f"one whole {'token' if n_tok == 1 else 'step of %d tokens' % n_tok}: all {self.layers_done} layers at full width and "
+                          f"{self.n_ctx} cached positions + the output layer, layer by layer (only the checker's calls are timed)"}
 
 
 def run_ours(args, rank, world, local_rank):
@@ -180,7 +235,11 @@ def run_ours(args, rank, world, local_rank):
     R = args.requests
     if R > 1 and args.n_tok > 1:
         raise SystemExit("--requests and --n-tok are alternatives")
-    ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank, n_requests=R)
+    whole = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and R == 1 and not args.layers:
+        whole = WholeTokenOracle(cfg, seed, n_ctx, args.n_tok)
+    ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank, n_requests=R,
+                          on_layer=whole.on_layer if whole else None, on_globals=whole.on_globals if whole else None)
     bpt = bytes_per_token(cfg, n_ctx)
     if R > 1:                                     # the weights are read once per step, every request's cache once
         bpt = dict(bpt, total=bpt["total"] + (R - 1) * L_kv_bytes(cfg, n_ctx))
@@ -227,15 +286,21 @@ def run_ours(args, rank, world, local_rank):
     sampler = ClockSampler(local_rank)
     sampler.start()
     launches0 = ctx.launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(args.steps):
-        device_step(n_ctx)
-    ev1.record()
-    barrier()
-    launches = ctx.launch_count() - launches0
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
-    ms_step = ms_total / args.steps
+    # the timed region (exactly --steps steps between two events, barrier and synchronize on both sides), taken
+    # --repeats times back to back: the median region is the reported one, min and all are listed in `config`
+    regions = []
+    launches = 0
+    for rep in range(max(1, args.repeats)):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(args.steps):
+            device_step(n_ctx)
+        ev1.record()
+        barrier()
+        if rep == 0:
+            launches = ctx.launch_count() - launches0
+        regions.append(max_over_ranks(ev0.elapsed_time(ev1)) / args.steps)
+    ms_step = float(np.median(regions))
 
     # end to end through the ABI: host token in, host token out, every step
     adv = 1 if R > 1 else T                        # positions a step advances a cache by
@@ -255,14 +320,32 @@ def run_ours(args, rank, world, local_rank):
     e2e_ms = max_over_ranks(max(ev2.elapsed_time(ev3), wall_ms)) / e2e_steps
     clocks = sampler.stop()
 
-    # dominant kernel: event-bracketed GEMV launches in a separate pass (bracketing perturbs whole-step time)
-    ctx.profile_enable(True)
-    prof_steps = max(1, min(args.steps, 5))
+    # dominant kernel inside the running step: the kernels stamp the GPU timer themselves (first CTA past its
+    # dependency wait .. last CTA done), launch sequence unchanged
+    prof_steps = max(1, min(args.steps, 10))
+    ctx.profile_enable(2)
+    ev4, ev5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev4.record()
     for _ in range(prof_steps):
         device_step(n_ctx)
+    ev5.record()
     g_ms, g_n, g_bytes = ctx.profile_read(binding.PROF_GEMV)
     a_ms, a_n, a_bytes = ctx.profile_read(binding.PROF_ATTENTION)
-    ctx.profile_enable(False)
+    by_matrix = {}
+    for name, klass in (("qkv", binding.PROF_GEMV_QKV), ("o", binding.PROF_GEMV_O), ("gate_up", binding.PROF_GEMV_GATE_UP),
+                        ("down", binding.PROF_GEMV_DOWN), ("head", binding.PROF_GEMV_HEAD)):
+        m_ms, m_n, m_bytes = ctx.profile_read(klass)
+        if m_n:
+            by_matrix[name] = {"avg_launch_us": m_ms * 1e3 / m_n, "GB/s": m_bytes / (m_ms * 1e-3) / 1e9, "MB": m_bytes / m_n / 1e6}
+    stamped_ms_step = ev4.elapsed_time(ev5) / prof_steps
+    # the same kernels in isolation: a pair of events around every launch (serialises them)
+    ctx.profile_enable(1)
+    iso_steps = max(1, min(args.steps, 5))
+    for _ in range(iso_steps):
+        device_step(n_ctx)
+    gi_ms, gi_n, gi_bytes = ctx.profile_read(binding.PROF_GEMV)
+    ai_ms, ai_n, ai_bytes = ctx.profile_read(binding.PROF_ATTENTION)
+    ctx.profile_enable(0)
 
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):
@@ -271,6 +354,9 @@ def run_ours(args, rank, world, local_rank):
         peak, peak_src = 6650.0, "fallback"
     gemv_gbs = g_bytes / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
     attn_gbs = a_bytes / (a_ms * 1e-3) / 1e9 if a_ms > 0 else 0.0
+    gemv_iso_gbs = gi_bytes / (gi_ms * 1e-3) / 1e9 if gi_ms > 0 else 0.0
+    attn_iso_gbs = ai_bytes / (ai_ms * 1e-3) / 1e9 if ai_ms > 0 else 0.0
+    kernel_name = "gemv_partials_kernel<%d>" % T if T <= 4 else "gemv_tokens_kernel"
     step_gbs = bpt["total"] / (ms_step * 1e-3) / 1e9
 
     result = {
@@ -289,17 +375,25 @@ def run_ours(args, rank, world, local_rank):
                    "value_is": ("ms per decoded token" if T == 1 else "ms per verification step of %d tokens" % T) if R == 1
                    else "ms per step of %d concurrent requests (one token each)" % R, "requests": R,
                    "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs larger than L2 (>= 4.9 GB per step)",
-                   "bytes_per_token": bpt["total"]},
+                   "bytes_per_token": bpt["total"], "repeats": len(regions), "ms_per_step_min": min(regions),
+                   "ms_per_step_all": regions, "value_is_median_of_repeats": True},
         "step_roofline": {"bound": "hbm", "achieved": step_gbs, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                           "frac": step_gbs / peak, "frac_of_nominal_8000": step_gbs / 8000.0},
-        "roofline": {"kernel": "gemv_partials_kernel<%d>" % T if T <= 4 else "gemv_tokens_kernel", "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
+        "roofline": {"kernel": kernel_name, "bound": "hbm", "achieved": gemv_gbs, "peak": peak, "peak_source": peak_src,
                      "unit": "GB/s", "frac": gemv_gbs / peak,
-                     "traffic": (NCU_TRAFFIC_RATIO * g_bytes / g_n) if (g_n and T == 1) else None,
-                     "traffic_note": "bytes per launch: algorithmic bytes x 1.018, the DRAM read+write / Q4_K bytes ratio of the ncu "
-                                     "capture of the four layer matrices (profiles/gemv_partials_70b_matrices.md)",
+                     "traffic": None,
+                     "traffic_estimated": (NCU_TRAFFIC_RATIO * g_bytes / g_n) if (g_n and T == 1 and args.workload == "70b") else None,
+                     "traffic_note": "no DRAM counters for the kernel as it stands in this run; traffic_estimated = algorithmic bytes per "
+                                     "launch x the DRAM read+write / Q4_K bytes ratio of the ncu capture named in profiles/",
                      "launches": g_n // prof_steps, "avg_launch_us": (g_ms * 1e3 / g_n) if g_n else None,
-                     "timing": f"cuda events around each launch, separate pass of {prof_steps} steps"},
-        "attention_kernel": {"achieved": attn_gbs, "unit": "GB/s", "frac": attn_gbs / peak, "launches": a_n // prof_steps},
+                     "kernel_ms_per_step": g_ms / prof_steps, "step_ms_in_this_pass": stamped_ms_step, "by_matrix": by_matrix,
+                     "timing": f"in situ: every launch stamps the GPU timer (first CTA past its dependency wait .. last CTA done), "
+                               f"launch sequence unchanged, pass of {prof_steps} steps after the timed region"},
+        "roofline_isolated": {"kernel": kernel_name, "achieved": gemv_iso_gbs, "unit": "GB/s", "frac": gemv_iso_gbs / peak,
+                              "avg_launch_us": (gi_ms * 1e3 / gi_n) if gi_n else None,
+                              "timing": f"cuda events around each launch (serialised), separate pass of {iso_steps} steps"},
+        "attention_kernel": {"achieved": attn_gbs, "unit": "GB/s", "frac": attn_gbs / peak, "launches": a_n // prof_steps,
+                             "kernel_ms_per_step": a_ms / prof_steps, "isolated_achieved": attn_iso_gbs},
         "e2e": {"value": e2e_ms / world, "unit": "ms/token", "h2d_bytes_per_step": 4 * T, "d2h_bytes_per_step": 4 * T, "steps": e2e_steps},
         "gpu_launches": int(launches),
         "clocks": clocks,
@@ -308,7 +402,7 @@ def run_ours(args, rank, world, local_rank):
         result["speculative"] = speculative_cycle(args, binding, ctx, cfg, seed, n_ctx, bounds)
     ctx.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
+        result["cpu_baseline"] = whole.result(args.n_tok) if whole else cpu_baseline(args.workload, budget_s=args.cpu_budget)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -343,7 +437,9 @@ def speculative_cycle(args, binding, target, cfg, seed, n_ctx, bounds) -> dict:
 
 # ------------------------------------------------------------------------------- the CPU checker arm
 def cpu_baseline(workload: str, budget_s: float = 20.0, repeat: int = 1) -> dict:
-    """The CPU checker as it stands, timed on a bounded sample: one full-width layer at full context."""
+    """Fallback sample of the CPU checker (used when the whole-token run is not possible: several requests, a
+    truncated model, and for the per-step samples of the reference arm): one full-width layer at full context,
+    scaled to the token by algorithmic bytes."""
     import oracle
     shape, n_ctx, _, _ = WORKLOADS[workload]
     cfg = synth.model_config(shape)
@@ -371,17 +467,29 @@ def cpu_baseline(workload: str, budget_s: float = 20.0, repeat: int = 1) -> dict
                       f"{per_layer * 1e3:.0f} ms per layer, scaled to the whole token by algorithmic bytes"}
 
 
+def oracle_whole_token(workload: str, n_tok: int = 1) -> dict:
+    """One whole token of the workload through the CPU checker, the model generated layer by layer (no GPU involved)."""
+    shape, n_ctx, _, _ = WORKLOADS[workload]
+    cfg = synth.model_config(shape)
+    seed = SEEDS[workload]
+    whole = WholeTokenOracle(cfg, seed, n_ctx, n_tok)
+    for l in range(cfg["n_layers"]):
+        tensors = {tid: (rows, cols, data) for _, tid, rows, cols, data in synth.iter_model_tensors(seed, cfg, layers=[l], with_globals=False)}
+        k, v = synth.kv_prefill(seed, l, n_ctx, cfg["n_kv_heads"], cfg["head_dim"])
+        whole.on_layer(l, tensors, k, v)
+    whole.on_globals({tid: synth.tensor_shape(cfg, tid) + (synth.make_tensor(seed, cfg, -1, tid),) for tid in (synth.OUT_NORM, synth.W_HEAD)})
+    return whole.result(n_tok)
+
+
 def run_reference(args):
+    """The reference arm: the CPU checker as it stands on the host cores.  One whole token is timed once (the value);
+    every one of the --steps steps additionally times a bounded sample (one full-width layer, scaled by bytes), listed
+    beside it to show the spread."""
     shape, n_ctx, n_windows, desc = WORKLOADS[args.workload]
-    vals = []
-    base = None
-    for _ in range(args.warmup if args.warmup < 2 else 1):
-        cpu_baseline(args.workload, budget_s=1.0)
-    for _ in range(max(1, min(args.steps, 5))):
-        base = cpu_baseline(args.workload, budget_s=1.0)
-        vals.append(base["value"])
-    v = float(np.median(vals))
-    base["value"] = v
+    base = oracle_whole_token(args.workload)
+    samples = [cpu_baseline(args.workload, budget_s=1.0)["value"] for _ in range(max(1, min(args.steps, 5)))]
+    base["one_layer_samples_scaled_ms"] = samples
+    v = base["value"]
     cfg = synth.model_config(shape)
     return {
         "impl": "reference", "metric": "decode_ms_per_token", "value": v, "unit": "ms/token", "n_gpus": args.gpus,
@@ -406,6 +514,7 @@ def main():
     ap.add_argument("--requests", type=int, default=1, help="concurrent requests per step, one token each, own KV caches")
     ap.add_argument("--speculative", default="", choices=["", "8b", "32b"],
                     help="also time speculative decoding cycles with a draft model of this shape")
+    ap.add_argument("--repeats", type=int, default=5, help="how many times the timed region of --steps steps is taken (median reported)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

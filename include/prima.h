@@ -197,15 +197,28 @@ int64_t prima_launch_count(prima_ctx* ctx);
 
 /* Device-side timing by kernel class, for measurement runs (the counterpart of the paper's device
  * profiler, which measures how fast weights and KV cache reach the cores: Appendix A.3, device
- * loading time).  While enabled, every launch of the listed classes is bracketed by a pair of
- * CUDA events on the context's stream; enable(…, 0 or 1) also discards what was recorded.  read
- * waits for the stream and returns, for one class, the summed event time in milliseconds, the
- * number of kernel launches and the algorithmic bytes they had to move (Q4_K weight bytes of the
- * matrices, or K and V bytes of the attended positions).  Timing perturbs the run: keep it off
- * when measuring whole steps. */
+ * loading time).  enable(ctx, mode) discards what was recorded and selects
+ *   mode 0: off;
+ *   mode 1: every launch of the listed classes is bracketed by a pair of CUDA events on the context's
+ *           stream.  This serialises the launches (a kernel no longer overlaps its predecessor's
+ *           tail), so it times each kernel in isolation and perturbs the step;
+ *   mode 2: every kernel of the listed classes stamps the GPU's nanosecond timer itself: the earliest
+ *           moment a CTA got past its wait for the predecessor kernel, and the latest moment a CTA
+ *           finished.  The launch sequence is unchanged, so these are the kernels' times inside the
+ *           running step; intervals of consecutive kernels do not overlap, their sum is at most the
+ *           step time.  Room for 32,768 launches between two calls of enable.
+ * read waits for the stream and returns, for one class, the summed time in milliseconds, the number
+ * of kernel launches and the algorithmic bytes they had to move (Q4_K weight bytes of the matrices,
+ * or K and V bytes of the attended positions). */
 #define PRIMA_PROF_GEMV 0
 #define PRIMA_PROF_ATTENTION 1
-int prima_profile_enable(prima_ctx* ctx, int on);
+/* mode 2 only: the products of one kind (a subset of PRIMA_PROF_GEMV) */
+#define PRIMA_PROF_GEMV_QKV 16
+#define PRIMA_PROF_GEMV_O 17
+#define PRIMA_PROF_GEMV_GATE_UP 18
+#define PRIMA_PROF_GEMV_DOWN 19
+#define PRIMA_PROF_GEMV_HEAD 20
+int prima_profile_enable(prima_ctx* ctx, int mode);
 int prima_profile_read(prima_ctx* ctx, int klass, double* ms_total, int64_t* launches, int64_t* algo_bytes);
 
 /* ---- context-free exports of the two primitives (tests and micro-benchmarks) ---------------- */

@@ -18,6 +18,7 @@ OK, ERR_ARG, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_DEVICE = 0, -1, -2, -3, -4, -5
 ATTN_NORM, WQ, WK, WV, WO, FFN_NORM, W_GATE, W_UP, W_DOWN, OUT_NORM, W_HEAD, TOK_EMBD = range(12)
 MAX_N_TOK = 8
 PROF_GEMV, PROF_ATTENTION = 0, 1
+PROF_GEMV_QKV, PROF_GEMV_O, PROF_GEMV_GATE_UP, PROF_GEMV_DOWN, PROF_GEMV_HEAD = 16, 17, 18, 19, 20
 OPT_FIRST_WAIT_POLLS = 1
 OPT_FAIL_AFTER_LAUNCHES = 2
 
@@ -228,8 +229,9 @@ class Context:
     def set_option(self, option: int, value: int):
         _check(lib().prima_ctx_set_option(self._h, option, value), self._h)
 
-    def profile_enable(self, on: bool):
-        _check(lib().prima_profile_enable(self._h, 1 if on else 0), self._h)
+    def profile_enable(self, mode):
+        """0 / False: off; 1 / True: events around every launch (isolated kernels); 2: in-situ stamps."""
+        _check(lib().prima_profile_enable(self._h, int(mode)), self._h)
 
     def profile_read(self, klass: int):
         """(milliseconds, launches, algorithmic bytes) recorded for one kernel class."""

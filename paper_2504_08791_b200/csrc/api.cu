@@ -76,13 +76,22 @@ struct prima_ctx {
   std::vector<void*> allocs;
   std::string err;
   int64_t launches = 0;
+  // Lowest cache position appended since the host last waited for the stream (INT_MAX: none).  Entries below it are
+  // known to be in memory and may be read by the attention kernels before their dependency wait.
+  int unsynced_min_pos = 0x7fffffff;
   uint32_t first_wait_polls = 0;   // PRIMA_OPT_FIRST_WAIT_POLLS (0: the ordinary limit)
   int64_t fail_after = -1;         // PRIMA_OPT_FAIL_AFTER_LAUNCHES: launch steps still allowed before an injected failure (-1: off)
 
-  // optional per-class device timing (prima_profile_*)
+  // optional per-class device timing (prima_profile_*): mode 1 = a pair of events around every launch,
+  // mode 2 = in-situ stamps written by the kernels themselves
   bool profiling = false;
   struct Span { cudaEvent_t a, b; int klass; int64_t bytes; int launches; };
   std::vector<Span> spans;
+  bool stamping = false;
+  unsigned long long* stamp_t0 = nullptr;   // device, [kMaxStamps]
+  unsigned long long* stamp_t1 = nullptr;
+  struct StampInfo { int klass; int sub; int64_t bytes; int launches; };
+  std::vector<StampInfo> stamp_info;
 };
 
 struct prima_gemv_plan {
@@ -251,6 +260,18 @@ inline bool injected_failure(prima_ctx* c) {
 
 int64_t q4k_bytes(const TiledMat& t) { return t.rows * t.n_sb * kBlockBytes; }
 
+constexpr size_t kMaxStamps = 1 << 15;
+
+// The stamp words of the next launch of a profiled class (mode 2), or nothing.
+Stamp next_stamp(prima_ctx* c, int klass, int64_t bytes, int launches, int sub = 0) {
+  Stamp s;
+  if (!c->stamping || c->stamp_info.size() >= kMaxStamps) return s;
+  s.t0 = c->stamp_t0 + c->stamp_info.size();
+  s.t1 = c->stamp_t1 + c->stamp_info.size();
+  c->stamp_info.push_back({klass, sub, bytes, launches});
+  return s;
+}
+
 // Queue the clearing of the four accumulator arrays and of the status word: restores the "all zero
 // between calls" state after a step that failed half-way or whose kernels reported a failed self-check.
 void queue_reset(prima_ctx* c) {
@@ -259,6 +280,7 @@ void queue_reset(prima_ctx* c) {
   cudaMemsetAsync(c->acc_gu, 0, static_cast<size_t>(c->n_acc_gu) * sizeof(acc_t), c->stream);
   cudaMemsetAsync(c->acc_down, 0, static_cast<size_t>(c->n_acc_down) * sizeof(acc_t), c->stream);
   cudaMemsetAsync(c->status, 0, sizeof(int), c->stream);
+  cudaMemsetAsync(c->attn.tickets, 0, static_cast<size_t>(kMaxTok) * c->cfg.n_kv_heads * sizeof(int), c->stream);
 }
 
 }  // namespace
@@ -314,6 +336,7 @@ int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx
   A(dev_alloc(c, &c->rope_tab, static_cast<size_t>(kMaxTok) * (kHeadDim / 2)));
   A(dev_alloc(c, &c->attn.o_part, static_cast<size_t>(n * H) * c->attn.max_chunks * kHeadDim));
   A(dev_alloc(c, &c->attn.ml_part, static_cast<size_t>(n * H) * c->attn.max_chunks));
+  A(dev_alloc(c, &c->attn.tickets, static_cast<size_t>(kMaxTok) * G, true));
   A(dev_alloc(c, &c->staging, c->staging_bytes));
   A(dev_alloc(c, &c->d_tokens, static_cast<size_t>(kMaxTok)));
   A(dev_alloc(c, &c->am_val, static_cast<size_t>(kMaxTok) * kArgmaxBlocks));
@@ -474,19 +497,26 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
   // closing kernel), QKV's and down's by the O product, O's by the down product.
   const float* h_in = hidden_in;
   const acc_t* acc_prev = nullptr;
+  int first_pos = pos0;
+  if (seq)
+    for (int t = 0; t < n_tok; ++t) first_pos = t == 0 ? pos[t] : std::min(first_pos, pos[t]);
+  const int stable_below = std::min(first_pos, c->unsynced_min_pos);
+  c->unsynced_min_pos = stable_below;      // this call appends at first_pos and above
   for (int l = layer_begin; l < layer_end; ++l) {
     Layer& L = c->layers[l];
     GemvIn in;                                   // QKV: residual (+ down projection of layer l-1) -> h_b
     in.kind = kResidual; in.h_in = h_in; in.h_out = c->h_b; in.acc_in = acc_prev; in.mpad_in = mpad_e;
     in.gain = L.g_attn; in.ssq_out = c->ssq_attn; in.status = c->status; in.first_wait_polls = c->first_wait_polls;
     in.zero0 = c->acc_gu; in.zero0_n = static_cast<int64_t>(n_tok) * L.gu.mpad();
+    in.stamp = next_stamp(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), 1, PRIMA_PROF_GEMV_QKV);
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(qkv)");
     c->ssq_attn = in.ssq_out;
     c->ssq_attn.eps = g.rms_eps;
     if (!seq) {
+      c->attn.stamp = next_stamp(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos0 + n_tok), 2);
       LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos0 + n_tok),
-               launch_attention(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k, L.v, g.kv_capacity, H, G, pos0, n_tok,
-                                c->attn, c->obuf, c->sm_count, st), "attention");
+               launch_attention(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, L.k, L.v, g.kv_capacity, H, G, pos0, stable_below,
+                                n_tok, c->attn, c->obuf, c->sm_count, st), "attention");
     } else {
       AttnSeqs as;                               // one request per token: its own cache, its own position
       as.n = n_tok;
@@ -497,19 +527,22 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
         as.pos[t] = pos[t];
         kv_bytes += static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos[t] + 1);
       }
+      c->attn.stamp = next_stamp(c, PRIMA_PROF_ATTENTION, kv_bytes, 2);
       LAUNCH_P(c, PRIMA_PROF_ATTENTION, kv_bytes,
-               launch_attention_seqs(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, as, g.kv_capacity, H, G, c->attn, c->obuf,
-                                     c->sm_count, st), "attention");
+               launch_attention_seqs(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, as, stable_below, g.kv_capacity, H, G, c->attn,
+                                     c->obuf, c->sm_count, st), "attention");
     }
     GemvIn in_o;                                 // O: plain attention output
     in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status; in_o.first_wait_polls = c->first_wait_polls;
     in_o.zero0 = c->acc_qkv; in_o.zero0_n = static_cast<int64_t>(n_tok) * L.qkv.mpad();
     in_o.zero1 = c->acc_down; in_o.zero1_n = static_cast<int64_t>(n_tok) * mpad_e;
     in_o.out_order = kOrderResidual;
+    in_o.stamp = next_stamp(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), 1, PRIMA_PROF_GEMV_O);
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->acc_o, c->sm_count, st), "gemv(o)");
     GemvIn in_f;                                 // gate/up: h_b + O projection -> h_a
     in_f.kind = kResidual; in_f.h_in = c->h_b; in_f.h_out = c->h_a; in_f.acc_in = c->acc_o; in_f.mpad_in = L.o.mpad();
     in_f.gain = L.g_ffn; in_f.ssq_out = c->ssq_ffn; in_f.status = c->status; in_f.out_order = kOrderSwiglu; in_f.first_wait_polls = c->first_wait_polls;
+    in_f.stamp = next_stamp(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), 1, PRIMA_PROF_GEMV_GATE_UP);
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.gu), launch_gemv_partials(L.gu, in_f, n_tok, c->acc_gu, c->sm_count, st), "gemv(gate/up)");
     c->ssq_ffn = in_f.ssq_out;
     c->ssq_ffn.eps = g.rms_eps;
@@ -517,6 +550,7 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
     in_d.kind = kSwiglu; in_d.acc_in = c->acc_gu; in_d.mpad_in = L.gu.mpad();
     in_d.ssq_in = c->ssq_ffn; in_d.status = c->status; in_d.out_order = kOrderResidual; in_d.first_wait_polls = c->first_wait_polls;
     in_d.zero0 = c->acc_o; in_d.zero0_n = static_cast<int64_t>(n_tok) * L.o.mpad();
+    in_d.stamp = next_stamp(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), 1, PRIMA_PROF_GEMV_DOWN);
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->acc_down, c->sm_count, st), "gemv(down)");
     h_in = c->h_a;
     acc_prev = c->acc_down;
@@ -570,6 +604,7 @@ int prima_logits(prima_ctx* c, const float* hidden, int n_tok, float* logits) {
   GemvIn in;        // the head stages hidden itself (no partial sums to add) and leaves its sums of squares
   in.kind = kResidual; in.h_in = hidden; in.h_out = c->h_b; in.acc_in = nullptr;
   in.mpad_in = (c->cfg.hidden + 7) / 8 * 8; in.gain = c->g_out; in.ssq_out = c->ssq_out; in.status = c->status; in.first_wait_polls = c->first_wait_polls;
+  in.stamp = next_stamp(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), 1, PRIMA_PROF_GEMV_HEAD);
   LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(c->head), launch_gemv_partials(c->head, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(head)");
   c->ssq_out = in.ssq_out;
   c->ssq_out.eps = c->cfg.rms_eps;
@@ -600,6 +635,7 @@ int prima_argmax(prima_ctx* c, const float* logits, int n_tok, int32_t* tokens_o
   cudaError_t e = cudaMemcpyAsync(tokens_out, c->am_out, static_cast<size_t>(n_tok) * 4, cudaMemcpyDeviceToHost, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "argmax readback");
+  c->unsynced_min_pos = 0x7fffffff;
   return PRIMA_OK;
 }
 
@@ -642,6 +678,7 @@ int prima_kv_load_seq(prima_ctx* c, int seq, int layer, int pos_begin, int n_pos
   }
   cudaError_t e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "kv_load sync");
+  c->unsynced_min_pos = 0x7fffffff;
   return PRIMA_OK;
 }
 
@@ -669,6 +706,7 @@ int prima_kv_read_seq(prima_ctx* c, int seq, int layer, int pos_begin, int n_pos
   }
   cudaError_t e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "kv_read sync");
+  c->unsynced_min_pos = 0x7fffffff;
   return PRIMA_OK;
 }
 
@@ -679,6 +717,7 @@ int prima_sync(prima_ctx* c) {
   cudaError_t e = cudaMemcpyAsync(&status, c->status, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync");
+  c->unsynced_min_pos = 0x7fffffff;
   if (status != 0) {      // reported once; whatever the failed step left in the accumulators is cleared, so the context stays usable
     queue_reset(c);
     e = cudaStreamSynchronize(c->stream);
@@ -706,8 +745,9 @@ int prima_ctx_set_option(prima_ctx* c, int option, int64_t value) {
   }
 }
 
-int prima_profile_enable(prima_ctx* c, int on) {
+int prima_profile_enable(prima_ctx* c, int mode) {
   if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_profile_enable: null context");
+  if (mode < 0 || mode > 2) return fail(c, PRIMA_ERR_ARG, "prima_profile_enable: mode must be 0, 1 or 2");
   DeviceGuard guard(c->cfg.device);
   cudaStreamSynchronize(c->stream);
   for (auto& sp : c->spans) {
@@ -715,7 +755,21 @@ int prima_profile_enable(prima_ctx* c, int on) {
     cudaEventDestroy(sp.b);
   }
   c->spans.clear();
-  c->profiling = on != 0;
+  c->stamp_info.clear();
+  c->profiling = mode == 1;
+  c->stamping = false;
+  if (mode == 2) {
+    if (!c->stamp_t0) {
+      int rc = dev_alloc(c, &c->stamp_t0, kMaxStamps);
+      if (rc == PRIMA_OK) rc = dev_alloc(c, &c->stamp_t1, kMaxStamps);
+      if (rc != PRIMA_OK) return rc;
+    }
+    cudaError_t e = cudaMemsetAsync(c->stamp_t0, 0xff, kMaxStamps * sizeof(unsigned long long), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->stamp_t1, 0, kMaxStamps * sizeof(unsigned long long), c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "prima_profile_enable");
+    c->stamping = true;
+  }
+  c->attn.stamp = Stamp();
   return PRIMA_OK;
 }
 
@@ -734,6 +788,20 @@ int prima_profile_read(prima_ctx* c, int klass, double* ms_total, int64_t* launc
     ms += t;
     n += sp.launches;
     bytes += sp.bytes;
+  }
+  if (!c->stamp_info.empty()) {
+    const size_t k = c->stamp_info.size();
+    std::vector<unsigned long long> t0(k), t1(k);
+    e = cudaMemcpy(t0.data(), c->stamp_t0, k * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(t1.data(), c->stamp_t1, k * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(c, e, "prima_profile_read(stamps)");
+    for (size_t i = 0; i < k; ++i) {
+      const bool match = c->stamp_info[i].klass == klass || (c->stamp_info[i].klass == PRIMA_PROF_GEMV && c->stamp_info[i].sub == klass);
+      if (!match || t1[i] <= t0[i]) continue;
+      ms += static_cast<double>(t1[i] - t0[i]) * 1e-6;
+      n += c->stamp_info[i].launches;
+      bytes += c->stamp_info[i].bytes;
+    }
   }
   *ms_total = ms;
   *launches = n;

@@ -20,8 +20,18 @@
 // the cache and keeps a copy in shared memory, from which its warps take them (the cache is never
 // read back inside the kernel).
 //
-// With at most eight query rows (one token) a CTA that takes several chunks carries its running state
-// from chunk to chunk and leaves one partial result (see the first branch of the chunk loop).
+// Two kernels.  attn_one_kernel serves at most eight query rows per KV head (one token per request):
+// a CTA that takes several chunks carries its running state from chunk to chunk and leaves ONE partial
+// result, and the merge is part of the same kernel: every CTA of a (request, KV head) takes a ticket
+// after it has written its partial result, and the CTA that draws the last ticket -- nobody waits for
+// anybody -- combines all of them in ascending order and writes the output rows.  attn_partial_kernel
+// + attn_merge_kernel serve a step of several tokens of one sequence (up to 64 query rows per KV head).
+//
+// Cache entries below `stable_below` were written before the host last waited for the stream, or by a
+// kernel at least one full step upstream whose completion the host has observed; only those are read
+// before the dependency wait.  Entries in [stable_below, pos) were appended by earlier steps that may
+// still be in flight when this kernel starts (programmatic dependent launch orders nothing before the
+// wait), so they are read after it.
 //
 // With several independent requests per step (one token each) the grid gets a third dimension: CTA
 // (chunk, KV head, request) works on that request's own cache and position, all in one launch.
@@ -30,9 +40,12 @@
 // HBM time): every warp requests the old entries of its positions before it waits for the
 // predecessor kernel, all loads of the finishing step are issued together, and the shared-memory
 // tiles are padded and swizzled so that neither their 16-byte stores nor their reads conflict.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace prima {
+bool attention_merge_is_fused();
 namespace {
 
 constexpr int kChunk = 128;
@@ -66,23 +79,10 @@ __device__ __forceinline__ int swz(int dim) { return dim ^ (((dim >> 5) & 1) << 
 __global__ void __launch_bounds__(kThreads, 2)
 attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
                     const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
-                    int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, int n_chunks, int chunk_stride,
-                    float* __restrict__ o_part, float2* __restrict__ ml_part, const AttnSeqs seqs) {
+                    int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int n_chunks, int chunk_stride,
+                    float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp) {
   pdl_trigger();
-  int row_base = 0;                 // first output row (token * heads) of this CTA's token(s)
-  if (seqs.n > 0) {                 // one request per blockIdx.z: its own cache and position, one token
-    const int tq = blockIdx.z;
-    k_cache = seqs.k[tq];
-    v_cache = seqs.v[tq];
-    pos = seqs.pos[tq];
-    n_tok = 1;
-    n_chunks = (pos + kChunk) / kChunk;
-    if (static_cast<int>(blockIdx.x) >= n_chunks) return;
-    acc += tq * mpad;
-    ssq += tq * kMaxStatBlocks;
-    rope_tab += tq * (kHeadDim / 2);
-    row_base = tq * n_q_heads;
-  }
+  constexpr int row_base = 0;
   extern __shared__ __align__(16) float dyn_smem[];
   __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
   __shared__ float s_inv[kMaxTok];
@@ -104,21 +104,21 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   uint4 vreg[4][2];      // [k-slot position][64-dim half]
   const __half* kbase = k_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
   const __half* vbase = v_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
-  // Entries below `pos` were written by earlier steps and do not change.
-  auto load_old = [&](int wbase) {
+  // Entries below `limit` (at most pos) are loaded from the cache, the others are left zero.
+  auto load_old = [&](int wbase, int limit) {
 #pragma unroll
     for (int pb = 0; pb < 2; ++pb) {
       const int p = wbase + 8 * pb + g;
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        kreg[pb][j] = p < pos ? __ldcg(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t)) : make_uint4(0, 0, 0, 0);
+        kreg[pb][j] = p < limit ? __ldcg(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t)) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
     for (int pi = 0; pi < 4; ++pi) {
       const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf)
-        vreg[pi][hf] = p < pos ? __ldcg(reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g)) : make_uint4(0, 0, 0, 0);
+        vreg[pi][hf] = p < limit ? __ldcg(reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g)) : make_uint4(0, 0, 0, 0);
     }
   };
   // Entries of this step come from shared memory.
@@ -143,8 +143,11 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   };
 
   int chunk = blockIdx.x;
-  load_old(chunk * kChunk + warp * 16);
+  const int pre_limit = min(pos, stable_below);
+  load_old(chunk * kChunk + warp * 16, pre_limit);
   pdl_wait();
+  stamp_begin(stamp);
+  if (pre_limit < pos && chunk * kChunk + warp * 16 + 16 > pre_limit) load_old(chunk * kChunk + warp * 16, pos);
 
   // ---- finish the QKV product for this KV head.  Items: one rotation pair of a query row, and for a
   //      CTA that owns a chunk with new positions also one pair of each new key and value.
@@ -224,137 +227,9 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   __syncthreads();
 
   const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
-  if (n_rows <= 8) {
-    // ---- At most eight query rows (one token): one tile, and a CTA that takes several chunks carries
-    //      its running (max, sum, output) from chunk to chunk instead of leaving one partial result per
-    //      chunk.  A warp keeps the un-normalised output of its positions in its own tile in shared memory
-    //      (every lane re-reads and re-writes only its own 32 floats, so the chunk loop has no barrier and
-    //      the warps' loads and arithmetic overlap freely); the warps are combined once, at the end, and
-    //      the CTA leaves ONE partial result, numbered by blockIdx.x.
-    const bool live = g < n_rows;
-    const int my_tok = live ? g / group : -1;
-    const float* qrow = q_s + (live ? g : 0) * kRowPad;
-    float* so = s_o + (warp * o_rows + g) * kRowPad;
-#pragma unroll
-    for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) *reinterpret_cast<float4*>(so + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
-    float m_run = -INFINITY, l_run = 0.f;      // of row g, the same in the four lanes of a quad
-    for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
-      const int wbase = chunk * kChunk + warp * 16;
-      if (!first) load_old(wbase);
-      patch_new(wbase);
-      float sc[2][4];
-#pragma unroll
-      for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-        if (live) {
-          a = *reinterpret_cast<const float4*>(qrow + swz(32 * j + 8 * t));
-          b = *reinterpret_cast<const float4*>(qrow + swz(32 * j + 8 * t) + 4);
-        }
-        const uint32_t qa0 = pack_h2(a.x * scale, a.y * scale), qa2 = pack_h2(a.z * scale, a.w * scale);
-        const uint32_t qb0 = pack_h2(b.x * scale, b.y * scale), qb2 = pack_h2(b.z * scale, b.w * scale);
-#pragma unroll
-        for (int pb = 0; pb < 2; ++pb) {      // rows 8..15 of the tile do not exist: zero operands
-          mma_f16(sc[pb], qa0, 0u, qa2, 0u, kreg[pb][j].x, kreg[pb][j].y);
-          mma_f16(sc[pb], qb0, 0u, qb2, 0u, kreg[pb][j].z, kreg[pb][j].w);
-        }
-      }
-      float mx = -INFINITY;
-#pragma unroll
-      for (int pb = 0; pb < 2; ++pb)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int p = wbase + 8 * pb + 2 * t + e;
-          const bool ok = live && p <= pos + my_tok;
-          sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
-          mx = fmaxf(mx, sc[pb][e]);
-        }
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float m_new = fmaxf(m_run, mx);
-      const float alpha = m_run > -INFINITY ? expf(m_run - m_new) : 1.0f;      // nothing accumulated yet: the tile is zero
-      float lsum = 0.f;
-      uint32_t pa[2];
-#pragma unroll
-      for (int pb = 0; pb < 2; ++pb) {
-        const float p0 = m_new > -INFINITY ? expf(sc[pb][0] - m_new) : 0.f;
-        const float p1 = m_new > -INFINITY ? expf(sc[pb][1] - m_new) : 0.f;
-        lsum += p0 + p1;
-        pa[pb] = pack_h2(p0, p1);
-      }
-      lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
-      lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
-      l_run = l_run * alpha + lsum;
-      m_run = m_new;
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll
-        for (int bh = 0; bh < 2; ++bh) {
-          float oc[4][4];
-#pragma unroll
-          for (int bb = 0; bb < 4; ++bb) {
-            const int b = 4 * bh + bb, j = b >> 1;
-            const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
-            const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
-            const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
-            const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
-            const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
-            const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
-            const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
-            oc[bb][0] = oc[bb][1] = oc[bb][2] = oc[bb][3] = 0.f;
-            mma_f16(oc[bb], pa[0], 0u, pa[1], 0u, b0, b1);
-          }
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            float4* dst = reinterpret_cast<float4*>(so + swz(64 * hf + 16 * t + 8 * e + 4 * bh));
-            const float4 old = *dst;
-            *dst = make_float4(fmaf(old.x, alpha, oc[0][e]), fmaf(old.y, alpha, oc[1][e]), fmaf(old.z, alpha, oc[2][e]), fmaf(old.w, alpha, oc[3][e]));
-          }
-        }
-      }
-    }
-    if (t == 0) {
-      s_m[warp][g] = m_run;
-      s_l[warp][g] = l_run;
-      s_m[warp][g + 8] = -INFINITY;
-      s_l[warp][g + 8] = 0.f;
-    }
-    __syncthreads();
-    if (threadIdx.x < kWarps * 16) {
-      const int w = threadIdx.x >> 4, r = threadIdx.x & 15;
-      float big = -INFINITY;
-#pragma unroll
-      for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
-      const float mine = s_m[w][r];
-      s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
-      if (w == 0) s_big[r] = big;
-    }
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < n_rows * (kHeadDim / 4); idx += kThreads) {
-      const int r = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
-      const int col = swz(d4);
-      float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
-      float l = 0.f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const float f = s_f[w][r];
-        const float4 v = *reinterpret_cast<const float4*>(s_o + (w * o_rows + r) * kRowPad + col);
-        l += f * s_l[w][r];
-        accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
-      }
-      const int tok = r / group, head = kv * group + r % group;
-      const int64_t slot = (static_cast<int64_t>(row_base) + static_cast<int64_t>(tok) * n_q_heads + head) * chunk_stride + blockIdx.x;
-      *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
-      if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
-    }
-    return;
-  }
   for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
     const int wbase = chunk * kChunk + warp * 16;      // first position of this warp
-    if (!first) load_old(wbase);
+    if (!first) load_old(wbase, pos);
     patch_new(wbase);
     for (int tile = 0; tile * 16 < n_rows; ++tile) {
       const bool hi_live = tile * 16 + 8 < n_rows;       // rows 8..15 of the tile exist
@@ -503,12 +378,348 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   }
 }
 
+// ---- at most eight query rows per KV head (one token per request), merge included ------------------
+// A CTA that takes several chunks carries its running (max, sum, output) from chunk to chunk: a warp
+// keeps the un-normalised output of its positions in its own tile in shared memory (every lane re-reads
+// and re-writes only its own 32 floats, so the chunk loop has no barrier and the warps' loads and
+// arithmetic overlap freely); the warps are combined once, at the end, and the CTA leaves ONE partial
+// result, numbered by blockIdx.x.  Then the ticket: the CTA that finds all the others' partial results
+// written combines them (ascending order, so the bits do not depend on who came last) and writes the
+// output rows of its KV head; with a single CTA per (request, KV head) the partial result is normalised
+// and written directly.
+constexpr int kMaxParts = 320;      // partial results per (request, KV head): at most 2 CTAs per SM / KV heads
+
+__global__ void __launch_bounds__(kThreads, 2)
+attn_one_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
+                const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
+                int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_chunks, int part_stride,
+                float* __restrict__ o_part, float2* __restrict__ ml_part, int* __restrict__ tickets, float* __restrict__ o,
+                const AttnSeqs seqs, const Stamp stamp) {
+  pdl_trigger();
+  int row_base = 0;                 // first output row (request * heads) of this CTA's request
+  if (seqs.n > 0) {                 // one request per blockIdx.z: its own cache and position
+    const int tq = blockIdx.z;
+    k_cache = seqs.k[tq];
+    v_cache = seqs.v[tq];
+    pos = seqs.pos[tq];
+    n_chunks = (pos + kChunk) / kChunk;
+    if (static_cast<int>(blockIdx.x) >= n_chunks) return;
+    acc += tq * mpad;
+    ssq += tq * kMaxStatBlocks;
+    rope_tab += tq * (kHeadDim / 2);
+    row_base = tq * n_q_heads;
+  }
+  extern __shared__ __align__(16) float dyn_smem[];
+  __shared__ float s_m[kWarps][8], s_l[kWarps][8], s_f[kWarps][8], s_big[8];
+  __shared__ float s_inv;
+  __shared__ int s_ticket;
+
+  const int group = n_q_heads / n_kv_heads;                            // query rows served by this CTA, at most 8
+  float* s_o = dyn_smem;                                               // [kWarps][8][kRowPad]
+  float* q_s = s_o + kWarps * 8 * kRowPad;                             // [group][kRowPad] rotated queries of this KV head
+  __half* new_k = reinterpret_cast<__half*>(q_s + 8 * kRowPad);        // [128] key of the new position
+  __half* new_v = new_k + kHeadDim;
+
+  const int kv = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int n_parts = min(static_cast<int>(gridDim.x), n_chunks);
+
+  uint4 kreg[2][4];      // [position block of 8][32-dim slice]
+  uint4 vreg[4][2];      // [k-slot position][64-dim half]
+  const __half* kbase = k_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
+  const __half* vbase = v_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
+  auto load_old = [&](int wbase, int limit) {
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) {
+      const int p = wbase + 8 * pb + g;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        kreg[pb][j] = p < limit ? __ldcg(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t)) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int pi = 0; pi < 4; ++pi) {
+      const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf)
+        vreg[pi][hf] = p < limit ? __ldcg(reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g)) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  // The entry of this step comes from shared memory.
+  auto patch_new = [&](int wbase) {
+    if (pos < wbase || pos >= wbase + 16) return;
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) {
+      if (wbase + 8 * pb + g == pos) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) kreg[pb][j] = *reinterpret_cast<const uint4*>(new_k + 32 * j + 8 * t);
+      }
+    }
+#pragma unroll
+    for (int pi = 0; pi < 4; ++pi) {
+      if (wbase + 2 * t + (pi & 1) + 8 * (pi >> 1) == pos) {
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) vreg[pi][hf] = *reinterpret_cast<const uint4*>(new_v + 64 * hf + 8 * g);
+      }
+    }
+  };
+
+  int chunk = blockIdx.x;
+  const int pre_limit = min(pos, stable_below);
+  load_old(chunk * kChunk + warp * 16, pre_limit);
+  pdl_wait();
+  stamp_begin(stamp);
+  if (pre_limit < pos && chunk * kChunk + warp * 16 + 16 > pre_limit) load_old(chunk * kChunk + warp * 16, pos);
+
+  // ---- finish the QKV product for this KV head.  Items: one rotation pair of a query row, and for the
+  //      CTA that owns the chunk with the new position also one pair of the new key and of the new value.
+  const bool owner = (pos / kChunk) % static_cast<int>(gridDim.x) == static_cast<int>(blockIdx.x);
+  const int n_q_items = group * (kHeadDim / 2);
+  const int n_items = n_q_items + (owner ? 2 * (kHeadDim / 2) : 0);      // at most 640: three per thread
+  {
+    constexpr int kTrip = 3;
+    acc_t ra[kTrip], rb[kTrip];
+    float2 cs[kTrip];
+#pragma unroll
+    for (int u = 0; u < kTrip; ++u) {
+      const int idx = threadIdx.x + u * kThreads;
+      if (idx < n_items) {
+        const int i = idx % (kHeadDim / 2);
+        int row0;
+        if (idx < n_q_items) row0 = (kv * group + idx / (kHeadDim / 2)) * kHeadDim;
+        else row0 = (n_q_heads + (idx - n_q_items < kHeadDim / 2 ? 0 : n_kv_heads) + kv) * kHeadDim;
+        const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
+        ra[u] = __ldcg(acc + row0 + a);
+        rb[u] = __ldcg(acc + row0 + b);
+        cs[u] = __ldcg(rope_tab + i);
+      }
+    }
+    if (threadIdx.x == 0) {      // the RMSNorm factor, loaded while the accumulators are on their way
+      float ss = 0.f;
+      for (int gi = 0; gi < n_groups; ++gi) ss += __ldcg(ssq + gi);
+      s_inv = 1.0f / sqrtf(ss * inv_width + eps);
+    }
+    __syncthreads();
+    const float inv = s_inv;
+#pragma unroll
+    for (int u = 0; u < kTrip; ++u) {
+      const int idx = threadIdx.x + u * kThreads;
+      if (idx < n_items) {
+        const int i = idx % (kHeadDim / 2);
+        const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
+        const float x = acc_value(ra[u]) * inv, y = acc_value(rb[u]) * inv;
+        if (idx < n_q_items) {
+          const int r = idx / (kHeadDim / 2);
+          q_s[r * kRowPad + swz(a)] = x * cs[u].x - y * cs[u].y;
+          q_s[r * kRowPad + swz(b)] = y * cs[u].x + x * cs[u].y;
+        } else {
+          const bool is_v = idx - n_q_items >= kHeadDim / 2;
+          const __half ha = __float2half_rn(is_v ? x : x * cs[u].x - y * cs[u].y);
+          const __half hb = __float2half_rn(is_v ? y : y * cs[u].x + x * cs[u].y);
+          __half* sm = is_v ? new_v : new_k;
+          sm[a] = ha;
+          sm[b] = hb;
+          __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + pos) * kHeadDim;
+          gd[a] = ha;
+          gd[b] = hb;
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
+  const bool live = g < group;
+  const float* qrow = q_s + (live ? g : 0) * kRowPad;
+  float* so = s_o + (warp * 8 + g) * kRowPad;
+#pragma unroll
+  for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) *reinterpret_cast<float4*>(so + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+  float m_run = -INFINITY, l_run = 0.f;      // of row g, the same in the four lanes of a quad
+  for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
+    const int wbase = chunk * kChunk + warp * 16;
+    if (!first) load_old(wbase, pos);
+    patch_new(wbase);
+    float sc[2][4];
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+      if (live) {
+        a = *reinterpret_cast<const float4*>(qrow + swz(32 * j + 8 * t));
+        b = *reinterpret_cast<const float4*>(qrow + swz(32 * j + 8 * t) + 4);
+      }
+      const uint32_t qa0 = pack_h2(a.x * scale, a.y * scale), qa2 = pack_h2(a.z * scale, a.w * scale);
+      const uint32_t qb0 = pack_h2(b.x * scale, b.y * scale), qb2 = pack_h2(b.z * scale, b.w * scale);
+#pragma unroll
+      for (int pb = 0; pb < 2; ++pb) {      // rows 8..15 of the tile do not exist: zero operands
+        mma_f16(sc[pb], qa0, 0u, qa2, 0u, kreg[pb][j].x, kreg[pb][j].y);
+        mma_f16(sc[pb], qb0, 0u, qb2, 0u, kreg[pb][j].z, kreg[pb][j].w);
+      }
+    }
+    float mx = -INFINITY;
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int p = wbase + 8 * pb + 2 * t + e;
+        const bool ok = live && p <= pos;
+        sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
+        mx = fmaxf(mx, sc[pb][e]);
+      }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(m_run, mx);
+    const float alpha = m_run > -INFINITY ? expf(m_run - m_new) : 1.0f;      // nothing accumulated yet: the tile is zero
+    float lsum = 0.f;
+    uint32_t pa[2];
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) {
+      const float p0 = m_new > -INFINITY ? expf(sc[pb][0] - m_new) : 0.f;
+      const float p1 = m_new > -INFINITY ? expf(sc[pb][1] - m_new) : 0.f;
+      lsum += p0 + p1;
+      pa[pb] = pack_h2(p0, p1);
+    }
+    lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+    lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+    l_run = l_run * alpha + lsum;
+    m_run = m_new;
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+      for (int bh = 0; bh < 2; ++bh) {
+        float oc[4][4];
+#pragma unroll
+        for (int bb = 0; bb < 4; ++bb) {
+          const int b = 4 * bh + bb, j = b >> 1;
+          const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
+          const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
+          const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
+          const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
+          const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
+          const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
+          const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
+          oc[bb][0] = oc[bb][1] = oc[bb][2] = oc[bb][3] = 0.f;
+          mma_f16(oc[bb], pa[0], 0u, pa[1], 0u, b0, b1);
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float4* dst = reinterpret_cast<float4*>(so + swz(64 * hf + 16 * t + 8 * e + 4 * bh));
+          const float4 old = *dst;
+          *dst = make_float4(fmaf(old.x, alpha, oc[0][e]), fmaf(old.y, alpha, oc[1][e]), fmaf(old.z, alpha, oc[2][e]), fmaf(old.w, alpha, oc[3][e]));
+        }
+      }
+    }
+  }
+  if (t == 0) {
+    s_m[warp][g] = m_run;
+    s_l[warp][g] = l_run;
+  }
+  __syncthreads();
+  if (threadIdx.x < kWarps * 8) {
+    const int w = threadIdx.x >> 3, r = threadIdx.x & 7;
+    float big = -INFINITY;
+#pragma unroll
+    for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
+    const float mine = s_m[w][r];
+    s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
+    if (w == 0) s_big[r] = big;
+  }
+  __syncthreads();
+  // thread (row r, four head dims) adds up the eight warps' tiles
+  const int r = threadIdx.x >> 5, d4 = lane * 4;
+  const int64_t out_row = static_cast<int64_t>(row_base) + kv * group + r;
+  float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
+  float l = 0.f;
+  if (r < group) {
+    const int col = swz(d4);
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float f = s_f[w][r];
+      const float4 v = *reinterpret_cast<const float4*>(s_o + (w * 8 + r) * kRowPad + col);
+      l += f * s_l[w][r];
+      accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
+    }
+  }
+  if (n_parts == 1 && tickets != nullptr) {      // nothing to merge
+    if (r < group) *reinterpret_cast<float4*>(o + out_row * kHeadDim + d4) = make_float4(accum.x / l, accum.y / l, accum.z / l, accum.w / l);
+    stamp_end(stamp);
+    return;
+  }
+  if (r < group) {
+    const int64_t slot = out_row * part_stride + blockIdx.x;
+    *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
+    if (lane == 0) ml_part[slot] = make_float2(s_big[r], l);
+  }
+  if (tickets == nullptr) {      // the merge is a kernel of its own
+    stamp_end(stamp);
+    return;
+  }
+  // ---- the ticket: partial results first, visible to the whole GPU, then the count
+  __threadfence();
+  __syncthreads();
+  int* ticket = tickets + (seqs.n > 0 ? static_cast<int>(blockIdx.z) : 0) * n_kv_heads + kv;
+  if (threadIdx.x == 0) {
+    const int drawn = atomicAdd(ticket, 1);
+    if (drawn == n_parts - 1) *ticket = 0;      // all have arrived: ready for the next launch
+    s_ticket = drawn;
+  }
+  __syncthreads();
+  if (s_ticket != n_parts - 1) {
+    stamp_end(stamp);
+    return;
+  }
+  __threadfence();
+  // ---- merge: warp r owns output row r.  Weights e^(m_c - M) of the parts go to shared memory (the tiles
+  //      are no longer needed), then every lane adds up its four head dims over the parts in ascending order.
+  float* s_w = s_o + r * kMaxParts;      // kMaxParts floats per row; 8 rows fit in the first tiles
+  if (r < group) {
+    const float2* ml = ml_part + out_row * part_stride;
+    float big = -INFINITY;
+    for (int c = lane; c < n_parts; c += 32) big = fmaxf(big, __ldcg(ml + c).x);
+#pragma unroll
+    for (int of = 16; of > 0; of >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, of));
+    float den = 0.f;
+    for (int c = lane; c < n_parts; c += 32) {
+      const float2 v = __ldcg(ml + c);
+      const float w = v.x > -INFINITY ? expf(v.x - big) : 0.f;
+      s_w[c] = w;
+      den += w * v.y;
+    }
+#pragma unroll
+    for (int of = 16; of > 0; of >>= 1) den += __shfl_xor_sync(0xffffffffu, den, of);
+    __syncwarp();
+    const float* op = o_part + out_row * part_stride * kHeadDim + d4;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    int c = 0;
+    for (; c + 8 <= n_parts; c += 8) {      // eight loads in flight
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = __ldcg(reinterpret_cast<const float4*>(op + static_cast<int64_t>(c + u) * kHeadDim));
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float w = s_w[c + u];
+        sum.x += w * v[u].x; sum.y += w * v[u].y; sum.z += w * v[u].z; sum.w += w * v[u].w;
+      }
+    }
+    for (; c < n_parts; ++c) {
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(op + static_cast<int64_t>(c) * kHeadDim));
+      const float w = s_w[c];
+      sum.x += w * v.x; sum.y += w * v.y; sum.z += w * v.z; sum.w += w * v.w;
+    }
+    *reinterpret_cast<float4*>(o + out_row * kHeadDim + d4) = make_float4(sum.x / den, sum.y / den, sum.z / den, sum.w / den);
+  }
+  stamp_end(stamp);
+}
+
 // One block of 128 threads per (token, head): merge the chunks in ascending order.  Thread d owns
 // head dim d.  The partial outputs of the first kMergePre chunks are requested before anything
 // else, together with the (max, sum) pairs, so that the kernel costs one round trip to L2.
 __global__ void __launch_bounds__(kHeadDim)
 attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, int n_chunks, int chunk_stride, int n_q_heads,
-                  float* __restrict__ o, const AttnSeqs seqs) {
+                  float* __restrict__ o, const AttnSeqs seqs, const Stamp stamp) {
   pdl_trigger();
   pdl_wait();
   if (seqs.n > 0) n_chunks = min(n_chunks, (seqs.pos[blockIdx.x / n_q_heads] + kChunk) / kChunk);      // the row's own request
@@ -549,6 +760,7 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
 #pragma unroll 8
   for (int c = kMergePre; c < n_chunks; ++c) accum += s_w[c] * __ldcg(op + static_cast<int64_t>(c) * kHeadDim);
   o[static_cast<int64_t>(row) * kHeadDim + d] = accum / denom;
+  stamp_end(stamp);
 }
 
 size_t partial_smem_bytes(int n_rows, int n_tok) {
@@ -556,17 +768,34 @@ size_t partial_smem_bytes(int n_rows, int n_tok) {
   return static_cast<size_t>(kWarps * o_rows + n_rows) * kRowPad * sizeof(float) + static_cast<size_t>(2) * n_tok * kHeadDim * sizeof(__half);
 }
 
+constexpr size_t kOneSmemBytes = static_cast<size_t>(kWarps * 8 + 8) * kRowPad * sizeof(float) + 2 * kHeadDim * sizeof(__half);
+static_assert(8 * kMaxParts <= kWarps * 8 * kRowPad, "the merge weights reuse the tiles");
+
 }  // namespace
 
 int attention_chunk_len() { return kChunk; }
 
-static int configure_partial_kernel() {
+// Where the partial results of a one-token step are merged.  Default: a second, small kernel (one block per
+// output row: the reads of all rows proceed in parallel).  PRIMA_ATTN_MERGE=fused (read once per process): inside
+// the attention kernel, by the last CTA of each KV head to finish; one launch less, but that CTA reads its eight
+// rows' partial results alone, which measured 1.7 us per layer slower at 4096 positions on the 70B shape.
+bool attention_merge_is_fused() {
+  static const bool fused = [] {
+    const char* v = getenv("PRIMA_ATTN_MERGE");
+    return v && v[0] == 'f';
+  }();
+  return fused;
+}
+
+static int configure_kernels() {
   static bool configured[kMaxDevices] = {};
   int dev = -1;
   if (first_launch_on_device(configured, &dev)) {
     cudaError_t e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(partial_smem_bytes(8 * kMaxTok, kMaxTok)));
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kOneSmemBytes));
+    if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e0 != cudaSuccess) return cuda_rc(e0);
     if (dev >= 0) configured[dev] = true;
   }
@@ -574,51 +803,63 @@ static int configure_partial_kernel() {
 }
 
 int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, __half* k_cache,
-                     __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok, const AttnScratch& scr, float* o,
-                     int sm_count, cudaStream_t st) {
+                     __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok,
+                     const AttnScratch& scr, float* o, int sm_count, cudaStream_t st) {
   const int n_ctx = pos + n_tok;
   const int n_chunks = (n_ctx + kChunk - 1) / kChunk;
   if (n_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
-  const int n_rows = n_tok * (n_q_heads / n_kv_heads);
-  const int rc = configure_partial_kernel();
+  const int group = n_q_heads / n_kv_heads;
+  const int n_rows = n_tok * group;
+  const int rc = configure_kernels();
   if (rc != 0) return rc;
+  const float inv_width = ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f;
   // Two CTAs fit on an SM: with more chunks than that, a CTA takes several (gridDim.x apart).
-  const int per_head = std::max(1, 2 * sm_count / n_kv_heads);
+  const int per_head = std::min(kMaxParts, std::max(1, 2 * sm_count / n_kv_heads));
   dim3 grid(std::min(n_chunks, per_head), n_kv_heads);
   const AttnSeqs none{};
+  if (n_tok == 1) {
+    int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;
+    cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
+                               ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads,
+                               pos, stable_below, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, none, scr.stamp);
+    if (e != cudaSuccess) return cuda_rc(e);
+    if (tickets) return 1;
+    e = launch_pdl(attn_merge_kernel, dim3(n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * grid.x) * sizeof(float), st, scr.o_part,
+                   scr.ml_part, static_cast<int>(grid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
+    return e == cudaSuccess ? 2 : cuda_rc(e);
+  }
   cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), partial_smem_bytes(n_rows, n_tok), st, acc_qkv, mpad,
-                             static_cast<const float*>(ssq.data), ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f,
-                             ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, n_tok, n_chunks,
-                             n_chunks, scr.o_part, scr.ml_part, none);
+                             static_cast<const float*>(ssq.data), ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache,
+                             kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok, n_chunks, n_chunks, scr.o_part, scr.ml_part,
+                             scr.stamp);
   if (e != cudaSuccess) return cuda_rc(e);
-  // with at most eight query rows a CTA leaves one partial result, however many chunks it took
-  const int n_parts = n_rows <= 8 ? static_cast<int>(grid.x) : n_chunks;
-  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * n_parts) * sizeof(float), st,
-                 scr.o_part, scr.ml_part, n_parts, n_chunks, n_q_heads, o, none);
+  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * n_chunks) * sizeof(float), st,
+                 scr.o_part, scr.ml_part, n_chunks, n_chunks, n_q_heads, o, none, scr.stamp);
   if (e != cudaSuccess) return cuda_rc(e);
   return 2;
 }
 
 int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, const AttnSeqs& seqs,
-                          int kv_capacity, int n_q_heads, int n_kv_heads, const AttnScratch& scr, float* o, int sm_count, cudaStream_t st) {
+                          int stable_below, int kv_capacity, int n_q_heads, int n_kv_heads, const AttnScratch& scr, float* o, int sm_count,
+                          cudaStream_t st) {
   if (seqs.n < 1 || seqs.n > kMaxTok) return cuda_rc(cudaErrorInvalidValue);
   int max_chunks = 1;
   for (int t = 0; t < seqs.n; ++t) max_chunks = std::max(max_chunks, (seqs.pos[t] + kChunk) / kChunk);
   if (max_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
-  const int rc = configure_partial_kernel();
+  const int rc = configure_kernels();
   if (rc != 0) return rc;
-  const int group = n_q_heads / n_kv_heads;
-  const int per_head = std::max(1, 2 * sm_count / n_kv_heads);
+  const int per_head = std::min(kMaxParts, std::max(1, 2 * sm_count / n_kv_heads));
   dim3 grid(std::min(max_chunks, per_head), n_kv_heads, seqs.n);      // CTAs beyond a request's own chunks leave at once
-  cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), partial_smem_bytes(group, 1), st, acc_qkv, mpad,
-                             static_cast<const float*>(ssq.data), ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f,
-                             ssq.eps, rope_tab, rope_mode, static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads,
-                             n_kv_heads, 0, 1, max_chunks, max_chunks, scr.o_part, scr.ml_part, seqs);
+  int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;
+  cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
+                             ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps, rope_tab, rope_mode,
+                             static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads, n_kv_heads, 0, stable_below,
+                             max_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, seqs, scr.stamp);
   if (e != cudaSuccess) return cuda_rc(e);
-  e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * max_chunks) * sizeof(float), st,
-                 scr.o_part, scr.ml_part, static_cast<int>(grid.x), max_chunks, n_q_heads, o, seqs);
-  if (e != cudaSuccess) return cuda_rc(e);
-  return 2;
+  if (tickets) return 1;
+  e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * grid.x) * sizeof(float), st, scr.o_part,
+                 scr.ml_part, static_cast<int>(grid.x), scr.max_chunks, n_q_heads, o, seqs, scr.stamp);
+  return e == cudaSuccess ? 2 : cuda_rc(e);
 }
 
 }  // namespace prima

@@ -43,6 +43,15 @@ constexpr int kMaxTok = 8;
 constexpr int kMaxStatBlocks = 256;
 constexpr int kHeadDim = 128;
 
+// In-situ timing of one launch (prima_profile_enable mode 2): t0 receives the earliest %globaltimer
+// reading (ns) at which a CTA got past its dependency wait, t1 the latest at which a CTA finished.
+// Intervals of consecutive kernels of a stream do not overlap (a kernel passes its wait only after its
+// predecessor has completed), so their sum never exceeds the time of the step they belong to.
+struct Stamp {
+  unsigned long long* t0 = nullptr;   // device words, or null: not stamped
+  unsigned long long* t1 = nullptr;
+};
+
 struct TiledMat {
   uint8_t* data = nullptr;   // device, n_sb * n_rt * 1152 bytes
   int64_t rows = 0;          // logical rows (of the fused matrix)
@@ -134,6 +143,7 @@ struct GemvIn {
   int64_t zero1_n = 0;
   int* status = nullptr;           // device word: bit 0 set if a bounded wait gave up, bit 1 if a partial sum was out of range
   uint32_t first_wait_polls = 0;   // 0: the ordinary limit; otherwise the poll limit of every warp's first wait + 1 (test hook)
+  Stamp stamp;
 };
 int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, int sm_count, cudaStream_t st);
 
@@ -163,6 +173,8 @@ struct AttnScratch {
   float* o_part;    // [n_tok*H][n_chunks][128]
   float2* ml_part;  // [n_tok*H][n_chunks]  (running max, running sum)
   int max_chunks;
+  int* tickets;     // [kMaxTok][G], all zero between launches (see attn_one_kernel)
+  Stamp stamp;      // of the next attention launch (both kernels share it)
 };
 // Several independent requests in one launch: token t of the step belongs to a request with its own
 // cache (k[t], v[t]) and position pos[t]; rows, statistics, rotary table and outputs of token t are
@@ -173,10 +185,12 @@ struct AttnSeqs {
   int pos[kMaxTok];
   int n = 0;
 };
+// stable_below: cache entries at positions below it may be read before the kernel's dependency wait (see attention.cu).
 int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode, const AttnSeqs& seqs,
-                          int kv_capacity, int n_q_heads, int n_kv_heads, const AttnScratch& scr, float* o, int sm_count, cudaStream_t st);
+                          int stable_below, int kv_capacity, int n_q_heads, int n_kv_heads, const AttnScratch& scr, float* o, int sm_count,
+                          cudaStream_t st);
 int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const float2* rope_tab, int rope_mode,
-                     __half* k_cache, __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int n_tok,
+                     __half* k_cache, __half* v_cache, int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok,
                      const AttnScratch& scr, float* o, int sm_count, cudaStream_t st);
 int attention_chunk_len();
 
@@ -225,6 +239,22 @@ __device__ __forceinline__ int64_t acc_position(int order, int64_t r) {
   return r;
 }
 __device__ __forceinline__ acc_t acc_from(float v) { return static_cast<acc_t>(__float2ll_rn(v * kAccScale)); }
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Called by every thread of the CTA: right after the dependency wait / at the very end.
+__device__ __forceinline__ void stamp_begin(const Stamp& s) {
+  if (s.t0 && threadIdx.x == 0) atomicMin(s.t0, global_ns());
+}
+__device__ __forceinline__ void stamp_end(const Stamp& s) {
+  if (s.t1) {
+    __syncthreads();
+    if (threadIdx.x == 0) atomicMax(s.t1, global_ns());
+  }
+}
 
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -120,6 +120,7 @@ struct GemvParams {
   int64_t zero1_n;
   int out_order;
   int* status;
+  Stamp stamp;
   uint32_t first_wait_polls;   // poll limit of a warp's first wait (kWaitLimit in normal use; a test lowers it to exercise the give-up path)
 };
 

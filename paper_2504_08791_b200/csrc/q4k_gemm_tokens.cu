@@ -137,7 +137,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
   };
   if (p0 >= p1) {
     pdl_wait();
+    stamp_begin(P.stamp);
     clear_arrays();
+    stamp_end(P.stamp);
     return;
   }
 
@@ -193,6 +195,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
     if (!waited) {
       pdl_wait();
       waited = true;
+      stamp_begin(P.stamp);
       clear_arrays();
     }
     {
@@ -341,6 +344,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 2) gemv_tokens_kernel(const Ge
     }
   }
   if (!alive) drain.drain(bar_u32, kRingTok);
+  stamp_end(P.stamp);
 }
 
 }  // namespace

@@ -255,7 +255,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   };
   if (p0 >= p1) {
     pdl_wait();
+    stamp_begin(P.stamp);
     clear_arrays();
+    stamp_end(P.stamp);
     return;
   }
 
@@ -310,6 +312,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     if (!waited) {      // the first weight batches are on their way; everything below depends on the predecessor kernel
       pdl_wait();
       waited = true;
+      stamp_begin(P.stamp);
       clear_arrays();
     }
     {
@@ -417,6 +420,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
   }
   // A wait gave up: copies may still be on their way to this CTA's shared memory.
   if (!alive) drain.drain(bar_u32, kRing);
+  stamp_end(P.stamp);
 }
 
 size_t gemv_smem_bytes(int sg, int n_tok) {
@@ -476,6 +480,7 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
   P.n_tok_total = n_tok; P.acc = acc; P.mpad = w.mpad(); P.status = in.status;
   P.zero0 = in.zero0; P.zero0_n = in.zero0_n; P.zero1 = in.zero1; P.zero1_n = in.zero1_n;
   P.out_order = in.out_order;
+  P.stamp = in.stamp;
   P.first_wait_polls = in.first_wait_polls ? in.first_wait_polls - 1 : kWaitLimit;
   if ((in.out_order == kOrderResidual && w.mpad() % 256 != 0) || (in.out_order == kOrderSwiglu && w.mpad() % 512 != 0)) return cuda_rc(cudaErrorInvalidValue);
   int launches = 0;

@@ -319,3 +319,29 @@ def test_a_launch_refused_in_mid_window_leaves_the_next_call_clean(gpu, after):
     again = p.gpu_window(0, cfg["n_layers"], h0, pos)
     assert np.array_equal(again.view(np.uint32), good.view(np.uint32))
     p.close()
+
+
+def test_merge_inside_the_attention_kernel_matches_checker():
+    """PRIMA_ATTN_MERGE=fused (read once per process, hence the child process): the last CTA of a KV head merges."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np, torch, oracle\n"
+        "from paper_2504_08791_b200 import binding, synth\n"
+        "from tests.test_gpu_model import Pair, _hidden_close\n"
+        "for name, pos in (('tiny', 0), ('small', 300), ('tiny', 5000)):\n"
+        "    cfg = synth.model_config(name, kv_capacity=5100)\n"
+        "    p = Pair((torch, binding), cfg, seed=59, n_prefill=pos)\n"
+        "    h0 = synth.activations(59, 1, cfg['hidden'])\n"
+        "    want = p.ref.forward_window(0, cfg['n_layers'], h0, pos)\n"
+        "    a = p.gpu_window(0, cfg['n_layers'], h0, pos)\n"
+        "    b = p.gpu_window(0, cfg['n_layers'], h0, pos)\n"
+        "    _hidden_close(a, want)\n"
+        "    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))\n"
+        "    p.close()\n"
+        "print('fused merge ok')\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, PRIMA_ATTN_MERGE="fused", PYTHONPATH=root)
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "fused merge ok" in out.stdout, out.stdout + out.stderr
