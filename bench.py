@@ -230,6 +230,7 @@ def run_ours(args, rank, world, local_rank):
     if args.layers:
         cfg["n_layers"] = args.layers
     cfg["kv_capacity"] = max(cfg["kv_capacity"], n_ctx + 64 * args.n_tok)
+    cfg["max_n_tok"] = max(cfg.get("max_n_tok", 8), args.requests)
     L = cfg["n_layers"]
     seed = SEEDS[args.workload] + 1000 * rank
     R = args.requests

@@ -53,7 +53,8 @@ extern "C" {
 
 #define PRIMA_Q4K_BLOCK_BYTES 144
 #define PRIMA_Q4K_BLOCK_WEIGHTS 256
-#define PRIMA_MAX_N_TOK 8
+#define PRIMA_MAX_N_TOK 8   /* tokens of one sequence per step (prima_forward_window)            */
+#define PRIMA_MAX_N_SEQ 16  /* requests per step (prima_forward_window_seqs), columns of a product  */
 
 /* tensor ids for prima_load_q4k_weights */
 enum {
@@ -83,7 +84,8 @@ typedef struct {
   int32_t ffn;         /* F; multiple of 256                                                    */
   int32_t vocab;       /* V                                                                     */
   int32_t kv_capacity; /* positions per layer in the fp16 KV cache                              */
-  int32_t max_n_tok;   /* largest n_tok of a step, 1..PRIMA_MAX_N_TOK                           */
+  int32_t max_n_tok;   /* largest number of tokens of a step, 1..PRIMA_MAX_N_SEQ (prima_forward_window
+                          itself takes at most PRIMA_MAX_N_TOK)                                 */
   float rms_eps;
   float rope_theta;
   int32_t rope_mode;   /* 0: rotate pairs (i, i + head_dim/2); 1: pairs (2i, 2i+1)              */
@@ -228,7 +230,7 @@ int prima_profile_read(prima_ctx* ctx, int klass, double* ms_total, int64_t* lau
  * cudaStream_t or NULL. */
 int prima_dequant_q4k(const void* dev_blocks, int64_t n_superblocks, float* dev_out, void* stream);
 
-/* y[c][r] = sum_k W[r][k] x[c][k] for c < n_cols (1..8).  dev_w: standard layout; dev_x: fp32
+/* y[c][r] = sum_k W[r][k] x[c][k] for c < n_cols (1..16).  dev_w: standard layout; dev_x: fp32
  * [n_cols x cols]; dev_y: fp32 [n_cols x rows].  Allocates and frees its own temporary buffers
  * (tiled copy of W and scratch) and waits for completion; meant for testing single projections.
  * Returns PRIMA_ERR_DEVICE if a partial sum left the accumulator range (see prima_forward_window).

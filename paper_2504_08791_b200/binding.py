@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libprima.so")
 
 OK, ERR_ARG, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_DEVICE = 0, -1, -2, -3, -4, -5
 ATTN_NORM, WQ, WK, WV, WO, FFN_NORM, W_GATE, W_UP, W_DOWN, OUT_NORM, W_HEAD, TOK_EMBD = range(12)
-MAX_N_TOK = 8
+MAX_N_TOK = 8      # tokens of one sequence per step
+MAX_N_SEQ = 16     # requests per step / columns of a product
 PROF_GEMV, PROF_ATTENTION = 0, 1
 PROF_GEMV_QKV, PROF_GEMV_O, PROF_GEMV_GATE_UP, PROF_GEMV_DOWN, PROF_GEMV_HEAD = 16, 17, 18, 19, 20
 OPT_FIRST_WAIT_POLLS = 1

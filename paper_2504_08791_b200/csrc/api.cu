@@ -294,7 +294,7 @@ int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx
   const prima_model_config& g = *cfg;
   if (g.n_layers < 1 || g.hidden < 256 || g.hidden % 256 || g.ffn < 256 || g.ffn % 256 || g.head_dim != kHeadDim ||
       g.n_q_heads < 1 || g.n_kv_heads < 1 || g.n_q_heads % g.n_kv_heads || g.n_q_heads / g.n_kv_heads > 8 ||
-      g.n_q_heads > kMaxStatBlocks || g.vocab < 1 || g.kv_capacity < 1 || g.max_n_tok < 1 || g.max_n_tok > PRIMA_MAX_N_TOK ||
+      g.n_q_heads > kMaxStatBlocks || g.vocab < 1 || g.kv_capacity < 1 || g.max_n_tok < 1 || g.max_n_tok > PRIMA_MAX_N_SEQ ||
       !(g.rms_eps >= 0.f) || !(g.rope_theta > 0.f) || (g.rope_mode != 0 && g.rope_mode != 1) || g.device < 0)
     return fail(nullptr, PRIMA_ERR_ARG, "prima_ctx_create: inconsistent model shape");
   int n_dev = 0;
@@ -575,6 +575,7 @@ int prima_forward_window(prima_ctx* c, int layer_begin, int layer_end, const flo
   if (!c) return fail(nullptr, PRIMA_ERR_ARG, "prima_forward_window: null context");
   int rc = window_args_ok(c, "prima_forward_window", layer_begin, layer_end, hidden_in, hidden_out, n_tok);
   if (rc != PRIMA_OK) return rc;
+  if (n_tok > PRIMA_MAX_N_TOK) return fail(c, PRIMA_ERR_ARG, "a step of one sequence takes at most 8 tokens");
   if (pos < 0 || static_cast<int64_t>(pos) + n_tok > c->cfg.kv_capacity) return fail(c, PRIMA_ERR_ARG, "pos + n_tok exceeds kv_capacity");
   return forward_window_impl(c, layer_begin, layer_end, hidden_in, hidden_out, pos, n_tok, nullptr, nullptr);
 }
@@ -824,7 +825,7 @@ int prima_dequant_q4k(const void* dev_blocks, int64_t n_superblocks, float* dev_
 
 int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int max_n_cols, prima_gemv_plan** out) {
   if (out) *out = nullptr;
-  if (!dev_w || !out || rows < 1 || cols < 256 || cols % 256 || max_n_cols < 1 || max_n_cols > PRIMA_MAX_N_TOK)
+  if (!dev_w || !out || rows < 1 || cols < 256 || cols % 256 || max_n_cols < 1 || max_n_cols > PRIMA_MAX_N_SEQ)
     return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_plan_create: bad argument");
   prima_gemv_plan* p = new (std::nothrow) prima_gemv_plan();
   if (!p) return fail(nullptr, PRIMA_ERR_NOMEM, "out of host memory");
@@ -874,7 +875,7 @@ int prima_gemv_plan_destroy(prima_gemv_plan* p) {
 }
 
 int prima_gemv_q4k(const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols, float* dev_y, void* stream) {
-  if (!dev_x || !dev_y || n_cols < 1 || n_cols > PRIMA_MAX_N_TOK) return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_q4k: bad argument");
+  if (!dev_x || !dev_y || n_cols < 1 || n_cols > PRIMA_MAX_N_SEQ) return fail(nullptr, PRIMA_ERR_ARG, "prima_gemv_q4k: bad argument");
   prima_gemv_plan* p = nullptr;
   int rc = prima_gemv_plan_create(dev_w, rows, cols, n_cols, &p);
   if (rc != PRIMA_OK) return rc;

@@ -85,7 +85,7 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   constexpr int row_base = 0;
   extern __shared__ __align__(16) float dyn_smem[];
   __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
-  __shared__ float s_inv[kMaxTok];
+  __shared__ float s_inv[kMaxStepTok];
 
   const int group = n_q_heads / n_kv_heads;
   const int n_rows = n_tok * group;                  // query rows served by this CTA
@@ -792,7 +792,7 @@ static int configure_kernels() {
   int dev = -1;
   if (first_launch_on_device(configured, &dev)) {
     cudaError_t e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(partial_smem_bytes(8 * kMaxTok, kMaxTok)));
+                                          static_cast<int>(partial_smem_bytes(8 * kMaxStepTok, kMaxStepTok)));
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kOneSmemBytes));
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);

@@ -21,9 +21,12 @@ namespace prima {
 //                     f_t = sc_t | sc_{t+4} << 6 | m_t << 12 | m_{t+4} << 18  (24 bits, t = 0..3)
 //                     word1 = f_0 | (f_3 & 0xff) << 24, word2 = f_1 | (f_3 >> 8 & 0xff) << 24,
 //                     word3 = f_2 | (f_3 >> 16) << 24
-//   bytes  128..639   nibbles of sub-blocks 0..3: lane (g, t) = g*4 + t owns 16 bytes at lane*16,
-//                     the 32 weights of row g, sub-block t
-//   bytes  640..1151  the same for sub-blocks 4..7 (lane (g, t) owns sub-block 4 + t)
+//   bytes  128..639   nibbles of sub-blocks 0..3: the 16-byte piece of (row g, sub-block t), its 32
+//                     weights, sits at piece slot  4 g + (t ^ ((g >> 1) & 3))  (unit_piece_slot below)
+//   bytes  640..1151  the same for sub-blocks 4..7 (piece of (row g, sub-block 4 + t))
+// The exchange of pieces inside a row serves two readers at once: lane (g, t) of a warp reading its own
+// piece (any eight consecutive lanes then cover eight different 16-byte bank groups), and a matrix load
+// (ldmatrix) of the eight rows' pieces of ONE sub-block, which also wants eight different bank groups.
 //
 // Inside a 16-byte sub-block chunk, word w (0..3) holds weights 8w..8w+7, weight 8w+i in bits
 // 4i..4i+3, so that (word & 0x0f0f0f0f) is four weights (8w, 8w+2, 8w+4, 8w+6) as unsigned bytes and
@@ -36,10 +39,13 @@ namespace prima {
 // Rows are padded with zero blocks up to a multiple of 8.
 // ---------------------------------------------------------------------------------------------
 constexpr int kUnitBytes = 1152;
+// Slot (of 16 bytes, inside a 512-byte nibble tile) of the piece of (row g, sub-block t of the tile's four).
+__host__ __device__ constexpr int unit_piece_slot(int g, int t) { return 4 * g + (t ^ ((g >> 1) & 3)); }
 constexpr int kUnitHdrBytes = 128;
 constexpr int kRowsPerTile = 8;
 constexpr int kBlockBytes = 144;
-constexpr int kMaxTok = 8;
+constexpr int kMaxTok = 16;        // tokens of a step of independent requests (one each)
+constexpr int kMaxStepTok = 8;     // tokens of a step of one sequence (causal among themselves)
 constexpr int kMaxStatBlocks = 256;
 constexpr int kHeadDim = 128;
 

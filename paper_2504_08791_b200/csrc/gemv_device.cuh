@@ -88,6 +88,13 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
 }
 
 
+// The same with a zero accumulator: D = A * B (no registers have to be cleared for it).
+__device__ __forceinline__ void mma_u8s8_zero(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+
 // Quantise the warp's 256 staged activations, every lane its own 8 values: lane l holds quarter
 // l % 4 of sub-block l / 4, i.e. exactly word l % 4 of that sub-block's byte registers
 // (q = [hi even, hi odd, lo even, lo odd]).  Maximum and sum over the sub-block come from shuffles.
@@ -263,7 +270,8 @@ struct Walk {
 
 }  // namespace gemv_detail
 
-// Launches the 5..8-token kernel on `grid` CTAs (defined in q4k_gemm_tokens.cu).
+// Launches the 5..16-token kernel on `grid` CTAs (defined in q4k_gemm_tokens.cu); CTAs of that kernel per SM.
+int gemv_tokens_ctas_per_sm(int n_tok);
 cudaError_t launch_gemv_tokens(const gemv_detail::GemvParams& P, int64_t grid, cudaStream_t st);
 
 }  // namespace prima

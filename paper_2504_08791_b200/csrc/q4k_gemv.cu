@@ -288,6 +288,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     if (++rslot == kRing) rslot = 0;
   };
 
+  const int my_piece = kUnitHdrBytes + unit_piece_slot(g, t) * 16;      // this lane's nibble piece inside a unit
   // lane-constant byte selectors that pull this lane's 24-bit field group out of header words 1..3
   const uint32_t sel_a = t == 1 ? 0x7654u : (t == 3 ? 0x0073u : 0x3210u);
   const uint32_t sel_b = t == 2 ? 0x7654u : (t == 3 ? 0x0710u : 0x3210u);
@@ -364,10 +365,10 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
       const uint8_t* u1 = u0 + kUnitBytes;
       const LaneScales s0 = decode_header(*reinterpret_cast<const uint4*>(u0 + g * 16), sel_a, sel_b);
       const LaneScales s1 = decode_header(*reinterpret_cast<const uint4*>(u1 + g * 16), sel_a, sel_b);
-      const uint4 qa0 = *reinterpret_cast<const uint4*>(u0 + kUnitHdrBytes + lane * 16);
-      const uint4 qa1 = *reinterpret_cast<const uint4*>(u1 + kUnitHdrBytes + lane * 16);
-      const uint4 qb0 = *reinterpret_cast<const uint4*>(u0 + kUnitHdrBytes + 512 + lane * 16);
-      const uint4 qb1 = *reinterpret_cast<const uint4*>(u1 + kUnitHdrBytes + 512 + lane * 16);
+      const uint4 qa0 = *reinterpret_cast<const uint4*>(u0 + my_piece);
+      const uint4 qa1 = *reinterpret_cast<const uint4*>(u1 + my_piece);
+      const uint4 qb0 = *reinterpret_cast<const uint4*>(u0 + my_piece + 512);
+      const uint4 qb1 = *reinterpret_cast<const uint4*>(u1 + my_piece + 512);
 #pragma unroll
       for (int k = 0; k < NTOK; ++k) {
         int ia0, ia1, ib0, ib1;
@@ -485,9 +486,9 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
   if ((in.out_order == kOrderResidual && w.mpad() % 256 != 0) || (in.out_order == kOrderSwiglu && w.mpad() % 512 != 0)) return cuda_rc(cudaErrorInvalidValue);
   int launches = 0;
   if (n_tok > 4 && gemv_uses_tensor_cores()) {
-    // 5..8 tokens: one pass over the weights with the tokens as columns of the tensor-core product (up to 4
+    // 5..16 tokens: one pass over the weights with the tokens as columns of the tensor-core product (up to 4
     // tokens the one-token formulation with one instruction per token is faster, measured)
-    int64_t grid = static_cast<int64_t>(sm_count) * std::max(1, 2 * kMaxWarps / sg);
+    int64_t grid = static_cast<int64_t>(sm_count) * std::max(1, gemv_tokens_ctas_per_sm(n_tok) * kMaxWarps / sg);
     if (grid > n_pos) grid = n_pos;
     P.tok0 = 0;
     const cudaError_t e = launch_gemv_tokens(P, grid, st);
@@ -496,9 +497,10 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
   }
   int tok = 0;
   while (tok < n_tok) {
-    // up to 4 tokens per pass; 5..8 tokens are split as evenly as possible over two passes
+    // up to 4 tokens per pass; more tokens are split as evenly as possible over the fewest passes
     const int left = n_tok - tok;
-    const int chunk = left <= 4 ? left : (left + 1) / 2;
+    const int passes = (left + 3) / 4;
+    const int chunk = (left + passes - 1) / passes;
     const int warps_per_sm = chunk == 1 ? 16 : 8;
     int64_t grid = static_cast<int64_t>(sm_count) * std::max(1, warps_per_sm / sg);
     if (grid > n_pos) grid = n_pos;

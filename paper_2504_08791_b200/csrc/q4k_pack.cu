@@ -102,7 +102,7 @@ __global__ void retile_kernel(const uint8_t* __restrict__ src, int64_t rows_src,
       words[w] = word;
     }
     const int half_idx = j >> 2, t = j & 3;
-    uint8_t* chunk = unit + kUnitHdrBytes + half_idx * 512 + (g * 4 + t) * 16;
+    uint8_t* chunk = unit + kUnitHdrBytes + half_idx * 512 + unit_piece_slot(g, t) * 16;
     *reinterpret_cast<uint4*>(chunk) = make_uint4(words[0], words[1], words[2], words[3]);
   }
 }

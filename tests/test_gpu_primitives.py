@@ -80,6 +80,7 @@ def _check_rows(got, want, s_abs, tol=ROW_TOL):
 @pytest.mark.parametrize("rows,cols,n_cols", [
     (4096, 4096, 1),      # the single-GEMV workload
     (8, 256, 1), (1, 256, 1), (13, 768, 1), (100, 512, 3), (4096, 4096, 2), (1000, 1024, 5), (264, 1280, 8),
+    (1000, 2048, 9), (264, 1280, 13), (520, 4096, 16), (9, 256, 16),      # two column blocks of eight
 ])
 def test_gemv_literal_distribution(gpu, rows, cols, n_cols):
     w, x = synth.gemv_case(seed=0, rows=rows, cols=cols, n_cols=n_cols)
@@ -119,9 +120,10 @@ def test_gemv_activation_scales_and_special_vectors(gpu):
     _check_rows(_gemv_gpu(gpu, w, rows, cols, x), want, s_abs)
 
 
-def test_gemv_several_tokens_with_outliers_and_mixed_scales(gpu):
-    # 5..8 columns go through the kernel that quantises a column's 256 activations with one step
-    rows, cols, n = 264, 2048, 6
+@pytest.mark.parametrize("n", [6, 11])
+def test_gemv_several_tokens_with_outliers_and_mixed_scales(gpu, n):
+    # 5..16 columns go through the kernel that quantises a column's 256 activations with one step
+    rows, cols = 264, 2048
     w = synth.model_tensor(8, 0, synth.WQ, rows, cols)
     x = synth.activations(8, n, cols)
     x[1] *= 1e-4
@@ -129,6 +131,7 @@ def test_gemv_several_tokens_with_outliers_and_mixed_scales(gpu):
     x[3, 5] = 700.0          # one large value in a block of small ones
     x[4, 256:512] = 0.0      # an all-zero block
     x[5] = np.abs(x[5])
+    x[n - 1] = -np.abs(x[n - 1]) * 40.0      # sub-block sums near the top of their 20-bit range
     want, s_abs = oracle.gemv_q4k(w, rows, cols, x)
     got = _gemv_gpu(gpu, w, rows, cols, x)
     _check_rows(got, want, s_abs)
@@ -165,4 +168,4 @@ def test_gemv_rejects_bad_arguments(gpu):
     with pytest.raises(binding.PrimaError):
         binding.prima_gemv_q4k(w, 1, 200, x, 1, y)
     with pytest.raises(binding.PrimaError):
-        binding.prima_gemv_q4k(w, 1, 256, x, 9, y)
+        binding.prima_gemv_q4k(w, 1, 256, x, 17, y)

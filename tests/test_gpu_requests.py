@@ -29,10 +29,13 @@ def _rel(got, want):
 @pytest.mark.parametrize("name,seqs,lengths", [
     ("tiny", [0, 1, 2], [5, 0, 33]),
     ("small", [3, 0, 7, 1, 2, 9], [130, 17, 255, 1, 64, 128]),      # 6 requests: the multi-token product kernel
+    ("small", [3, 0, 7, 1, 2, 9, 11, 5, 4], [130, 17, 255, 1, 64, 128, 0, 300, 77]),      # 9: two column blocks, the second nearly empty
+    ("small", list(range(12)), [13 * i + 1 for i in range(12)]),
+    ("small", list(range(15, -1, -1)), [19 * i for i in range(16)]),                    # 16 requests: both column blocks full
 ])
 def test_requests_step_matches_checker_per_request(gpu, name, seqs, lengths):
     torch, binding = gpu
-    cfg = synth.model_config(name)
+    cfg = synth.model_config(name, max_n_tok=16)
     L, n = cfg["n_layers"], len(seqs)
     ctx = binding.Context(cfg)
     refs = [oracle.Model(cfg) for _ in seqs]                       # the checker has one cache per model: one model per request
