@@ -139,13 +139,18 @@ def job_value(ms_per_step_max: float, world: int) -> dict:
 
 
 # ------------------------------------------------------------------------------------ the GPU arm
-def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None, n_requests=1, on_layer=None, on_globals=None):
+def build_gpu_model(binding, cfg, seed, n_ctx, device, n_layers=None, n_requests=1, on_layer=None, on_globals=None,
+                    resident_layers=None, stream_slots=None):
     """Generate the synthetic model layer by layer and make it resident.  on_layer(l, tensors, k, v) and
     on_globals(tensors) see the same host arrays (the CPU-baseline leg runs the checker on them, so the 39 GB of
     a 70B-shaped model are generated once and never held in host memory all at once)."""
     import torch
     t0 = time.time()
     ctx = binding.Context(cfg, device=device)
+    if resident_layers is not None:
+        ctx.set_option(binding.OPT_RESIDENT_LAYERS, resident_layers)
+        if stream_slots:
+            ctx.set_option(binding.OPT_STREAM_SLOTS, stream_slots)
     layers = range(cfg["n_layers"]) if n_layers is None else range(n_layers)
     for l in layers:
         tensors = {}
@@ -239,8 +244,10 @@ def run_ours(args, rank, world, local_rank):
     whole = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and R == 1 and not args.layers:
         whole = WholeTokenOracle(cfg, seed, n_ctx, args.n_tok)
+    resident = args.resident_layers if args.resident_layers >= 0 else None
     ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank, n_requests=R,
-                          on_layer=whole.on_layer if whole else None, on_globals=whole.on_globals if whole else None)
+                          on_layer=whole.on_layer if whole else None, on_globals=whole.on_globals if whole else None,
+                          resident_layers=resident, stream_slots=args.stream_slots)
     bpt = bytes_per_token(cfg, n_ctx)
     if R > 1:                                     # the weights are read once per step, every request's cache once
         bpt = dict(bpt, total=bpt["total"] + (R - 1) * L_kv_bytes(cfg, n_ctx))
@@ -399,6 +406,8 @@ def run_ours(args, rank, world, local_rank):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if resident is not None:
+        result["streaming"] = streaming_report(torch, ctx, cfg, resident, args, ms_step)
     if args.speculative and world == 1:
         result["speculative"] = speculative_cycle(args, binding, ctx, cfg, seed, n_ctx, bounds)
     ctx.close()
@@ -408,6 +417,33 @@ def run_ours(args, rank, world, local_rank):
         dist.barrier()
         dist.destroy_process_group()
     return result
+
+
+def streaming_report(torch, ctx, cfg, resident, args, ms_step) -> dict:
+    """Layers streamed from pinned host memory: what a token has to bring over the host link, the link's rate for a
+    plain pinned copy measured here, and the rate the decoding loop achieved."""
+    n_streamed = cfg["n_layers"] - resident
+    layer_bytes = synth.weight_bytes(cfg, (synth.WQ, synth.WK, synth.WV, synth.WO, synth.W_GATE, synth.W_UP, synth.W_DOWN))
+    per_token = n_streamed * layer_bytes if n_streamed > max(1, args.stream_slots or 2) - 0 else 0
+    src = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    dst.copy_(src, non_blocking=True)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        dst.copy_(src, non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    link_gbs = 3 * (1 << 30) / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    copied, copy_ms = ctx.stream_stats()
+    achieved = per_token / (ms_step * 1e-3) / 1e9
+    return {"resident_layers": resident, "streamed_layers": n_streamed, "slots": args.stream_slots or 2,
+            "streamed_bytes_per_token": per_token, "host_link_GBs_plain_pinned_copy": link_gbs,
+            "achieved_GBs_over_the_step": achieved, "frac_of_host_link": achieved / link_gbs if link_gbs else None,
+            "floor_ms_per_token_at_host_link": per_token / (link_gbs * 1e9) * 1e3 if link_gbs else None,
+            "copies_GBs_while_copying": copied / (copy_ms * 1e-3) / 1e9 if copy_ms else None,
+            "note": "bound: the host link, not HBM; step_roofline above is against HBM and does not apply to this run"}
 
 
 def speculative_cycle(args, binding, target, cfg, seed, n_ctx, bounds) -> dict:
@@ -516,6 +552,9 @@ def main():
     ap.add_argument("--speculative", default="", choices=["", "8b", "32b"],
                     help="also time speculative decoding cycles with a draft model of this shape")
     ap.add_argument("--repeats", type=int, default=5, help="how many times the timed region of --steps steps is taken (median reported)")
+    ap.add_argument("--resident-layers", type=int, default=-1,
+                    help="keep only the first N layers' matrices on the GPU, stream the others from pinned host memory every token")
+    ap.add_argument("--stream-slots", type=int, default=0, help="device buffers for streamed layers (default 2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

@@ -188,7 +188,27 @@ int prima_sync(prima_ctx* ctx);
  * rejected it (nothing is sent to the GPU for it), once; -1 switches the injection off. */
 #define PRIMA_OPT_FIRST_WAIT_POLLS 1
 #define PRIMA_OPT_FAIL_AFTER_LAUNCHES 2
+
+/* A model larger than the device's memory (the paper's case: Section 3.1, "Pipelined-ring parallelism (PRP) with
+ * prefetching"; Appendix A.1-A.2: the weights of the windows that do not fit are (re)loaded while other work
+ * runs, so that loading overlaps with computing).  Here the slow tier is pinned host memory instead of a disk:
+ *   PRIMA_OPT_RESIDENT_LAYERS  the first `value` layers keep their matrices on the device; the matrices of the
+ *       layers from `value` on live in pinned host memory (in the library's tiled layout) and are streamed to the
+ *       device every time they are needed; -1 or n_layers: everything resident (default).
+ *   PRIMA_OPT_STREAM_SLOTS     number of device buffers, each holding one streamed layer (2..16, default 2).
+ * Both must be set before the first layer matrix is loaded.  The matrices of a streamed layer must be loaded
+ * layer by layer (all seven of one layer before those of the next streamed layer; PRIMA_ERR_STATE otherwise).
+ * prima_forward_window then waits, on the context's stream, only for the copy of the layer it is about to run
+ * (one cudaMemcpyAsync per matrix on a second stream, ordered by events), and queues the copies of the streamed
+ * layers that come next in decoding order (cyclically: after the last layer comes the first streamed layer of
+ * the next token), as many as there are other slots, so that they stream in underneath the computation.  KV
+ * caches, norm gains and the input / output layers stay on the device.  Results are bit-identical to those of a
+ * fully resident context.  prima_stream_stats: bytes copied host-to-device for streamed layers since the context
+ * was created, and the summed duration of those copies in milliseconds (waits for the copy stream). */
+#define PRIMA_OPT_RESIDENT_LAYERS 3
+#define PRIMA_OPT_STREAM_SLOTS 4
 int prima_ctx_set_option(prima_ctx* ctx, int option, int64_t value);
+int prima_stream_stats(prima_ctx* ctx, int64_t* bytes_copied, double* copy_ms);
 
 /* Text of the most recent error of this context (never NULL; "" if none).  With ctx == NULL,
  * the most recent error of a context-free call on this thread. */

@@ -22,13 +22,15 @@ PROF_GEMV, PROF_ATTENTION = 0, 1
 PROF_GEMV_QKV, PROF_GEMV_O, PROF_GEMV_GATE_UP, PROF_GEMV_DOWN, PROF_GEMV_HEAD = 16, 17, 18, 19, 20
 OPT_FIRST_WAIT_POLLS = 1
 OPT_FAIL_AFTER_LAUNCHES = 2
+OPT_RESIDENT_LAYERS = 3
+OPT_STREAM_SLOTS = 4
 
 EXPORTS = [
     "prima_ctx_create", "prima_ctx_destroy", "prima_load_q4k_weights", "prima_forward_window", "prima_logits",
     "prima_embed", "prima_argmax", "prima_kv_load", "prima_kv_read", "prima_sync", "prima_last_error",
     "prima_launch_count", "prima_profile_enable", "prima_profile_read", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
     "prima_gemv_plan_destroy", "prima_gemv_q4k_noalloc", "prima_gemv_q4k_noalloc_error",
-    "prima_forward_window_seqs", "prima_kv_load_seq", "prima_kv_read_seq", "prima_ctx_set_option",
+    "prima_forward_window_seqs", "prima_kv_load_seq", "prima_kv_read_seq", "prima_ctx_set_option", "prima_stream_stats",
 ]
 
 
@@ -70,6 +72,7 @@ def lib():
         L.prima_kv_read_seq.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.prima_sync.argtypes = [vp]
         L.prima_ctx_set_option.argtypes = [vp, i32, i64]
+        L.prima_stream_stats.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double)]
         L.prima_last_error.argtypes = [vp]
         L.prima_last_error.restype = C.c_char_p
         L.prima_launch_count.argtypes = [vp]
@@ -229,6 +232,12 @@ class Context:
 
     def set_option(self, option: int, value: int):
         _check(lib().prima_ctx_set_option(self._h, option, value), self._h)
+
+    def stream_stats(self):
+        """(bytes copied host-to-device for streamed layers, summed copy time in ms)."""
+        b, ms = C.c_int64(), C.c_double()
+        _check(lib().prima_stream_stats(self._h, C.byref(b), C.byref(ms)), self._h)
+        return b.value, ms.value
 
     def profile_enable(self, mode):
         """0 / False: off; 1 / True: events around every launch (isolated kernels); 2: in-situ stamps."""

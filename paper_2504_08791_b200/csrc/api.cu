@@ -36,9 +36,21 @@ struct Layer {
   __half* k = nullptr;        // cache of sequence 0 (the only one that prima_forward_window uses)
   __half* v = nullptr;
   std::vector<__half*> k_seq, v_seq;   // caches of sequences 1.. (index seq - 1), allocated on first use
+  uint8_t* host = nullptr;    // streamed layers: the four tiled matrices in pinned host memory (qkv | o | gate/up | down)
 };
 
+// A device buffer that holds the matrices of ONE streamed layer at a time.
+struct StreamSlot {
+  uint8_t* dev = nullptr;
+  int layer = -1;              // layer whose copy was queued into the slot (or -1)
+  bool waited = false;         // the compute stream already waits for that copy
+  bool used = false;           // a compute pass over the slot's content has been queued (compute_done is recorded)
+  cudaEvent_t copy_done = nullptr, compute_done = nullptr;
+};
+struct CopySpan { cudaEvent_t t0, t1; };      // around one layer's copy, for the statistics
+
 constexpr uint32_t kLayerMask = (1u << 9) - 1;
+constexpr uint32_t kMatrixMask = kLayerMask & ~((1u << PRIMA_ATTN_NORM) | (1u << PRIMA_FFN_NORM));
 
 }  // namespace
 
@@ -72,6 +84,18 @@ struct prima_ctx {
   int32_t* am_idx = nullptr;
   int32_t* am_out = nullptr;
   int* status = nullptr;
+
+  // ---- layers streamed from pinned host memory (PRIMA_OPT_RESIDENT_LAYERS) ----
+  int n_resident = -1;                 // -1: every layer lives on the device
+  int n_slots = 2;
+  std::vector<StreamSlot> slots;
+  cudaStream_t copy_stream = nullptr;
+  size_t off_o = 0, off_gu = 0, off_down = 0, layer_bytes = 0;
+  int loading_layer = -1;              // streamed layer being assembled in slot 0
+  int64_t streamed_bytes = 0;
+  double copy_ms = 0;
+  std::vector<void*> pinned;
+  std::vector<CopySpan> spans_pending, spans_free;
 
   std::vector<void*> allocs;
   std::string err;
@@ -148,6 +172,162 @@ int ensure_tiled(prima_ctx* c, TiledMat* t, int64_t rows, int64_t cols) {
   int rc = dev_alloc(c, &s.data, s.bytes(), true);
   if (rc != PRIMA_OK) return rc;
   *t = s;
+  return PRIMA_OK;
+}
+
+bool is_streamed(const prima_ctx* c, int layer) { return c->n_resident >= 0 && layer >= c->n_resident; }
+
+// Shapes and offsets of a layer's four matrices inside a slot / a pinned host copy.
+void stream_layout(prima_ctx* c, TiledMat* qkv, TiledMat* o, TiledMat* gu, TiledMat* down) {
+  const prima_model_config& g = c->cfg;
+  *qkv = shape_tiled(static_cast<int64_t>(g.n_q_heads + 2 * g.n_kv_heads) * kHeadDim, g.hidden);
+  *o = shape_tiled(g.hidden, static_cast<int64_t>(g.n_q_heads) * kHeadDim);
+  *gu = shape_tiled(2 * static_cast<int64_t>(g.ffn), g.hidden);
+  *down = shape_tiled(g.hidden, g.ffn);
+  c->off_o = qkv->bytes();
+  c->off_gu = c->off_o + o->bytes();
+  c->off_down = c->off_gu + gu->bytes();
+  c->layer_bytes = c->off_down + down->bytes();
+}
+
+void point_layer_at(prima_ctx* c, Layer& L, uint8_t* base) {
+  TiledMat qkv, o, gu, down;
+  stream_layout(c, &qkv, &o, &gu, &down);
+  qkv.data = base;
+  o.data = base ? base + c->off_o : nullptr;
+  gu.data = base ? base + c->off_gu : nullptr;
+  down.data = base ? base + c->off_down : nullptr;
+  L.qkv = qkv; L.o = o; L.gu = gu; L.down = down;
+}
+
+// Slots and the copy stream, created when the first streamed layer is loaded.
+int ensure_slots(prima_ctx* c) {
+  if (!c->slots.empty()) return PRIMA_OK;
+  TiledMat a, b, d, e2;
+  stream_layout(c, &a, &b, &d, &e2);
+  cudaError_t e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaStreamCreate(copy stream)");
+  c->slots.resize(c->n_slots);
+  for (auto& sl : c->slots) {
+    int rc = dev_alloc(c, &sl.dev, c->layer_bytes);
+    if (rc != PRIMA_OK) return rc;
+    e = cudaEventCreateWithFlags(&sl.copy_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.compute_done, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaEventCreate(slot)");
+  }
+  return PRIMA_OK;
+}
+
+// Add the times of the copies that have completed to the statistics; never waits unless asked to.
+void harvest_copy_times(prima_ctx* c, bool wait) {
+  size_t kept = 0;
+  for (size_t i = 0; i < c->spans_pending.size(); ++i) {
+    CopySpan sp = c->spans_pending[i];
+    cudaError_t q = wait ? cudaEventSynchronize(sp.t1) : cudaEventQuery(sp.t1);
+    if (q == cudaSuccess) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, sp.t0, sp.t1) == cudaSuccess) c->copy_ms += ms;
+      c->spans_free.push_back(sp);
+    } else {
+      c->spans_pending[kept++] = sp;
+    }
+  }
+  c->spans_pending.resize(kept);
+}
+
+// Queue, on the copy stream, the copy of streamed layer `l` into slot `s`: after the compute pass that last used
+// the slot, one cudaMemcpyAsync per matrix, then the slot's copy_done event.
+int queue_layer_copy(prima_ctx* c, int l, int s) {
+  StreamSlot& sl = c->slots[s];
+  Layer& L = c->layers[l];
+  harvest_copy_times(c, false);
+  CopySpan sp{nullptr, nullptr};
+  cudaError_t e = cudaSuccess;
+  if (!c->spans_free.empty()) {
+    sp = c->spans_free.back();
+    c->spans_free.pop_back();
+  } else {
+    e = cudaEventCreate(&sp.t0);
+    if (e == cudaSuccess) e = cudaEventCreate(&sp.t1);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaEventCreate(copy span)");
+  }
+  if (sl.used) e = cudaStreamWaitEvent(c->copy_stream, sl.compute_done, 0);
+  if (e == cudaSuccess) e = cudaEventRecord(sp.t0, c->copy_stream);
+  const size_t off[5] = {0, c->off_o, c->off_gu, c->off_down, c->layer_bytes};
+  for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+    e = cudaMemcpyAsync(sl.dev + off[i], L.host + off[i], off[i + 1] - off[i], cudaMemcpyHostToDevice, c->copy_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(sp.t1, c->copy_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(sl.copy_done, c->copy_stream);
+  c->spans_pending.push_back(sp);
+  if (e != cudaSuccess) return cuda_fail(c, e, "queueing the copy of a streamed layer");
+  sl.layer = l;
+  sl.waited = false;
+  sl.used = false;
+  c->streamed_bytes += static_cast<int64_t>(c->layer_bytes);
+  return PRIMA_OK;
+}
+
+int slot_of_layer(const prima_ctx* c, int l) {
+  for (size_t s = 0; s < c->slots.size(); ++s)
+    if (c->slots[s].layer == l) return static_cast<int>(s);
+  return -1;
+}
+
+// The streamed layer that follows l in the order in which a decoding loop visits them (cyclic).
+int next_streamed(const prima_ctx* c, int l) { return l + 1 < c->cfg.n_layers ? l + 1 : c->n_resident; }
+
+// Make streamed layer l's matrices available to the compute stream; returns the slot in *slot.
+int acquire_layer(prima_ctx* c, int l, int* slot) {
+  int s = slot_of_layer(c, l);
+  if (s < 0) {
+    // not queued yet (first use, or layers visited out of order): take the slot whose layer comes last in the cyclic
+    // order that starts at l
+    int best = 0, best_d = -1;
+    const int n_str = c->cfg.n_layers - c->n_resident;
+    for (size_t i = 0; i < c->slots.size(); ++i) {
+      const int other = c->slots[i].layer;
+      const int d = other < 0 ? 1 << 30 : ((other - l) % n_str + n_str) % n_str;
+      if (d > best_d) { best_d = d; best = static_cast<int>(i); }
+    }
+    s = best;
+    const int rc = queue_layer_copy(c, l, s);
+    if (rc != PRIMA_OK) return rc;
+  }
+  StreamSlot& sl = c->slots[s];
+  if (!sl.waited) {
+    const cudaError_t e = cudaStreamWaitEvent(c->stream, sl.copy_done, 0);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaStreamWaitEvent(copy done)");
+    sl.waited = true;
+  }
+  point_layer_at(c, c->layers[l], sl.dev);
+  *slot = s;
+  return PRIMA_OK;
+}
+
+// After layer l's kernels were queued: mark its slot and queue the copies of the streamed layers that follow
+// it, as many as there are other slots, so that they stream in while l and its successors compute.
+int release_and_prefetch(prima_ctx* c, int l, int slot) {
+  StreamSlot& sl = c->slots[slot];
+  cudaError_t e = cudaEventRecord(sl.compute_done, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaEventRecord(compute done)");
+  sl.used = true;
+  const int n_str = c->cfg.n_layers - c->n_resident;
+  int nxt = l;
+  for (int k = 1; k < static_cast<int>(c->slots.size()) && k < n_str; ++k) {
+    nxt = next_streamed(c, nxt);
+    if (slot_of_layer(c, nxt) >= 0) continue;
+    // victim: not the slot that layer l is being computed from (a copy into it would have to wait for that
+    // computation, and nothing would overlap); of the others, the one whose layer is needed last
+    int best = -1, best_d = -1;
+    for (size_t i = 0; i < c->slots.size(); ++i) {
+      if (static_cast<int>(i) == slot) continue;
+      const int other = c->slots[i].layer;
+      const int d = other < 0 ? 1 << 30 : ((other - l - 1) % n_str + n_str) % n_str;
+      if (d > best_d) { best_d = d; best = static_cast<int>(i); }
+    }
+    const int rc = queue_layer_copy(c, nxt, best);
+    if (rc != PRIMA_OK) return rc;
+  }
   return PRIMA_OK;
 }
 
@@ -361,6 +541,20 @@ int prima_ctx_destroy(prima_ctx* c) {
     cudaEventDestroy(sp.a);
     cudaEventDestroy(sp.b);
   }
+  if (c->copy_stream) {
+    cudaStreamSynchronize(c->copy_stream);
+    cudaStreamDestroy(c->copy_stream);
+  }
+  for (auto& sl : c->slots) {
+    if (sl.copy_done) cudaEventDestroy(sl.copy_done);
+    if (sl.compute_done) cudaEventDestroy(sl.compute_done);
+  }
+  for (auto* v : {&c->spans_pending, &c->spans_free})
+    for (auto& sp : *v) {
+      cudaEventDestroy(sp.t0);
+      cudaEventDestroy(sp.t1);
+    }
+  for (void* p : c->pinned) cudaFreeHost(p);
   for (void* p : c->allocs) cudaFree(p);
   delete c;
   return PRIMA_OK;
@@ -416,6 +610,27 @@ int prima_load_q4k_weights(prima_ctx* c, int layer, int tensor_id, const void* d
   Layer& L = c->layers[layer];
   rc = ensure_kv(c, layer);
   if (rc != PRIMA_OK) return rc;
+  const bool matrix = tensor_id != PRIMA_ATTN_NORM && tensor_id != PRIMA_FFN_NORM;
+  if (is_streamed(c, layer) && matrix) {
+    // A streamed layer is assembled in slot 0 and moved to pinned host memory when its seventh matrix has arrived.
+    rc = ensure_slots(c);
+    if (rc != PRIMA_OK) return rc;
+    if (c->loading_layer != layer) {
+      if (c->loading_layer >= 0)
+        return fail(c, PRIMA_ERR_STATE, "the matrices of a streamed layer must be loaded layer by layer: layer " +
+                                            std::to_string(c->loading_layer) + " is not complete yet");
+      cudaError_t e = cudaStreamSynchronize(c->stream);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(c->copy_stream);
+      if (e == cudaSuccess) e = cudaMemsetAsync(c->slots[0].dev, 0, c->layer_bytes, c->stream);
+      if (e != cudaSuccess) return cuda_fail(c, e, "preparing the assembly slot");
+      harvest_copy_times(c, true);
+      c->slots[0].layer = -1;
+      c->slots[0].used = false;
+      c->loading_layer = layer;
+      L.have &= ~kMatrixMask;
+    }
+    point_layer_at(c, L, c->slots[0].dev);
+  }
   switch (tensor_id) {
     case PRIMA_ATTN_NORM: rc = load_norm(c, &L.g_attn, &L.gmax_attn, data, cols); break;
     case PRIMA_FFN_NORM: rc = load_norm(c, &L.g_ffn, &L.gmax_ffn, data, cols); break;
@@ -439,6 +654,20 @@ int prima_load_q4k_weights(prima_ctx* c, int layer, int tensor_id, const void* d
       break;
   }
   if (rc == PRIMA_OK) L.have |= 1u << tensor_id;
+  if (rc == PRIMA_OK && is_streamed(c, layer) && matrix && (L.have & kMatrixMask) == kMatrixMask) {
+    if (!L.host) {
+      void* hp = nullptr;
+      cudaError_t e = cudaHostAlloc(&hp, c->layer_bytes, cudaHostAllocDefault);
+      if (e != cudaSuccess) return cuda_fail(c, e, "cudaHostAlloc(streamed layer)");
+      c->pinned.push_back(hp);
+      L.host = static_cast<uint8_t*>(hp);
+    }
+    cudaError_t e = cudaMemcpyAsync(L.host, c->slots[0].dev, c->layer_bytes, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "moving a streamed layer to pinned host memory");
+    c->loading_layer = -1;
+    point_layer_at(c, L, nullptr);
+  }
   return rc;
 }
 
@@ -504,6 +733,11 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
   c->unsynced_min_pos = stable_below;      // this call appends at first_pos and above
   for (int l = layer_begin; l < layer_end; ++l) {
     Layer& L = c->layers[l];
+    int slot = -1;
+    if (is_streamed(c, l)) {
+      const int rc = acquire_layer(c, l, &slot);
+      if (rc != PRIMA_OK) return rc;
+    }
     GemvIn in;                                   // QKV: residual (+ down projection of layer l-1) -> h_b
     in.kind = kResidual; in.h_in = h_in; in.h_out = c->h_b; in.acc_in = acc_prev; in.mpad_in = mpad_e;
     in.gain = L.g_attn; in.ssq_out = c->ssq_attn; in.status = c->status; in.first_wait_polls = c->first_wait_polls;
@@ -554,6 +788,10 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.down), launch_gemv_partials(L.down, in_d, n_tok, c->acc_down, c->sm_count, st), "gemv(down)");
     h_in = c->h_a;
     acc_prev = c->acc_down;
+    if (slot >= 0) {
+      const int rc = release_and_prefetch(c, l, slot);
+      if (rc != PRIMA_OK) return rc;
+    }
   }
   LAUNCH(c, launch_finish_residual(c->acc_down, mpad_e, e_, n_tok, c->h_a, hidden_out, c->acc_gu,
                                    static_cast<int64_t>(n_tok) * c->layers[layer_end - 1].gu.mpad(), st), "finish_residual");
@@ -566,7 +804,8 @@ static int window_args_ok(prima_ctx* c, const char* who, int layer_begin, int la
   if (layer_begin < 0 || layer_end > g.n_layers || layer_begin > layer_end) return fail(c, PRIMA_ERR_ARG, "bad layer range");
   if (n_tok < 1 || n_tok > g.max_n_tok) return fail(c, PRIMA_ERR_ARG, "n_tok outside 1..max_n_tok");
   for (int l = layer_begin; l < layer_end; ++l)
-    if ((c->layers[l].have & kLayerMask) != kLayerMask) return fail(c, PRIMA_ERR_STATE, "a layer of the window is not fully loaded");
+    if ((c->layers[l].have & kLayerMask) != kLayerMask || l == c->loading_layer)
+      return fail(c, PRIMA_ERR_STATE, "a layer of the window is not fully loaded");
   return PRIMA_OK;
 }
 
@@ -737,6 +976,20 @@ int prima_ctx_set_option(prima_ctx* c, int option, int64_t value) {
       if (value < -1 || value > (int64_t(1) << 30)) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_FIRST_WAIT_POLLS: value outside -1 .. 2^30");
       c->first_wait_polls = value < 0 ? 0u : static_cast<uint32_t>(value) + 1u;
       return PRIMA_OK;
+    case PRIMA_OPT_RESIDENT_LAYERS:
+    case PRIMA_OPT_STREAM_SLOTS: {
+      for (const Layer& L : c->layers)
+        if (L.have & kMatrixMask) return fail(c, PRIMA_ERR_STATE, "residency options must be set before any layer matrix is loaded");
+      if (option == PRIMA_OPT_RESIDENT_LAYERS) {
+        if (value < -1 || value > c->cfg.n_layers) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_RESIDENT_LAYERS: value outside -1 .. n_layers");
+        c->n_resident = value == c->cfg.n_layers ? -1 : static_cast<int>(value);
+      } else {
+        if (value < 2 || value > 16) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_STREAM_SLOTS: value outside 2 .. 16");
+        if (!c->slots.empty()) return fail(c, PRIMA_ERR_STATE, "the slots exist already");
+        c->n_slots = static_cast<int>(value);
+      }
+      return PRIMA_OK;
+    }
     case PRIMA_OPT_FAIL_AFTER_LAUNCHES:
       if (value < -1) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_FAIL_AFTER_LAUNCHES: value below -1");
       c->fail_after = value;
@@ -744,6 +997,19 @@ int prima_ctx_set_option(prima_ctx* c, int option, int64_t value) {
     default:
       return fail(c, PRIMA_ERR_ARG, "prima_ctx_set_option: unknown option");
   }
+}
+
+int prima_stream_stats(prima_ctx* c, int64_t* bytes_copied, double* copy_ms) {
+  if (!c || !bytes_copied || !copy_ms) return fail(c, PRIMA_ERR_ARG, "prima_stream_stats: null argument");
+  DeviceGuard guard(c->cfg.device);
+  if (c->copy_stream) {
+    cudaError_t e = cudaStreamSynchronize(c->copy_stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "prima_stream_stats");
+    harvest_copy_times(c, true);
+  }
+  *bytes_copied = c->streamed_bytes;
+  *copy_ms = c->copy_ms;
+  return PRIMA_OK;
 }
 
 int prima_profile_enable(prima_ctx* c, int mode) {
