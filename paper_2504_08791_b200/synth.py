@@ -83,6 +83,60 @@ def build_blocks(d_bits, dmin_bits, sc, m, q) -> np.ndarray:
 
 
 # ---------------------------------------------------------------------------------------------
+# the other block formats: Q8_0 (34 bytes per 32 weights), Q6_K (210 bytes per 256 weights), FP16
+# ---------------------------------------------------------------------------------------------
+FMT_Q4_K, FMT_Q6_K, FMT_Q8_0, FMT_F16 = 0, 1, 2, 3
+FMT_BLOCK_WEIGHTS = {FMT_Q4_K: 256, FMT_Q6_K: 256, FMT_Q8_0: 32, FMT_F16: 1}
+FMT_BLOCK_BYTES = {FMT_Q4_K: 144, FMT_Q6_K: 210, FMT_Q8_0: 34, FMT_F16: 2}
+
+
+def build_q8_0_blocks(d_bits, q) -> np.ndarray:
+    """[n] binary16 bit patterns and [n, 32] signed values -128..127 -> [n, 34] bytes."""
+    d_bits = np.asarray(d_bits, dtype=np.uint16).reshape(-1)
+    n = d_bits.size
+    out = np.empty((n, 34), np.uint8)
+    out[:, 0:2] = d_bits.view(np.uint8).reshape(n, 2)
+    out[:, 2:] = np.asarray(q).reshape(n, 32).astype(np.int8).view(np.uint8)
+    return out
+
+
+def build_q6k_blocks(d_bits, scales, v) -> np.ndarray:
+    """[n] binary16 bit patterns, [n, 16] signed scales and [n, 256] six-bit values 0..63 -> [n, 210] bytes.
+    Weight k = 128 h + 32 i + l keeps its low nibble in byte 64 h + 32 (i & 1) + l of the first 128 bytes (low half
+    of the byte for i < 2, high half otherwise) and its two high bits in bits 2i, 2i+1 of byte 128 + 32 h + l."""
+    d_bits = np.asarray(d_bits, dtype=np.uint16).reshape(-1)
+    n = d_bits.size
+    v = np.asarray(v).reshape(n, 2, 4, 32).astype(np.uint8)
+    out = np.zeros((n, 210), np.uint8)
+    lo, hi = v & 15, v >> 4
+    for h in range(2):
+        for i in range(4):
+            seg = out[:, 64 * h + 32 * (i & 1):64 * h + 32 * (i & 1) + 32]
+            seg |= lo[:, h, i] << (0 if i < 2 else 4)
+            out[:, 128 + 32 * h:128 + 32 * h + 32] |= hi[:, h, i] << (2 * i)
+    out[:, 192:208] = np.asarray(scales).reshape(n, 16).astype(np.int8).view(np.uint8)
+    out[:, 208:210] = d_bits.view(np.uint8).reshape(n, 2)
+    return out
+
+
+def fmt_tensor(seed: int, fmt: int, rows: int, cols: int, gain: float = 1.0) -> np.ndarray:
+    """Random-init matrix in one of the other formats, roughly unit gain per row (weights ~ N(0, gain^2 / cols))."""
+    rng = _rng(seed, 606, fmt, rows, cols)
+    sigma = gain / np.sqrt(cols)
+    if fmt == FMT_F16:
+        return rng.normal(0.0, sigma, (rows, cols)).astype(np.float16).view(np.uint8).reshape(-1)
+    n = rows * cols // FMT_BLOCK_WEIGHTS[fmt]
+    blocks = _random_bytes(rng, n * FMT_BLOCK_BYTES[fmt]).reshape(n, FMT_BLOCK_BYTES[fmt]).copy()
+    if fmt == FMT_Q8_0:
+        d = (sigma * (0.5 + rng.random(n)) / 73.9).astype(np.float16)          # uniform signed bytes have sigma 73.9
+        blocks[:, 0:2] = d.view(np.uint8).reshape(n, 2)
+    else:
+        d = (sigma * (0.5 + rng.random(n)) / (18.5 * 73.9)).astype(np.float16)   # uniform 6-bit values: sigma 18.5
+        blocks[:, 208:210] = d.view(np.uint8).reshape(n, 2)
+    return blocks.reshape(-1)
+
+
+# ---------------------------------------------------------------------------------------------
 # the literal single-GEMV distribution
 # ---------------------------------------------------------------------------------------------
 def gemv_weights(seed: int, rows: int, cols: int) -> np.ndarray:

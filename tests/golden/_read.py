@@ -57,3 +57,34 @@ def prp_schedules():
         else:
             out[cur][key] = nums if key == "window_sizes" else nums[0]
     return out
+
+
+def kquants_blocks():
+    """Parse kquants_handbuilt.txt -> {name: dict(fmt='q8_0'|'q6_k', bytes=uint8[...], w={index: value})}."""
+    rules = {
+        "(n-16)&255": lambda n: (n - 16) & 255, "128": lambda n: np.full_like(n, 128), "0": lambda n: np.zeros_like(n),
+        "(n%16) | ((n//4)%16)<<4": lambda n: (n % 16) | (((n // 4) % 16) << 4), "(7*n+3)%256": lambda n: (7 * n + 3) % 256,
+        "(n-8)&255": lambda n: (n - 8) & 255,
+    }
+    out, cur = {}, None
+    for line in open(os.path.join(HERE, "kquants_handbuilt.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("["):
+            cur = line.strip("[]")
+            out[cur] = {}
+            continue
+        key, val = line.split(":", 1)
+        out[cur][key.strip()] = val.strip()
+    blocks = {}
+    for name, f in out.items():
+        fmt = name.split(".")[0]
+        d = np.array([int(t, 16) for t in f["d_hex"].split()], np.uint8)
+        if fmt == "q8_0":
+            raw = np.concatenate([d, rules[f["payload_rule"]](np.arange(32)).astype(np.uint8)])
+        else:
+            raw = np.concatenate([rules[f["ql_rule"]](np.arange(128)).astype(np.uint8), rules[f["qh_rule"]](np.arange(64)).astype(np.uint8),
+                                  rules[f["sc_rule"]](np.arange(16)).astype(np.uint8), d])
+        blocks[name] = dict(fmt=fmt, bytes=raw, w={int(t.split(":")[0]): float(t.split(":")[1]) for t in f["w"].split()})
+    return blocks
