@@ -538,6 +538,40 @@ def run_reference(args):
     }
 
 
+def run_gemv_fmt(args):
+    """Micro-benchmark of the single product in one of the other formats (not the headline): 70B-shaped matrices in
+    standard layout, a ring of distinct matrices larger than L2 so that every launch reads from HBM."""
+    import torch
+    from paper_2504_08791_b200 import binding
+    binding.lib()
+    fmt = {"q6_k": synth.FMT_Q6_K, "q8_0": synth.FMT_Q8_0, "f16": synth.FMT_F16}[args.gemv_fmt]
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+    out = {"metric": "gemv_GBs", "format": args.gemv_fmt, "unit": "GB/s", "peak": peak, "shapes": {}}
+    for rows, cols in ((8192, 8192), (8192, 28672)):
+        nbytes = rows * cols // synth.FMT_BLOCK_WEIGHTS[fmt] * synth.FMT_BLOCK_BYTES[fmt]
+        n_mats = max(2, int(400e6 // nbytes) + 1)
+        mats = [torch.from_numpy(synth.fmt_tensor(20 + i, fmt, rows, cols)).cuda() for i in range(n_mats)]
+        x = torch.from_numpy(synth.activations(20, 1, cols)).cuda()
+        y = torch.empty((1, rows), dtype=torch.float32, device="cuda")
+        for m in mats:
+            binding.prima_gemv_fmt(fmt, m, rows, cols, x, 1, y)
+        torch.cuda.synchronize()
+        reps = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for m in mats:
+                binding.prima_gemv_fmt(fmt, m, rows, cols, x, 1, y)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * n_mats)
+        gbs = nbytes / (us * 1e-6) / 1e9
+        out["shapes"][f"{rows}x{cols}"] = {"bytes": nbytes, "us": us, "GB/s": gbs, "frac_of_measured_peak": gbs / peak,
+                                           "distinct_matrices": n_mats}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -555,6 +589,8 @@ def main():
     ap.add_argument("--resident-layers", type=int, default=-1,
                     help="keep only the first N layers' matrices on the GPU, stream the others from pinned host memory every token")
     ap.add_argument("--stream-slots", type=int, default=0, help="device buffers for streamed layers (default 2)")
+    ap.add_argument("--gemv-fmt", default="", choices=["", "q6_k", "q8_0", "f16"],
+                    help="micro-benchmark of the single product in another weight format instead of the decoding loop")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
@@ -565,6 +601,10 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             print(json.dumps(run_reference(args)), flush=True)
+        return
+    if args.gemv_fmt:
+        if rank == 0:
+            print(json.dumps(run_gemv_fmt(args)), flush=True)
         return
     if args.warmup < 3:
         log("[bench] fewer than 3 warm-up steps: the number is not a valid measurement")

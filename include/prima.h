@@ -266,6 +266,34 @@ int prima_gemv_plan_create(const void* dev_w, int64_t rows, int64_t cols, int ma
 int prima_gemv_plan_run(prima_gemv_plan* plan, const float* dev_x, int n_cols, float* dev_y, void* stream);
 int prima_gemv_plan_destroy(prima_gemv_plan* plan);
 
+/* ---- the other weight formats of the paper's set Q (Appendix A.3, computation latency: Q = {Q4_K, Q5_K, Q6_K,
+ * Q8_0, FP16, FP32}; checkpoints called "Q4K" mix them).  The paper prints none of the layouts; these are the
+ * public ones of the file format its system reads:
+ *   PRIMA_FMT_Q8_0  34-byte block of 32 weights: binary16 d, 32 signed bytes q;  weight = d * q
+ *   PRIMA_FMT_Q6_K  210-byte super-block of 256 weights: ql[128], qh[64], signed byte scales sc[16], binary16 d;
+ *                   weight k = d * sc[k/16] * (v_k - 32); with k = 128 n + 32 i + l the low four bits of v_k are in
+ *                   byte ql[64 n + 32 (i & 1) + l] (low nibble for i < 2, high nibble otherwise) and its high two
+ *                   bits are bits 2i, 2i+1 of byte qh[32 n + l]
+ *   PRIMA_FMT_F16   binary16 values
+ *   PRIMA_FMT_Q4_K  the 144-byte super-block described at the top (the calls below forward to the _q4k calls)
+ * Matrices are row-major, cols a multiple of 256.  prima_dequant_fmt: n_blocks blocks (dev) -> fp32 (dev), the exact
+ * value (no rounding is needed: it fits binary32).  prima_gemv_fmt: y[c][r] = sum_k W[r][k] x[c][k], 1 <= n_cols <= 4;
+ * dev_w in its standard layout, read in place (nothing is allocated or re-tiled); the fp32 activations of all columns
+ * plus two rows of the matrix must fit 200 KiB of shared memory (PRIMA_ERR_ARG otherwise, with a message in
+ * prima_fmt_last_error).  dev_w must lie in an allocation whose size is a multiple of 16 bytes, as every cudaMalloc
+ * allocation is: rows are fetched in 16-byte pieces from the boundary at or below their first byte.  Per row
+ * |y - y_ref| <= 1e-3 * sum |w x| (fp32 accumulation).  Queued on `stream`, no waiting. */
+#define PRIMA_FMT_Q4_K 0
+#define PRIMA_FMT_Q6_K 1
+#define PRIMA_FMT_Q8_0 2
+#define PRIMA_FMT_F16 3
+int prima_fmt_block_weights(int fmt);   /* weights per block (0: unknown format) */
+int prima_fmt_block_bytes(int fmt);     /* bytes per block */
+int prima_dequant_fmt(int fmt, const void* dev_blocks, int64_t n_blocks, float* dev_out, void* stream);
+int prima_gemv_fmt(int fmt, const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols,
+                   float* dev_y, void* stream);
+const char* prima_fmt_last_error(void);
+
 /* The same product as prima_gemv_q4k for callers that cannot allocate device memory: programs that
  * gave all of the GPU's memory to their own arena at start-up, or latency-critical loops in which
  * cudaMalloc / cudaFree (which may stall the device, and may fail late) are not allowed.  The paper

@@ -31,6 +31,7 @@ EXPORTS = [
     "prima_launch_count", "prima_profile_enable", "prima_profile_read", "prima_dequant_q4k", "prima_gemv_q4k", "prima_gemv_plan_create", "prima_gemv_plan_run",
     "prima_gemv_plan_destroy", "prima_gemv_q4k_noalloc", "prima_gemv_q4k_noalloc_error",
     "prima_forward_window_seqs", "prima_kv_load_seq", "prima_kv_read_seq", "prima_ctx_set_option", "prima_stream_stats",
+    "prima_fmt_block_weights", "prima_fmt_block_bytes", "prima_dequant_fmt", "prima_gemv_fmt", "prima_fmt_last_error",
 ]
 
 
@@ -84,11 +85,17 @@ def lib():
         L.prima_gemv_plan_create.argtypes = [vp, i64, i64, i32, C.POINTER(vp)]
         L.prima_gemv_plan_run.argtypes = [vp, vp, i32, vp, vp]
         L.prima_gemv_plan_destroy.argtypes = [vp]
+        L.prima_fmt_block_weights.argtypes = [i32]
+        L.prima_fmt_block_bytes.argtypes = [i32]
+        L.prima_dequant_fmt.argtypes = [i32, vp, i64, vp, vp]
+        L.prima_gemv_fmt.argtypes = [i32, vp, i64, i64, vp, i32, vp, vp]
+        L.prima_fmt_last_error.argtypes = []
+        L.prima_fmt_last_error.restype = C.c_char_p
         L.prima_gemv_q4k_noalloc.argtypes = [vp, i64, i64, vp, i32, vp, vp]
         L.prima_gemv_q4k_noalloc_error.argtypes = []
         L.prima_gemv_q4k_noalloc_error.restype = C.c_char_p
         for name in EXPORTS:
-            if name not in ("prima_last_error", "prima_launch_count", "prima_gemv_q4k_noalloc_error"):
+            if name not in ("prima_last_error", "prima_launch_count", "prima_gemv_q4k_noalloc_error", "prima_fmt_last_error"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -124,6 +131,23 @@ def prima_dequant_q4k(dev_blocks, n_superblocks: int, dev_out, stream=None):
 
 def prima_gemv_q4k(dev_w, rows: int, cols: int, dev_x, n_cols: int, dev_y, stream=None):
     _check(lib().prima_gemv_q4k(_dev_ptr(dev_w), rows, cols, _dev_ptr(dev_x), n_cols, _dev_ptr(dev_y), _stream_ptr(stream)))
+
+
+FMT_Q4_K, FMT_Q6_K, FMT_Q8_0, FMT_F16 = 0, 1, 2, 3
+
+
+def _check_fmt(rc: int):
+    if rc != OK:
+        msg = lib().prima_fmt_last_error() or lib().prima_last_error(None)
+        raise PrimaError(rc, msg.decode() if msg else "")
+
+
+def prima_dequant_fmt(fmt: int, dev_blocks, n_blocks: int, dev_out, stream=None):
+    _check_fmt(lib().prima_dequant_fmt(fmt, _dev_ptr(dev_blocks), n_blocks, _dev_ptr(dev_out), _stream_ptr(stream)))
+
+
+def prima_gemv_fmt(fmt: int, dev_w, rows: int, cols: int, dev_x, n_cols: int, dev_y, stream=None):
+    _check_fmt(lib().prima_gemv_fmt(fmt, _dev_ptr(dev_w), rows, cols, _dev_ptr(dev_x), n_cols, _dev_ptr(dev_y), _stream_ptr(stream)))
 
 
 def prima_gemv_q4k_noalloc(dev_w, rows: int, cols: int, dev_x, n_cols: int, dev_y, stream=None):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libprima.so")
-SOURCES = ["api.cu", "q4k_pack.cu", "q4k_gemv.cu", "q4k_gemm_tokens.cu", "finish.cu", "attention.cu", "gemv_noalloc.cu"]
+SOURCES = ["api.cu", "q4k_pack.cu", "q4k_gemv.cu", "q4k_gemm_tokens.cu", "finish.cu", "attention.cu", "gemv_noalloc.cu", "formats.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "-Xptxas", "-v"]
 

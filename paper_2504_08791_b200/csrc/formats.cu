@@ -1,0 +1,269 @@
+// The other weight formats of the paper's set Q (Appendix A.3, computation latency): Q6_K, Q8_0 and FP16 matrices
+// in their standard row-major block layouts.  Bit-exact dequantisation and a streaming matrix-vector product.
+//
+// Layouts (the public ones of the file format the paper's system reads; the paper prints none):
+//   Q8_0  34-byte block of 32 weights: binary16 d, then 32 signed bytes q;            w = d * q
+//   Q6_K  210-byte super-block of 256 weights: ql[128] low nibbles, qh[64] high bit pairs, sc[16] signed byte
+//         scales (one per 16 weights), binary16 d;                                     w = d * sc * (v - 32)
+//         weight k = 128 n + 32 i + l: low nibble in byte ql[64 n + 32 (i & 1) + l] (low half for i < 2, high half
+//         otherwise), high two bits in bits 2i, 2i+1 of byte qh[32 n + l]
+//   FP16  binary16 values.
+//
+// The product.  One CTA works on one row at a time (persistent grid, rows dealt round-robin): the row's bytes are
+// brought into shared memory with 16-byte asynchronous copies (the copy starts at the 16-byte boundary at or
+// below the row's first byte, since rows of these formats need not start on one), the next row is requested
+// before the current one is used, and the activations of all columns sit in shared memory as fp32 for the
+// whole kernel.  Weights are converted to fp32 exactly (an integer placed in the mantissa of 2^23, minus the
+// bias) and accumulated with fp32 multiply-adds; the threads' sums are added in a fixed order, so the result
+// is the same from run to run.  Bound: HBM (0.82 / 1.06 / 2 bytes per weight); the conversion work makes the
+// kernel issue-limited before it reaches the copy bandwidth (see the measured fractions in the profiles).
+#include <cstdio>
+
+#include "../../include/prima.h"
+#include "common.cuh"
+
+namespace prima {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr float kMagic = 8388608.0f;      // 2^23: the integers 0..2^23-1 are the mantissas of [2^23, 2^24)
+
+__device__ __forceinline__ float half_bits_to_float(uint32_t bits) { return __half2float(__ushort_as_half(static_cast<unsigned short>(bits))); }
+__device__ __forceinline__ uint32_t lds_u16(const uint8_t* p) { return *reinterpret_cast<const uint16_t*>(p); }
+// Byte `sel` (0..3) of w as an exact float, plus 2^23.
+__device__ __forceinline__ float byte_plus_magic(uint32_t w, uint32_t sel) { return __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7440u | sel)); }
+
+// ---- dequantisation (the bit-exact definitions) ---------------------------------------------------------------
+__global__ void dequant_q8_0_kernel(const uint8_t* __restrict__ blocks, int64_t n_blocks, float* __restrict__ out) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= n_blocks * 32) return;
+  const uint8_t* b = blocks + (idx >> 5) * 34;
+  const float d = half_bits_to_float(b[0] | (b[1] << 8));
+  out[idx] = d * static_cast<float>(static_cast<int8_t>(b[2 + (idx & 31)]));      // 11 x 8 bits: exact
+}
+
+__global__ void dequant_q6k_kernel(const uint8_t* __restrict__ blocks, int64_t n_blocks, float* __restrict__ out) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= n_blocks * 256) return;
+  const uint8_t* b = blocks + (idx >> 8) * 210;
+  const int k = static_cast<int>(idx & 255);
+  const int n = k >> 7, i = (k >> 5) & 3, l = k & 31;
+  const uint32_t lo_byte = b[64 * n + 32 * (i & 1) + l];
+  const int v = static_cast<int>((i < 2 ? (lo_byte & 15u) : (lo_byte >> 4)) | (((b[128 + 32 * n + l] >> (2 * i)) & 3u) << 4));
+  const int sc = static_cast<int8_t>(b[192 + (k >> 4)]);
+  const float d = half_bits_to_float(b[208] | (b[209] << 8));
+  // 11 x 13 bits: exact; the factors are multiplied as floats so that a zero weight gets the sign of the product of
+  // the three signs, as in d * sc * (v - 32) evaluated in any order
+  out[idx] = d * (static_cast<float>(sc) * static_cast<float>(v - 32));
+}
+
+__global__ void dequant_f16_kernel(const uint8_t* __restrict__ blocks, int64_t n, float* __restrict__ out) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx < n) out[idx] = half_bits_to_float(blocks[2 * idx] | (blocks[2 * idx + 1] << 8));
+}
+
+// ---- the product ----------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(__cvta_generic_to_global(src)) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Sum over a row's weights of w * x for NC columns: the thread's share.  `row` points at the row's first byte
+// in shared memory (2-byte aligned), xs at the activations [NC][cols].
+template <int FMT, int NC>
+__device__ __forceinline__ void row_partial(const uint8_t* row, const float* xs, int64_t cols, float (&acc)[NC]) {
+  const int t = threadIdx.x;
+  if (FMT == PRIMA_FMT_Q8_0) {
+    // eight threads per block of 32 weights, four consecutive weights each
+    const int64_t n_blk = cols >> 5;
+    const int j = t & 7;
+    for (int64_t b = t >> 3; b < n_blk; b += kThreads / 8) {
+      const uint8_t* blk = row + b * 34;
+      const float d = half_bits_to_float(lds_u16(blk));
+      const uint32_t q = (lds_u16(blk + 2 + 4 * j) | (lds_u16(blk + 4 + 4 * j) << 16)) ^ 0x80808080u;      // q + 128 as unsigned bytes
+      float f[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) f[e] = byte_plus_magic(q, e) - (kMagic + 128.0f);
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const float4 x = *reinterpret_cast<const float4*>(xs + c * cols + 32 * b + 4 * j);
+        acc[c] = fmaf(d, fmaf(f[0], x.x, fmaf(f[1], x.y, fmaf(f[2], x.z, f[3] * x.w))), acc[c]);
+      }
+    }
+  } else if (FMT == PRIMA_FMT_Q6_K) {
+    // sixteen threads per super-block: thread u = (half n, four consecutive positions l0..l0+3), 16 weights each
+    const int64_t n_sb = cols >> 8;
+    const int u = t & 15, n = u >> 3, l0 = 4 * (u & 7);
+    for (int64_t s = t >> 4; s < n_sb; s += kThreads / 16) {
+      const uint8_t* sb = row + s * 210;
+      const uint8_t* pa = sb + 64 * n + l0;
+      const uint32_t ql_a = lds_u16(pa) | (lds_u16(pa + 2) << 16);
+      const uint32_t ql_b = lds_u16(pa + 32) | (lds_u16(pa + 34) << 16);
+      const uint8_t* ph = sb + 128 + 32 * n + l0;
+      const uint32_t qh = lds_u16(ph) | (lds_u16(ph + 2) << 16);
+      const float d = half_bits_to_float(lds_u16(sb + 208));
+      const int8_t* scp = reinterpret_cast<const int8_t*>(sb + 192 + 8 * n + (l0 >> 4));
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t src = (i & 1) ? ql_b : ql_a;
+        const uint32_t lo = i < 2 ? (src & 0x0f0f0f0fu) : ((src >> 4) & 0x0f0f0f0fu);
+        const uint32_t v4 = lo | (((qh >> (2 * i)) & 0x03030303u) << 4);      // four values 0..63
+        const float dsc = d * static_cast<float>(scp[2 * i]);
+        float f[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) f[e] = byte_plus_magic(v4, e) - (kMagic + 32.0f);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          const float4 x = *reinterpret_cast<const float4*>(xs + c * cols + 256 * s + 128 * n + 32 * i + l0);
+          acc[c] = fmaf(dsc, fmaf(f[0], x.x, fmaf(f[1], x.y, fmaf(f[2], x.z, f[3] * x.w))), acc[c]);
+        }
+      }
+    }
+  } else {      // FP16: two weights per 32-bit word
+    for (int64_t k = 2 * static_cast<int64_t>(t); k < cols; k += 2 * kThreads) {
+      const uint32_t w2 = lds_u16(row + 2 * k) | (lds_u16(row + 2 * k + 2) << 16);
+      const float2 wf = __half22float2(*reinterpret_cast<const __half2*>(&w2));
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const float2 x = *reinterpret_cast<const float2*>(xs + c * cols + k);
+        acc[c] = fmaf(wf.x, x.x, fmaf(wf.y, x.y, acc[c]));
+      }
+    }
+  }
+}
+
+template <int FMT, int NC>
+__global__ void __launch_bounds__(kThreads) gemv_fmt_kernel(const uint8_t* __restrict__ w, int64_t rows, int64_t cols, int64_t row_bytes,
+                                                             int64_t buf_bytes, const float* __restrict__ x, float* __restrict__ y) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  float* xs = reinterpret_cast<float*>(smem);                                            // [NC][cols]
+  uint8_t* bufs = smem + static_cast<size_t>(NC) * cols * sizeof(float);                 // two row buffers of buf_bytes
+  __shared__ float s_part[kThreads / 32][NC];
+  const int t = threadIdx.x;
+  // The bytes of row r, from the 16-byte boundary at or below its first byte; every 16-byte piece that the row
+  // touches lies inside the matrix's allocation rounded up to 16 bytes, which every CUDA allocation is.
+  auto request = [&](int64_t r, int slot) {
+    const uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(r * row_bytes);
+    const uintptr_t a0 = first & ~static_cast<uintptr_t>(15), a1 = (first + row_bytes + 15) & ~static_cast<uintptr_t>(15);
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(bufs + static_cast<size_t>(slot) * buf_bytes));
+    for (uintptr_t off = static_cast<uintptr_t>(t) * 16; off < a1 - a0; off += kThreads * 16) cp_async16(dst + static_cast<uint32_t>(off), reinterpret_cast<const void*>(a0 + off));
+  };
+  int64_t r = blockIdx.x;
+  if (r < rows) request(r, 0);
+  cp_async_commit();
+  for (int64_t i = t; i < NC * cols / 4; i += kThreads) reinterpret_cast<float4*>(xs)[i] = __ldg(reinterpret_cast<const float4*>(x) + i);
+  int slot = 0;
+  for (; r < rows; r += gridDim.x, slot ^= 1) {
+    const int64_t nxt = r + gridDim.x;
+    if (nxt < rows) request(nxt, slot ^ 1);
+    cp_async_commit();
+    cp_async_wait<1>();      // the current row's copies of this thread; the barrier makes everybody's visible
+    __syncthreads();
+    const uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(r * row_bytes);
+    const uint8_t* row = bufs + static_cast<size_t>(slot) * buf_bytes + (first & 15);
+    float acc[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) acc[c] = 0.f;
+    row_partial<FMT, NC>(row, xs, cols, acc);
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+      if ((t & 31) == 0) s_part[t >> 5][c] = acc[c];
+    }
+    __syncthreads();      // also: everybody is done with this row's buffer before the request after next overwrites it
+    if (t < NC) {
+      float sum = 0.f;
+#pragma unroll
+      for (int wp = 0; wp < kThreads / 32; ++wp) sum += s_part[wp][t];
+      y[static_cast<int64_t>(t) * rows + r] = sum;
+    }
+  }
+  cp_async_wait<0>();
+}
+
+template <int FMT>
+int launch_gemv_fmt(const uint8_t* w, int64_t rows, int64_t cols, int64_t row_bytes, const float* x, int n_cols, float* y, int sm_count,
+                    cudaStream_t st) {
+  const int64_t buf_bytes = ((row_bytes + 15) / 16 + 1) * 16;
+  const size_t smem = static_cast<size_t>(n_cols) * cols * sizeof(float) + 2 * static_cast<size_t>(buf_bytes);
+  if (smem > 200 * 1024) return cuda_rc(cudaErrorInvalidValue);
+  void (*kern)(const uint8_t*, int64_t, int64_t, int64_t, int64_t, const float*, float*) = nullptr;
+  switch (n_cols) {
+    case 1: kern = gemv_fmt_kernel<FMT, 1>; break;
+    case 2: kern = gemv_fmt_kernel<FMT, 2>; break;
+    case 3: kern = gemv_fmt_kernel<FMT, 3>; break;
+    default: kern = gemv_fmt_kernel<FMT, 4>; break;
+  }
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return cuda_rc(e);
+  const int per_sm = static_cast<int>(std::max<size_t>(1, std::min<size_t>(8, (220 * 1024) / (smem + 1024))));
+  const int64_t grid = std::min<int64_t>(rows, static_cast<int64_t>(sm_count) * per_sm);
+  kern<<<static_cast<unsigned>(grid), kThreads, smem, st>>>(w, rows, cols, row_bytes, buf_bytes, x, y);
+  e = cudaGetLastError();
+  return e == cudaSuccess ? 1 : cuda_rc(e);
+}
+
+thread_local char g_fmt_error[200] = "";
+int fmt_fail(const char* msg) {
+  snprintf(g_fmt_error, sizeof(g_fmt_error), "%s", msg);
+  return PRIMA_ERR_ARG;
+}
+
+}  // namespace
+}  // namespace prima
+
+using namespace prima;
+
+extern "C" {
+
+int prima_fmt_block_weights(int fmt) { return fmt == PRIMA_FMT_Q4_K || fmt == PRIMA_FMT_Q6_K ? 256 : fmt == PRIMA_FMT_Q8_0 ? 32 : fmt == PRIMA_FMT_F16 ? 1 : 0; }
+int prima_fmt_block_bytes(int fmt) { return fmt == PRIMA_FMT_Q4_K ? 144 : fmt == PRIMA_FMT_Q6_K ? 210 : fmt == PRIMA_FMT_Q8_0 ? 34 : fmt == PRIMA_FMT_F16 ? 2 : 0; }
+const char* prima_fmt_last_error(void) { return g_fmt_error; }
+
+int prima_dequant_fmt(int fmt, const void* dev_blocks, int64_t n_blocks, float* dev_out, void* stream) {
+  if (fmt == PRIMA_FMT_Q4_K) return prima_dequant_q4k(dev_blocks, n_blocks, dev_out, stream);
+  if (prima_fmt_block_weights(fmt) == 0) return fmt_fail("prima_dequant_fmt: unknown format");
+  if (n_blocks == 0) return PRIMA_OK;
+  if (!dev_blocks || !dev_out || n_blocks < 0) return fmt_fail("prima_dequant_fmt: bad argument");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t n = n_blocks * prima_fmt_block_weights(fmt);
+  const unsigned grid = static_cast<unsigned>((n + 255) / 256);
+  const uint8_t* b = static_cast<const uint8_t*>(dev_blocks);
+  if (fmt == PRIMA_FMT_Q8_0) dequant_q8_0_kernel<<<grid, 256, 0, st>>>(b, n_blocks, dev_out);
+  else if (fmt == PRIMA_FMT_Q6_K) dequant_q6k_kernel<<<grid, 256, 0, st>>>(b, n_blocks, dev_out);
+  else dequant_f16_kernel<<<grid, 256, 0, st>>>(b, n, dev_out);
+  if (cudaGetLastError() != cudaSuccess) {
+    snprintf(g_fmt_error, sizeof(g_fmt_error), "prima_dequant_fmt: launch failed");
+    return PRIMA_ERR_CUDA;
+  }
+  return PRIMA_OK;
+}
+
+int prima_gemv_fmt(int fmt, const void* dev_w, int64_t rows, int64_t cols, const float* dev_x, int n_cols, float* dev_y, void* stream) {
+  if (fmt == PRIMA_FMT_Q4_K) return prima_gemv_q4k(dev_w, rows, cols, dev_x, n_cols, dev_y, stream);
+  if (prima_fmt_block_weights(fmt) == 0) return fmt_fail("prima_gemv_fmt: unknown format");
+  if (!dev_w || !dev_x || !dev_y || rows < 1 || cols < 256 || cols % 256 != 0 || n_cols < 1 || n_cols > 4)
+    return fmt_fail("prima_gemv_fmt: rows >= 1, cols a positive multiple of 256 and 1 <= n_cols <= 4 are required");
+  const int64_t row_bytes = cols / prima_fmt_block_weights(fmt) * prima_fmt_block_bytes(fmt);
+  if (static_cast<int64_t>(n_cols) * cols * 4 + 2 * (row_bytes + 32) > 200 * 1024)
+    return fmt_fail("prima_gemv_fmt: the activations of all columns and two rows of the matrix must fit 200 KiB of shared memory");
+  int dev = 0, sm_count = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const uint8_t* w = static_cast<const uint8_t*>(dev_w);
+  int k;
+  if (fmt == PRIMA_FMT_Q8_0) k = launch_gemv_fmt<PRIMA_FMT_Q8_0>(w, rows, cols, row_bytes, dev_x, n_cols, dev_y, sm_count, st);
+  else if (fmt == PRIMA_FMT_Q6_K) k = launch_gemv_fmt<PRIMA_FMT_Q6_K>(w, rows, cols, row_bytes, dev_x, n_cols, dev_y, sm_count, st);
+  else k = launch_gemv_fmt<PRIMA_FMT_F16>(w, rows, cols, row_bytes, dev_x, n_cols, dev_y, sm_count, st);
+  if (k < 0) {
+    snprintf(g_fmt_error, sizeof(g_fmt_error), "prima_gemv_fmt: launch failed: %s", cudaGetErrorString(static_cast<cudaError_t>(-k)));
+    return PRIMA_ERR_CUDA;
+  }
+  return PRIMA_OK;
+}
+
+}  // extern "C"
