@@ -848,7 +848,9 @@ int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, 
   if (max_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
   const int rc = configure_kernels();
   if (rc != 0) return rc;
-  const int per_head = std::min(kMaxParts, std::max(1, 2 * sm_count / n_kv_heads));
+  // The whole launch should be about one wave of CTAs (two per SM): with many requests a CTA takes several chunks of
+  // its request and carries its running state from one to the next, instead of many waves of short-lived CTAs.
+  const int per_head = std::min(kMaxParts, std::max(1, 2 * sm_count / (n_kv_heads * seqs.n)));
   dim3 grid(std::min(max_chunks, per_head), n_kv_heads, seqs.n);      // CTAs beyond a request's own chunks leave at once
   int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;
   cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
