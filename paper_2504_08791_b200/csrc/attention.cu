@@ -76,23 +76,32 @@ __device__ __forceinline__ int swz(int dim) { return dim ^ (((dim >> 5) & 1) << 
 //    k slots are the positions  2t, 2t+1, 2t+8, 2t+9  of the warp's 16.  Over the eight instructions
 //    of one 64-dim half a lane therefore collects, for row g, the 16 consecutive head dims
 //    64 hf + 16 t + [0, 16)  (element 0 of instruction b -> + b, element 1 -> + 8 + b).
+
+// ---- a step of several tokens of one sequence: up to 64 query rows per KV head --------------------------
+// The query rows of a KV head (tokens x heads of the group) are cut into tiles of 16 (one m16n8k16 tile of rows),
+// and a CTA serves ONE tile: CTA (x, KV head, tile).  It takes the chunks x, x + gridDim.x, ... of the context and
+// carries the running (max, sum, output) of its 16 rows from chunk to chunk exactly as the one-token kernel does
+// (per-warp tiles in shared memory, no barrier in the chunk loop), so it leaves one partial result per CTA and the
+// merge kernel sees gridDim.x of them instead of one per chunk.  The cache is read once per tile (the re-reads
+// come from L2).  Every CTA that meets new positions forms their keys and values itself; the CTAs of tile 0 append
+// them to the cache.
 __global__ void __launch_bounds__(kThreads, 2)
-attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
-                    const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
-                    int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int n_chunks, int chunk_stride,
-                    float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp) {
+attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
+                 const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
+                 int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int n_chunks, int part_stride,
+                 float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp) {
   pdl_trigger();
-  constexpr int row_base = 0;
   extern __shared__ __align__(16) float dyn_smem[];
   __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
   __shared__ float s_inv[kMaxStepTok];
 
   const int group = n_q_heads / n_kv_heads;
-  const int n_rows = n_tok * group;                  // query rows served by this CTA
-  const int o_rows = n_rows <= 8 ? 8 : 16;           // rows kept of a 16-row tile
-  float* s_o = dyn_smem;                                               // [kWarps][o_rows][kRowPad]
-  float* q_s = s_o + kWarps * o_rows * kRowPad;                        // [n_rows][kRowPad] rotated queries of this KV head
-  __half* new_k = reinterpret_cast<__half*>(q_s + n_rows * kRowPad);   // [n_tok][128] keys of the new positions
+  const int n_rows = n_tok * group;                  // query rows of this KV head
+  const int row0 = 16 * static_cast<int>(blockIdx.z);       // first row of this CTA's tile
+  const int tile_rows = min(16, n_rows - row0);
+  float* s_o = dyn_smem;                                               // [kWarps][16][kRowPad]
+  float* q_s = s_o + kWarps * 16 * kRowPad;                            // [16][kRowPad] rotated queries of the tile
+  __half* new_k = reinterpret_cast<__half*>(q_s + 16 * kRowPad);       // [n_tok][128] keys of the new positions
   __half* new_v = new_k + n_tok * kHeadDim;
 
   const int kv = blockIdx.y;
@@ -149,13 +158,15 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   stamp_begin(stamp);
   if (pre_limit < pos && chunk * kChunk + warp * 16 + 16 > pre_limit) load_old(chunk * kChunk + warp * 16, pos);
 
-  // ---- finish the QKV product for this KV head.  Items: one rotation pair of a query row, and for a
-  //      CTA that owns a chunk with new positions also one pair of each new key and value.
+  // ---- finish the QKV product for this tile.  Items: one rotation pair of a query row of the tile, and for a CTA
+  //      that meets new positions also one pair of each new key and value.
   const int c_lo = pos / kChunk, c_hi = (n_ctx - 1) / kChunk;
-  const bool own_lo = c_lo % static_cast<int>(gridDim.x) == static_cast<int>(blockIdx.x);
-  const bool own_hi = c_hi % static_cast<int>(gridDim.x) == static_cast<int>(blockIdx.x);
-  const int n_q_items = n_rows * (kHeadDim / 2);
-  const int n_items = n_q_items + ((own_lo || own_hi) ? 2 * n_tok * (kHeadDim / 2) : 0);
+  const int gx = static_cast<int>(gridDim.x);
+  const bool meets_new = c_lo % gx == static_cast<int>(blockIdx.x) || c_hi % gx == static_cast<int>(blockIdx.x) ||
+                         (c_hi - c_lo >= 2);      // more than two chunks of new positions cannot happen (n_tok <= 8 < 128)
+  const bool appends = meets_new && blockIdx.z == 0;
+  const int n_q_items = tile_rows * (kHeadDim / 2);
+  const int n_items = n_q_items + (meets_new ? 2 * n_tok * (kHeadDim / 2) : 0);      // at most 1024 + 1024
   constexpr int kTrip = 4;
   for (int trip = 0; trip * kTrip * kThreads < n_items; ++trip) {      // same trip count for every thread
     const int base = trip * kTrip * kThreads + threadIdx.x;
@@ -165,20 +176,20 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
     for (int u = 0; u < kTrip; ++u) {
       const int idx = base + u * kThreads;
       if (idx < n_items) {
-        int tok, row0;
+        int tok, rowbase;
         const int i = idx % (kHeadDim / 2);
         if (idx < n_q_items) {
-          const int r = idx / (kHeadDim / 2);
+          const int r = row0 + idx / (kHeadDim / 2);
           tok = r / group;
-          row0 = (kv * group + r % group) * kHeadDim;
+          rowbase = (kv * group + r % group) * kHeadDim;
         } else {
           const int j = (idx - n_q_items) / (kHeadDim / 2);      // 0 .. 2 n_tok - 1: keys, then values
           tok = j % n_tok;
-          row0 = (n_q_heads + (j < n_tok ? 0 : n_kv_heads) + kv) * kHeadDim;
+          rowbase = (n_q_heads + (j < n_tok ? 0 : n_kv_heads) + kv) * kHeadDim;
         }
         const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
-        ra[u] = __ldcg(acc + tok * mpad + row0 + a);
-        rb[u] = __ldcg(acc + tok * mpad + row0 + b);
+        ra[u] = __ldcg(acc + tok * mpad + rowbase + a);
+        rb[u] = __ldcg(acc + tok * mpad + rowbase + b);
         cs[u] = __ldcg(rope_tab + tok * (kHeadDim / 2) + i);
       }
     }
@@ -197,11 +208,11 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
         const int i = idx % (kHeadDim / 2);
         const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
         if (idx < n_q_items) {
-          const int r = idx / (kHeadDim / 2);
-          const float inv = s_inv[r / group];
+          const int rl = idx / (kHeadDim / 2);      // row inside the tile
+          const float inv = s_inv[(row0 + rl) / group];
           const float x = acc_value(ra[u]) * inv, y = acc_value(rb[u]) * inv;
-          q_s[r * kRowPad + swz(a)] = x * cs[u].x - y * cs[u].y;
-          q_s[r * kRowPad + swz(b)] = y * cs[u].x + x * cs[u].y;
+          q_s[rl * kRowPad + swz(a)] = x * cs[u].x - y * cs[u].y;
+          q_s[rl * kRowPad + swz(b)] = y * cs[u].x + x * cs[u].y;
         } else {
           const int j = (idx - n_q_items) / (kHeadDim / 2);
           const int tok = j % n_tok;
@@ -214,8 +225,7 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
           sm[a] = ha;
           sm[b] = hb;
           const int p = pos + tok;
-          const bool mine = p / kChunk == c_lo ? own_lo : own_hi;
-          if (mine) {
+          if (appends && (p / kChunk) % gx == static_cast<int>(blockIdx.x)) {      // one CTA of tile 0 owns each new position
             __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + p) * kHeadDim;
             gd[a] = ha;
             gd[b] = hb;
@@ -227,154 +237,164 @@ attn_partial_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __
   __syncthreads();
 
   const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
+  // rows g (lo) and g + 8 (hi) of the tile
+  int row_tok[2];
+  const float* qrow[2];
+#pragma unroll
+  for (int hr = 0; hr < 2; ++hr) {
+    const int rl = g + 8 * hr;
+    const bool live = rl < tile_rows;
+    row_tok[hr] = live ? (row0 + rl) / group : -1;
+    qrow[hr] = q_s + (live ? rl : 0) * kRowPad;
+  }
+  float* so_lo = s_o + (warp * 16 + g) * kRowPad;
+  float* so_hi = so_lo + 8 * kRowPad;
+#pragma unroll
+  for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      *reinterpret_cast<float4*>(so_lo + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+      *reinterpret_cast<float4*>(so_hi + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};      // of rows g and g + 8, the same in the four lanes of a quad
   for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
-    const int wbase = chunk * kChunk + warp * 16;      // first position of this warp
+    const int wbase = chunk * kChunk + warp * 16;
     if (!first) load_old(wbase, pos);
     patch_new(wbase);
-    for (int tile = 0; tile * 16 < n_rows; ++tile) {
-      const bool hi_live = tile * 16 + 8 < n_rows;       // rows 8..15 of the tile exist
-      // ---- scores of the 16 positions (two blocks of 8); the Q fragments of rows (tile*16 + g) and
-      //      (+ 8) are built 32 head dims at a time
-      int row_tok[2];
-      const float* qrow[2];
+    float sc[2][4];
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t qa[2][4];
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
-        const int r = tile * 16 + g + 8 * hr;
-        const bool live = r < n_rows;
-        row_tok[hr] = live ? r / group : -1;
-        qrow[hr] = q_s + (live ? r : 0) * kRowPad;
-      }
-      float sc[2][4];
-#pragma unroll
-      for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        uint32_t qa[2][4];
-#pragma unroll
-        for (int hr = 0; hr < 2; ++hr) {
-          float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-          if (row_tok[hr] >= 0) {
-            a = *reinterpret_cast<const float4*>(qrow[hr] + swz(32 * j + 8 * t));
-            b = *reinterpret_cast<const float4*>(qrow[hr] + swz(32 * j + 8 * t) + 4);
-          }
-          qa[0][hr] = pack_h2(a.x * scale, a.y * scale);
-          qa[0][2 + hr] = pack_h2(a.z * scale, a.w * scale);
-          qa[1][hr] = pack_h2(b.x * scale, b.y * scale);
-          qa[1][2 + hr] = pack_h2(b.z * scale, b.w * scale);
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (row_tok[hr] >= 0) {
+          a = *reinterpret_cast<const float4*>(qrow[hr] + swz(32 * j + 8 * t));
+          b = *reinterpret_cast<const float4*>(qrow[hr] + swz(32 * j + 8 * t) + 4);
         }
-#pragma unroll
-        for (int pb = 0; pb < 2; ++pb) {
-          mma_f16(sc[pb], qa[0][0], qa[0][1], qa[0][2], qa[0][3], kreg[pb][j].x, kreg[pb][j].y);
-          mma_f16(sc[pb], qa[1][0], qa[1][1], qa[1][2], qa[1][3], kreg[pb][j].z, kreg[pb][j].w);
-        }
+        qa[0][hr] = pack_h2(a.x * scale, a.y * scale);
+        qa[0][2 + hr] = pack_h2(a.z * scale, a.w * scale);
+        qa[1][hr] = pack_h2(b.x * scale, b.y * scale);
+        qa[1][2 + hr] = pack_h2(b.z * scale, b.w * scale);
       }
-      // ---- mask, row maxima, exponentials
-      float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-      for (int pb = 0; pb < 2; ++pb)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int hr = e >> 1;
-          const int p = wbase + 8 * pb + 2 * t + (e & 1);
-          const bool ok = row_tok[hr] >= 0 && p <= pos + row_tok[hr];
-          sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
-          mx[hr] = fmaxf(mx[hr], sc[pb][e]);
-        }
-      float lsum[2];
-#pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
-        mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
-        lsum[hr] = 0.f;
-      }
-      uint32_t pa[4];
 #pragma unroll
       for (int pb = 0; pb < 2; ++pb) {
-        float pv[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int hr = e >> 1;
-          pv[e] = mx[hr] > -INFINITY ? expf(sc[pb][e] - mx[hr]) : 0.f;
-          lsum[hr] += pv[e];
-        }
-        pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g,   k slots of this block
-        pa[2 * pb + 1] = pack_h2(pv[2], pv[3]);    // row g+8
+        mma_f16(sc[pb], qa[0][0], qa[0][1], qa[0][2], qa[0][3], kreg[pb][j].x, kreg[pb][j].y);
+        mma_f16(sc[pb], qa[1][0], qa[1][1], qa[1][2], qa[1][3], kreg[pb][j].z, kreg[pb][j].w);
       }
-#pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 1);
-        lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 2);
-      }
-      // ---- O = P V: per 64-dim half eight instructions of 8 head dims each, then four 16-byte
-      //      stores per live row of the lane
-      float* so_lo = s_o + (warp * o_rows + g) * kRowPad;
-      float* so_hi = s_o + (warp * o_rows + g + 8) * kRowPad;      // used only when o_rows == 16
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll
-        for (int bh = 0; bh < 2; ++bh) {      // instructions 4 bh .. 4 bh + 3 of this half
-          float oc[4][4];
-#pragma unroll
-          for (int bb = 0; bb < 4; ++bb) {
-            const int b = 4 * bh + bb, j = b >> 1;
-            const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
-            const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
-            const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
-            const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
-            const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
-            const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
-            const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
-            oc[bb][0] = oc[bb][1] = oc[bb][2] = oc[bb][3] = 0.f;
-            mma_f16(oc[bb], pa[0], pa[1], pa[2], pa[3], b0, b1);
-          }
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int col = swz(64 * hf + 16 * t + 8 * e + 4 * bh);
-            *reinterpret_cast<float4*>(so_lo + col) = make_float4(oc[0][e], oc[1][e], oc[2][e], oc[3][e]);
-            if (hi_live) *reinterpret_cast<float4*>(so_hi + col) = make_float4(oc[0][2 + e], oc[1][2 + e], oc[2][2 + e], oc[3][2 + e]);
-          }
-        }
-      }
-      if (t == 0) {
-        s_m[warp][g] = mx[0];
-        s_m[warp][g + 8] = mx[1];
-        s_l[warp][g] = lsum[0];
-        s_l[warp][g + 8] = lsum[1];
-      }
-      __syncthreads();
-      // ---- combine the warps.  First the factors e^(m_w - M) of every (warp, row), one thread each;
-      //      then thread (row, group of 4 head dims) adds up its 16 bytes of the eight tiles.
-      const int live_rows = min(16, n_rows - tile * 16);
-      if (threadIdx.x < kWarps * 16) {
-        const int w = threadIdx.x >> 4, r = threadIdx.x & 15;
-        float big = -INFINITY;
-#pragma unroll
-        for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
-        const float mine = s_m[w][r];
-        s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
-        if (w == 0) s_big[r] = big;
-      }
-      __syncthreads();
-      for (int idx = threadIdx.x; idx < live_rows * (kHeadDim / 4); idx += kThreads) {
-        const int r = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
-        const int col = swz(d4);
-        float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
-        float l = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-          const float f = s_f[w][r];
-          const float4 v = *reinterpret_cast<const float4*>(s_o + (w * o_rows + r) * kRowPad + col);
-          l += f * s_l[w][r];
-          accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
-        }
-        const int rr = tile * 16 + r;
-        const int tok = rr / group, head = kv * group + rr % group;
-        const int64_t slot = (static_cast<int64_t>(row_base) + static_cast<int64_t>(tok) * n_q_heads + head) * chunk_stride + chunk;
-        *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
-        if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
-      }
-      __syncthreads();
     }
+    // ---- mask, row maxima, rescaling factors, exponentials
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int hr = e >> 1;
+        const int p = wbase + 8 * pb + 2 * t + (e & 1);
+        const bool ok = row_tok[hr] >= 0 && p <= pos + row_tok[hr];
+        sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
+        mx[hr] = fmaxf(mx[hr], sc[pb][e]);
+      }
+    float alpha[2], lsum[2], m_new[2];
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+      mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
+      mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
+      m_new[hr] = fmaxf(m_run[hr], mx[hr]);
+      alpha[hr] = m_run[hr] > -INFINITY ? expf(m_run[hr] - m_new[hr]) : 1.0f;      // nothing accumulated yet: the tile is zero
+      lsum[hr] = 0.f;
+    }
+    uint32_t pa[4];
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb) {
+      float pv[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int hr = e >> 1;
+        pv[e] = m_new[hr] > -INFINITY ? expf(sc[pb][e] - m_new[hr]) : 0.f;
+        lsum[hr] += pv[e];
+      }
+      pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g,   k slots of this block
+      pa[2 * pb + 1] = pack_h2(pv[2], pv[3]);    // row g+8
+    }
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+      lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 1);
+      lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 2);
+      l_run[hr] = l_run[hr] * alpha[hr] + lsum[hr];
+      m_run[hr] = m_new[hr];
+    }
+    // ---- O = P V, added to the warp's own tile: per 64-dim half eight instructions of 8 head dims each
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+      for (int bh = 0; bh < 2; ++bh) {      // instructions 4 bh .. 4 bh + 3 of this half
+        float oc[4][4];
+#pragma unroll
+        for (int bb = 0; bb < 4; ++bb) {
+          const int b = 4 * bh + bb, j = b >> 1;
+          const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
+          const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
+          const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
+          const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
+          const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
+          const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
+          const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
+          oc[bb][0] = oc[bb][1] = oc[bb][2] = oc[bb][3] = 0.f;
+          mma_f16(oc[bb], pa[0], pa[1], pa[2], pa[3], b0, b1);
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int col = swz(64 * hf + 16 * t + 8 * e + 4 * bh);
+          float4* dlo = reinterpret_cast<float4*>(so_lo + col);
+          const float4 olo = *dlo;
+          *dlo = make_float4(fmaf(olo.x, alpha[0], oc[0][e]), fmaf(olo.y, alpha[0], oc[1][e]), fmaf(olo.z, alpha[0], oc[2][e]),
+                             fmaf(olo.w, alpha[0], oc[3][e]));
+          float4* dhi = reinterpret_cast<float4*>(so_hi + col);
+          const float4 ohi = *dhi;
+          *dhi = make_float4(fmaf(ohi.x, alpha[1], oc[0][2 + e]), fmaf(ohi.y, alpha[1], oc[1][2 + e]), fmaf(ohi.z, alpha[1], oc[2][2 + e]),
+                             fmaf(ohi.w, alpha[1], oc[3][2 + e]));
+        }
+      }
+    }
+  }
+  if (t == 0) {
+    s_m[warp][g] = m_run[0];
+    s_m[warp][g + 8] = m_run[1];
+    s_l[warp][g] = l_run[0];
+    s_l[warp][g + 8] = l_run[1];
+  }
+  __syncthreads();
+  if (threadIdx.x < kWarps * 16) {
+    const int w = threadIdx.x >> 4, r = threadIdx.x & 15;
+    float big = -INFINITY;
+#pragma unroll
+    for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
+    const float mine = s_m[w][r];
+    s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
+    if (w == 0) s_big[r] = big;
+  }
+  __syncthreads();
+  // thread (row, four head dims) adds up the eight warps' tiles: one partial result of the CTA, numbered by blockIdx.x
+  for (int idx = threadIdx.x; idx < tile_rows * (kHeadDim / 4); idx += kThreads) {
+    const int r = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
+    const int col = swz(d4);
+    float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
+    float l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float f = s_f[w][r];
+      const float4 v = *reinterpret_cast<const float4*>(s_o + (w * 16 + r) * kRowPad + col);
+      l += f * s_l[w][r];
+      accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
+    }
+    const int rr = row0 + r;
+    const int tok = rr / group, head = kv * group + rr % group;
+    const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * part_stride + blockIdx.x;
+    *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
+    if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
   }
 }
 
@@ -763,9 +783,8 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
   stamp_end(stamp);
 }
 
-size_t partial_smem_bytes(int n_rows, int n_tok) {
-  const int o_rows = n_rows <= 8 ? 8 : 16;
-  return static_cast<size_t>(kWarps * o_rows + n_rows) * kRowPad * sizeof(float) + static_cast<size_t>(2) * n_tok * kHeadDim * sizeof(__half);
+size_t tile_smem_bytes(int n_tok) {
+  return static_cast<size_t>(kWarps * 16 + 16) * kRowPad * sizeof(float) + static_cast<size_t>(2) * n_tok * kHeadDim * sizeof(__half);
 }
 
 constexpr size_t kOneSmemBytes = static_cast<size_t>(kWarps * 8 + 8) * kRowPad * sizeof(float) + 2 * kHeadDim * sizeof(__half);
@@ -791,9 +810,9 @@ static int configure_kernels() {
   static bool configured[kMaxDevices] = {};
   int dev = -1;
   if (first_launch_on_device(configured, &dev)) {
-    cudaError_t e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(partial_smem_bytes(8 * kMaxStepTok, kMaxStepTok)));
-    if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_partial_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaError_t e0 = cudaFuncSetAttribute(attn_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(tile_smem_bytes(kMaxStepTok)));
+    if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_tile_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kOneSmemBytes));
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e0 != cudaSuccess) return cuda_rc(e0);
@@ -828,13 +847,17 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
                    scr.ml_part, static_cast<int>(grid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
     return e == cudaSuccess ? 2 : cuda_rc(e);
   }
-  cudaError_t e = launch_pdl(attn_partial_kernel, grid, dim3(kThreads), partial_smem_bytes(n_rows, n_tok), st, acc_qkv, mpad,
+  // several tokens: one CTA per (slot of chunks, KV head, tile of 16 query rows); about one wave of CTAs in all
+  const int n_tiles = (n_rows + 15) / 16;
+  const int per_tile = std::min(kMaxParts, std::max(1, 2 * sm_count / (n_kv_heads * n_tiles)));
+  dim3 tgrid(std::min(n_chunks, per_tile), n_kv_heads, n_tiles);
+  cudaError_t e = launch_pdl(attn_tile_kernel, tgrid, dim3(kThreads), tile_smem_bytes(n_tok), st, acc_qkv, mpad,
                              static_cast<const float*>(ssq.data), ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache,
-                             kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok, n_chunks, n_chunks, scr.o_part, scr.ml_part,
+                             kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part,
                              scr.stamp);
   if (e != cudaSuccess) return cuda_rc(e);
-  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * n_chunks) * sizeof(float), st,
-                 scr.o_part, scr.ml_part, n_chunks, n_chunks, n_q_heads, o, none, scr.stamp);
+  e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * tgrid.x) * sizeof(float), st,
+                 scr.o_part, scr.ml_part, static_cast<int>(tgrid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
   if (e != cudaSuccess) return cuda_rc(e);
   return 2;
 }
