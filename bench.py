@@ -554,8 +554,12 @@ def run_gemv_fmt(args):
         mats = [torch.from_numpy(synth.fmt_tensor(20 + i, fmt, rows, cols)).cuda() for i in range(n_mats)]
         x = torch.from_numpy(synth.activations(20, 1, cols)).cuda()
         y = torch.empty((1, rows), dtype=torch.float32, device="cuda")
-        for m in mats:
-            binding.prima_gemv_fmt(fmt, m, rows, cols, x, 1, y)
+        try:
+            for m in mats:
+                binding.prima_gemv_fmt(fmt, m, rows, cols, x, 1, y)
+        except binding.PrimaError as err:      # a row too long for the kernel's shared memory: the library says so
+            out["shapes"][f"{rows}x{cols}"] = {"unsupported": str(err)}
+            continue
         torch.cuda.synchronize()
         reps = 20
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

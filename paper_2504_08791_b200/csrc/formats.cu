@@ -13,10 +13,13 @@
 // brought into shared memory with 16-byte asynchronous copies (the copy starts at the 16-byte boundary at or
 // below the row's first byte, since rows of these formats need not start on one), the next row is requested
 // before the current one is used, and the activations of all columns sit in shared memory as fp32 for the
-// whole kernel.  Weights are converted to fp32 exactly (an integer placed in the mantissa of 2^23, minus the
-// bias) and accumulated with fp32 multiply-adds; the threads' sums are added in a fixed order, so the result
-// is the same from run to run.  Bound: HBM (0.82 / 1.06 / 2 bytes per weight); the conversion work makes the
-// kernel issue-limited before it reaches the copy bandwidth (see the measured fractions in the profiles).
+// whole kernel.  FP16 weights are multiplied in fp32.  For the two block formats the activations are held as in the
+// Q4_K kernels: 16-bit integers x_q = round(x / s_b) with one fp32 step s_b per block of 32, cut into a high and a
+// low signed byte, so that the sum over a group of weights is an exact integer from 4-way byte dot products
+// (Q8_0: q * x_q; Q6_K: v * x_q - 32 * sum(x_q), v the unsigned 6-bit value), scaled once per group by
+// d * s_b (* sc for Q6_K) in fp32.  A CTA takes several consecutive rows per iteration when rows are short (their
+// bytes are contiguous: one copy range), each row worked on by its own team of threads; the threads' sums are
+// added in a fixed order, so the result is the same from run to run.  Bound: HBM (0.82 / 1.06 / 2 bytes per weight).
 #include <cstdio>
 
 #include "../../include/prima.h"
@@ -184,24 +187,243 @@ __global__ void __launch_bounds__(kThreads) gemv_fmt_kernel(const uint8_t* __res
   cp_async_wait<0>();
 }
 
+// ---- the block formats with 16-bit integer activations ---------------------------------------------------------
+__device__ __forceinline__ int dp4a_ss(uint32_t a, uint32_t b, int c) { return __dp4a(static_cast<int>(a), static_cast<int>(b), c); }
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {      // unsigned bytes of a times signed bytes of b
+  int d;
+  asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+// Eight bytes at an even offset `a` of shared memory: three aligned words, shifted by 0 or 16 bits.
+__device__ __forceinline__ uint2 lds8_even(const uint8_t* smem, int a) {
+  const uint32_t* p = reinterpret_cast<const uint32_t*>(smem + (a & ~3));
+  const uint32_t w0 = p[0], w1 = p[1], w2 = p[2], sh = (a & 2) * 8;
+  return make_uint2(__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh));
+}
+
+// The shared-memory image of one column of activations is cut into chunks of eight consecutive values; chunk j has
+// its eight high bytes at 8 j, its low bytes at P + 8 j and the pair (sum of its eight x_q, step of its block of 32
+// as fp32 bits) at 2 P + 8 j, P = cols rounded up to 1024.  For Q8_0 chunk j holds values 8 j ..; for Q6_K the chunk
+// of values 256 s + 128 n + 32 i + 8 o .. is j = 128 (s / 4) + 32 i + 8 (s % 4) + 4 n + o, so that the 32 lanes of a
+// warp (four super-blocks s, halves n, octets o) read 256 consecutive bytes at each i.
+template <int FMT>
+__device__ __forceinline__ int chunk_slot(int kc) {
+  if (FMT != PRIMA_FMT_Q6_K) return kc;
+  const int s = kc >> 5, n = (kc >> 4) & 1, i = (kc >> 2) & 3, o = kc & 3;
+  return 128 * (s >> 2) + 32 * i + 8 * (s & 3) + 4 * n + o;
+}
+
+template <int FMT, int NC>
+__device__ __forceinline__ void row_partial_q(const uint8_t* smem, int rowoff, int col_bytes, int padded, int cols, int tl, int tpr,
+                                              float (&acc)[NC]) {
+  if (FMT == PRIMA_FMT_Q8_0) {
+    // two threads per block of 32 weights, sixteen consecutive weights each
+    const int n_blk = cols >> 5, j = tl & 1;
+    for (int b = tl >> 1; b < n_blk; b += tpr >> 1) {
+      const int blk = rowoff + 34 * b;
+      const float d = half_bits_to_float(lds_u16(smem + blk));
+      const int a = blk + 2 + 16 * j;
+      const uint32_t* p = reinterpret_cast<const uint32_t*>(smem + (a & ~3));
+      const uint32_t sh = (a & 2) * 8, w0 = p[0], w1 = p[1], w2 = p[2], w3 = p[3], w4 = p[4];
+      const uint32_t q0 = __funnelshift_r(w0, w1, sh), q1 = __funnelshift_r(w1, w2, sh), q2 = __funnelshift_r(w2, w3, sh), q3 = __funnelshift_r(w3, w4, sh);
+      const int ch = 16 * (2 * b + j);
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const uint8_t* xc = smem + c * col_bytes + ch;
+        const uint4 xh = *reinterpret_cast<const uint4*>(xc);
+        const uint4 xl = *reinterpret_cast<const uint4*>(xc + padded);
+        const float step = *reinterpret_cast<const float*>(xc + 2 * padded + 4);
+        const int h = dp4a_ss(q3, xh.w, dp4a_ss(q2, xh.z, dp4a_ss(q1, xh.y, dp4a_ss(q0, xh.x, 0))));
+        const int l = dp4a_ss(q3, xl.w, dp4a_ss(q2, xl.z, dp4a_ss(q1, xl.y, dp4a_ss(q0, xl.x, 0))));
+        acc[c] = fmaf(static_cast<float>(h * 256 + l), d * step, acc[c]);
+      }
+    }
+  } else {
+    // eight threads per super-block: thread = (half n, eight consecutive positions 8 o .. 8 o + 7), 32 weights each
+    const int n_sb = cols >> 8, n = (tl >> 2) & 1, o = tl & 3;
+    for (int s = tl >> 3; s < n_sb; s += tpr >> 3) {
+      const int sb = rowoff + 210 * s;
+      const uint2 qa = lds8_even(smem, sb + 64 * n + 8 * o), qb = lds8_even(smem, sb + 64 * n + 32 + 8 * o);
+      const uint2 qh = lds8_even(smem, sb + 128 + 32 * n + 8 * o);
+      const float d = half_bits_to_float(lds_u16(smem + sb + 208));
+      const int8_t* scp = reinterpret_cast<const int8_t*>(smem + sb + 192 + 8 * n + (o >> 1));
+      const int ch0 = 8 * (128 * (s >> 2) + 8 * (s & 3) + 4 * n + o);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint2 src = (i & 1) ? qb : qa;
+        const uint32_t v0 = (i < 2 ? (src.x & 0x0f0f0f0fu) : ((src.x >> 4) & 0x0f0f0f0fu)) | (((qh.x >> (2 * i)) & 0x03030303u) << 4);
+        const uint32_t v1 = (i < 2 ? (src.y & 0x0f0f0f0fu) : ((src.y >> 4) & 0x0f0f0f0fu)) | (((qh.y >> (2 * i)) & 0x03030303u) << 4);
+        const float dsc = d * static_cast<float>(scp[2 * i]);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          const uint8_t* xc = smem + c * col_bytes + ch0 + 256 * i;
+          const uint2 xh = *reinterpret_cast<const uint2*>(xc);
+          const uint2 xl = *reinterpret_cast<const uint2*>(xc + padded);
+          const int2 ss = *reinterpret_cast<const int2*>(xc + 2 * padded);
+          const int h = dp4a_us(v1, xh.y, dp4a_us(v0, xh.x, 0)), l = dp4a_us(v1, xl.y, dp4a_us(v0, xl.x, 0));
+          acc[c] = fmaf(static_cast<float>(h * 256 + l - 32 * ss.x), dsc * __int_as_float(ss.y), acc[c]);
+        }
+      }
+    }
+  }
+}
+
+constexpr int kMaxQThreads = 512;
+
+// rows_per_it (1, 2, 4 or 8) consecutive rows per iteration, blockDim.x / rows_per_it threads per row; a ring of
+// `depth` (2..6) buffers of buf_bytes each holds the rows on their way in.
+template <int FMT, int NC>
+__global__ void __launch_bounds__(kMaxQThreads) gemv_fmtq_kernel(const uint8_t* __restrict__ w, int64_t rows, int cols, int row_bytes, int rows_per_it,
+                                                                  int buf_bytes, int depth, const float* __restrict__ x, float* __restrict__ y) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  __shared__ float s_part[kMaxQThreads / 32][NC];
+  const int padded = (cols + 1023) & ~1023, col_bytes = 3 * padded;
+  const int ring = NC * col_bytes;      // offset of the ring of buffers
+  const int t = threadIdx.x, nthr = blockDim.x, lane = t & 31, warp = t >> 5;
+  const int64_t n_groups = (rows + rows_per_it - 1) / rows_per_it;
+  auto request = [&](int64_t grp, int slot) {
+    const int64_t r0 = grp * rows_per_it;
+    const int nr = static_cast<int>(min(static_cast<int64_t>(rows_per_it), rows - r0));
+    const uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(r0 * row_bytes);
+    const uintptr_t a0 = first & ~static_cast<uintptr_t>(15);
+    const int n16 = static_cast<int>((first + static_cast<uintptr_t>(nr) * row_bytes + 15 - a0) >> 4);
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem + ring + slot * buf_bytes));
+    for (int k = t; k < n16; k += nthr) cp_async16(dst + 16 * k, reinterpret_cast<const void*>(a0 + 16 * static_cast<uintptr_t>(k)));
+  };
+  int64_t grp = blockIdx.x;
+  for (int j = 0; j < depth - 1; ++j) {
+    if (grp + j * static_cast<int64_t>(gridDim.x) < n_groups) request(grp + j * static_cast<int64_t>(gridDim.x), j);
+    cp_async_commit();
+  }
+  // quantise the activations: one thread per chunk of eight values, four neighbouring lanes per block of 32
+  // (the number of chunks is a multiple of 32 and so is the stride: a warp is in a pass as a whole)
+  const int n_chunks = cols >> 3;
+  const bool x_vec = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+  for (int task = t; task < NC * n_chunks; task += nthr) {
+    const int c = task / n_chunks, kc = task - c * n_chunks;
+    const float* xp = x + static_cast<int64_t>(c) * cols + 8 * kc;
+    float v[8];
+    if (x_vec) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(xp)), b = __ldg(reinterpret_cast<const float4*>(xp) + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __ldg(xp + e);
+    }
+    float amax = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[e]));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    const bool ok = amax > 0.f && amax < 3.0e38f;
+    const float inv = ok ? __fdividef(32639.0f, amax) : 0.f;
+    uint32_t hi[2] = {0u, 0u}, lo[2] = {0u, 0u};
+    int sum = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int q = max(-32639, min(32639, __float2int_rn(v[e] * inv)));
+      const int l = ((q + 128) & 255) - 128, h = (q - l) >> 8;
+      sum += q;
+      hi[e >> 2] |= static_cast<uint32_t>(h & 255) << (8 * (e & 3));
+      lo[e >> 2] |= static_cast<uint32_t>(l & 255) << (8 * (e & 3));
+    }
+    uint8_t* xc = smem + c * col_bytes + 8 * chunk_slot<FMT>(kc);
+    *reinterpret_cast<uint2*>(xc) = make_uint2(hi[0], hi[1]);
+    *reinterpret_cast<uint2*>(xc + padded) = make_uint2(lo[0], lo[1]);
+    *reinterpret_cast<int2*>(xc + 2 * padded) = make_int2(sum, __float_as_int(ok ? amax * (1.0f / 32639.0f) : 0.f));
+  }
+  const int tpr = nthr / rows_per_it;      // threads per row (>= 32)
+  const int row_in = t / tpr, tl = t - row_in * tpr;
+  const int warps_per_row = tpr >> 5;
+  int slot = 0;      // iteration number modulo depth
+  for (; grp < n_groups; grp += gridDim.x, slot = slot + 1 == depth ? 0 : slot + 1) {
+    const int64_t nxt = grp + static_cast<int64_t>(depth - 1) * gridDim.x;
+    if (nxt < n_groups) request(nxt, slot == 0 ? depth - 1 : slot - 1);      // the buffer read in the iteration before this one
+    cp_async_commit();
+    // this group's copies of this thread (all but the depth-1 newest groups); the barrier makes everybody's (and the
+    // activations) visible
+    switch (depth) {
+      case 2: cp_async_wait<1>(); break;
+      case 3: cp_async_wait<2>(); break;
+      case 4: cp_async_wait<3>(); break;
+      case 5: cp_async_wait<4>(); break;
+      default: cp_async_wait<5>(); break;
+    }
+    __syncthreads();
+    const int64_t r0 = grp * rows_per_it;
+    const uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(r0 * row_bytes);
+    const int rowoff = ring + slot * buf_bytes + static_cast<int>(first & 15) + row_in * row_bytes;
+    float acc[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) acc[c] = 0.f;
+    if (r0 + row_in < rows) row_partial_q<FMT, NC>(smem, rowoff, col_bytes, padded, cols, tl, tpr, acc);
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+      if (lane == 0) s_part[warp][c] = acc[c];
+    }
+    __syncthreads();      // also: everybody is done with this group's buffer before the request after next overwrites it
+    if (t < rows_per_it * NC) {
+      const int rr = t / NC, c = t - rr * NC;
+      if (r0 + rr < rows) {
+        float sum = 0.f;
+        for (int wp = 0; wp < warps_per_row; ++wp) sum += s_part[rr * warps_per_row + wp][c];
+        y[static_cast<int64_t>(c) * rows + r0 + rr] = sum;
+      }
+    }
+  }
+  cp_async_wait<0>();
+}
+
 template <int FMT>
 int launch_gemv_fmt(const uint8_t* w, int64_t rows, int64_t cols, int64_t row_bytes, const float* x, int n_cols, float* y, int sm_count,
                     cudaStream_t st) {
-  const int64_t buf_bytes = ((row_bytes + 15) / 16 + 1) * 16;
-  const size_t smem = static_cast<size_t>(n_cols) * cols * sizeof(float) + 2 * static_cast<size_t>(buf_bytes);
-  if (smem > 200 * 1024) return cuda_rc(cudaErrorInvalidValue);
-  void (*kern)(const uint8_t*, int64_t, int64_t, int64_t, int64_t, const float*, float*) = nullptr;
+  if (FMT == PRIMA_FMT_F16) {
+    const int64_t buf_bytes = ((row_bytes + 15) / 16 + 1) * 16;
+    const size_t smem = static_cast<size_t>(n_cols) * cols * sizeof(float) + 2 * static_cast<size_t>(buf_bytes);
+    if (smem > 200 * 1024) return cuda_rc(cudaErrorInvalidValue);
+    void (*kern)(const uint8_t*, int64_t, int64_t, int64_t, int64_t, const float*, float*) = nullptr;
+    switch (n_cols) {
+      case 1: kern = gemv_fmt_kernel<PRIMA_FMT_F16, 1>; break;
+      case 2: kern = gemv_fmt_kernel<PRIMA_FMT_F16, 2>; break;
+      case 3: kern = gemv_fmt_kernel<PRIMA_FMT_F16, 3>; break;
+      default: kern = gemv_fmt_kernel<PRIMA_FMT_F16, 4>; break;
+    }
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_rc(e);
+    const int per_sm = static_cast<int>(std::max<size_t>(1, std::min<size_t>(8, (220 * 1024) / (smem + 1024))));
+    const int64_t grid = std::min<int64_t>(rows, static_cast<int64_t>(sm_count) * per_sm);
+    kern<<<static_cast<unsigned>(grid), kThreads, smem, st>>>(w, rows, cols, row_bytes, buf_bytes, x, y);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? 1 : cuda_rc(e);
+  }
+  constexpr int F = FMT == PRIMA_FMT_F16 ? PRIMA_FMT_Q8_0 : FMT;      // (the block formats only; keeps the F16 instantiation out)
+  // two CTAs of 256 threads a SM while the activations are small, one of 512 otherwise; what is left of a CTA's share
+  // of shared memory holds the ring: groups of 1..8 rows of up to 56 KiB, small enough for a ring of three
+  const size_t x_bytes = static_cast<size_t>(n_cols) * 3 * static_cast<size_t>((cols + 1023) / 1024 * 1024);
+  if (x_bytes + 2 * (static_cast<size_t>(row_bytes) + 32) > 215 * 1024) return cuda_rc(cudaErrorInvalidValue);
+  const int per_sm = x_bytes <= 40 * 1024 && x_bytes + 3 * (static_cast<size_t>(row_bytes) + 32) <= 107 * 1024 ? 2 : 1;
+  const size_t share = (216 * 1024) / per_sm - 1024;
+  const size_t max_group = std::min<size_t>(56 * 1024, (share - x_bytes) / 3);
+  int rows_per_it = 1;
+  while (rows_per_it < 8 && static_cast<size_t>(row_bytes) * rows_per_it * 2 + 32 <= max_group) rows_per_it *= 2;
+  const int64_t buf_bytes = ((row_bytes * rows_per_it + 15) / 16 + 1) * 16;
+  const int depth = static_cast<int>(std::min<size_t>(6, (share - x_bytes) / static_cast<size_t>(buf_bytes)));      // >= 2 by the check above
+  const size_t smem = x_bytes + static_cast<size_t>(depth) * buf_bytes;
+  void (*kern)(const uint8_t*, int64_t, int, int, int, int, int, const float*, float*) = nullptr;
   switch (n_cols) {
-    case 1: kern = gemv_fmt_kernel<FMT, 1>; break;
-    case 2: kern = gemv_fmt_kernel<FMT, 2>; break;
-    case 3: kern = gemv_fmt_kernel<FMT, 3>; break;
-    default: kern = gemv_fmt_kernel<FMT, 4>; break;
+    case 1: kern = gemv_fmtq_kernel<F, 1>; break;
+    case 2: kern = gemv_fmtq_kernel<F, 2>; break;
+    case 3: kern = gemv_fmtq_kernel<F, 3>; break;
+    default: kern = gemv_fmtq_kernel<F, 4>; break;
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return cuda_rc(e);
-  const int per_sm = static_cast<int>(std::max<size_t>(1, std::min<size_t>(8, (220 * 1024) / (smem + 1024))));
-  const int64_t grid = std::min<int64_t>(rows, static_cast<int64_t>(sm_count) * per_sm);
-  kern<<<static_cast<unsigned>(grid), kThreads, smem, st>>>(w, rows, cols, row_bytes, buf_bytes, x, y);
+  const int64_t n_groups = (rows + rows_per_it - 1) / rows_per_it;
+  const int64_t grid = std::min<int64_t>(n_groups, static_cast<int64_t>(sm_count) * per_sm);
+  kern<<<static_cast<unsigned>(grid), kMaxQThreads / per_sm, smem, st>>>(w, rows, static_cast<int>(cols), static_cast<int>(row_bytes), rows_per_it,
+                                                                                   static_cast<int>(buf_bytes), depth, x, y);
   e = cudaGetLastError();
   return e == cudaSuccess ? 1 : cuda_rc(e);
 }
@@ -247,8 +469,10 @@ int prima_gemv_fmt(int fmt, const void* dev_w, int64_t rows, int64_t cols, const
   if (prima_fmt_block_weights(fmt) == 0) return fmt_fail("prima_gemv_fmt: unknown format");
   if (!dev_w || !dev_x || !dev_y || rows < 1 || cols < 256 || cols % 256 != 0 || n_cols < 1 || n_cols > 4)
     return fmt_fail("prima_gemv_fmt: rows >= 1, cols a positive multiple of 256 and 1 <= n_cols <= 4 are required");
+  if (reinterpret_cast<uintptr_t>(dev_w) & 1) return fmt_fail("prima_gemv_fmt: dev_w must be at an even address");
   const int64_t row_bytes = cols / prima_fmt_block_weights(fmt) * prima_fmt_block_bytes(fmt);
-  if (static_cast<int64_t>(n_cols) * cols * 4 + 2 * (row_bytes + 32) > 200 * 1024)
+  const int64_t x_bytes = fmt == PRIMA_FMT_F16 ? cols * 4 : 3 * ((cols + 1023) / 1024 * 1024);
+  if (static_cast<int64_t>(n_cols) * x_bytes + 2 * (row_bytes + 32) > 200 * 1024)
     return fmt_fail("prima_gemv_fmt: the activations of all columns and two rows of the matrix must fit 200 KiB of shared memory");
   int dev = 0, sm_count = 0;
   cudaGetDevice(&dev);
