@@ -248,6 +248,10 @@ def run_ours(args, rank, world, local_rank):
     ctx = build_gpu_model(binding, cfg, seed, n_ctx, local_rank, n_requests=R,
                           on_layer=whole.on_layer if whole else None, on_globals=whole.on_globals if whole else None,
                           resident_layers=resident, stream_slots=args.stream_slots)
+    if args.l2_ahead_mb >= 0:
+        ctx.set_option(binding.OPT_L2_AHEAD_BYTES, args.l2_ahead_mb << 20)
+    if args.l2_ahead_o_mb >= 0:
+        ctx.set_option(binding.OPT_L2_AHEAD_O_BYTES, args.l2_ahead_o_mb << 20)
     bpt = bytes_per_token(cfg, n_ctx)
     if R > 1:                                     # the weights are read once per step, every request's cache once
         bpt = dict(bpt, total=bpt["total"] + (R - 1) * L_kv_bytes(cfg, n_ctx))
@@ -593,6 +597,8 @@ def main():
     ap.add_argument("--resident-layers", type=int, default=-1,
                     help="keep only the first N layers' matrices on the GPU, stream the others from pinned host memory every token")
     ap.add_argument("--stream-slots", type=int, default=0, help="device buffers for streamed layers (default 2)")
+    ap.add_argument("--l2-ahead-mb", type=int, default=-1, help="MiB of the gate/up matrix asked into L2 during attention (default: the library's)")
+    ap.add_argument("--l2-ahead-o-mb", type=int, default=-1, help="MiB more of it asked into L2 during the O product (default: the library's)")
     ap.add_argument("--gemv-fmt", default="", choices=["", "q6_k", "q8_0", "f16"],
                     help="micro-benchmark of the single product in another weight format instead of the decoding loop")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -207,6 +207,15 @@ int prima_sync(prima_ctx* ctx);
  * was created, and the summed duration of those copies in milliseconds (waits for the copy stream). */
 #define PRIMA_OPT_RESIDENT_LAYERS 3
 #define PRIMA_OPT_STREAM_SLOTS 4
+/* PRIMA_OPT_L2_AHEAD_BYTES, PRIMA_OPT_L2_AHEAD_O_BYTES: attention reads little and leaves HBM idle, and so does the
+ * short O product (Section 4's footnote: decoding is bound by the memory stream, so every idle stretch of it is
+ * lost time).  In a step of one token the attention kernel of a layer therefore asks for the first `value` bytes
+ * of the gate/up matrix, the long stream that comes next, into L2, with requests nothing waits for, and the O
+ * product for the PRIMA_OPT_L2_AHEAD_O_BYTES that follow them.  -1 (default): a sixteenth of the matrix each;
+ * 0 switches one off; otherwise a multiple of 16 up to 2^30.  Results do not depend on them.  May be set at any
+ * time between steps. */
+#define PRIMA_OPT_L2_AHEAD_BYTES 5
+#define PRIMA_OPT_L2_AHEAD_O_BYTES 6
 int prima_ctx_set_option(prima_ctx* ctx, int option, int64_t value);
 int prima_stream_stats(prima_ctx* ctx, int64_t* bytes_copied, double* copy_ms);
 

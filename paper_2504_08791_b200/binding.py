@@ -24,6 +24,8 @@ OPT_FIRST_WAIT_POLLS = 1
 OPT_FAIL_AFTER_LAUNCHES = 2
 OPT_RESIDENT_LAYERS = 3
 OPT_STREAM_SLOTS = 4
+OPT_L2_AHEAD_BYTES = 5
+OPT_L2_AHEAD_O_BYTES = 6
 
 EXPORTS = [
     "prima_ctx_create", "prima_ctx_destroy", "prima_load_q4k_weights", "prima_forward_window", "prima_logits",

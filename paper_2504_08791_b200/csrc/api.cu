@@ -104,6 +104,8 @@ struct prima_ctx {
   // known to be in memory and may be read by the attention kernels before their dependency wait.
   int unsynced_min_pos = 0x7fffffff;
   uint32_t first_wait_polls = 0;   // PRIMA_OPT_FIRST_WAIT_POLLS (0: the ordinary limit)
+  int64_t l2_ahead_bytes = -1;     // PRIMA_OPT_L2_AHEAD_BYTES (-1: a sixteenth of the gate/up matrix)
+  int64_t l2_ahead_o_bytes = -1;   // PRIMA_OPT_L2_AHEAD_O_BYTES
   int64_t fail_after = -1;         // PRIMA_OPT_FAIL_AFTER_LAUNCHES: launch steps still allowed before an injected failure (-1: off)
 
   // optional per-class device timing (prima_profile_*): mode 1 = a pair of events around every launch,
@@ -677,6 +679,31 @@ int prima_load_q4k_weights(prima_ctx* c, int layer, int tensor_id, const void* d
 static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos0,
                                  int n_tok, const int32_t* seq, const int32_t* pos);
 
+// Attention reads little and leaves HBM idle, and so does the O product (its matrix is short: the kernel is bound by
+// its start-up, not by the stream).  In a step of one token their CTAs ask for the head of the gate/up matrix, the
+// long HBM-bound stream that follows, into L2: attention for the first l2_ahead_bytes, the O product for the next
+// l2_ahead_o_bytes; by default a sixteenth of the matrix each (measured: larger requests slow attention down by
+// more than they save; steps of several tokens are not bound by the stream and gain nothing).
+static int64_t ahead_share(const Layer& L, int64_t option) {
+  const int64_t all = static_cast<int64_t>(L.gu.bytes());
+  return std::min(all, option >= 0 ? option : all / 16 / 16384 * 16384);
+}
+static L2Ahead attn_ahead(const prima_ctx* c, const Layer& L, int n_tok) {
+  L2Ahead a;
+  if (n_tok != 1) return a;
+  a.ptr[0] = L.gu.data;
+  a.bytes[0] = static_cast<unsigned long long>(ahead_share(L, c->l2_ahead_bytes));
+  return a;
+}
+static L2Ahead o_ahead(const prima_ctx* c, const Layer& L, int n_tok) {
+  L2Ahead a;
+  if (n_tok != 1) return a;
+  const int64_t first = ahead_share(L, c->l2_ahead_bytes);
+  a.ptr[0] = L.gu.data + first;
+  a.bytes[0] = static_cast<unsigned long long>(std::min(static_cast<int64_t>(L.gu.bytes()) - first, ahead_share(L, c->l2_ahead_o_bytes)));
+  return a;
+}
+
 static int forward_window_impl(prima_ctx* c, int layer_begin, int layer_end, const float* hidden_in, float* hidden_out, int pos0,
                                int n_tok, const int32_t* seq, const int32_t* pos) {
   DeviceGuard guard(c->cfg.device);
@@ -746,6 +773,7 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.qkv), launch_gemv_partials(L.qkv, in, n_tok, c->acc_qkv, c->sm_count, st), "gemv(qkv)");
     c->ssq_attn = in.ssq_out;
     c->ssq_attn.eps = g.rms_eps;
+    c->attn.ahead = attn_ahead(c, L, n_tok);
     if (!seq) {
       c->attn.stamp = next_stamp(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos0 + n_tok), 2);
       LAUNCH_P(c, PRIMA_PROF_ATTENTION, static_cast<int64_t>(2) * G * kHeadDim * 2 * (pos0 + n_tok),
@@ -766,11 +794,14 @@ static int forward_window_launch(prima_ctx* c, int layer_begin, int layer_end, c
                launch_attention_seqs(c->acc_qkv, L.qkv.mpad(), c->ssq_attn, c->rope_tab, g.rope_mode, as, stable_below, g.kv_capacity, H, G, c->attn,
                                      c->obuf, c->sm_count, st), "attention");
     }
+    // Attention leaves HBM idle: its CTAs ask for the O matrix and the head of the gate/up matrix into L2, and the O
+    // product, which then finds its weights there, asks for the next stretch of gate/up.
     GemvIn in_o;                                 // O: plain attention output
     in_o.kind = kPlain; in_o.x = c->obuf; in_o.status = c->status; in_o.first_wait_polls = c->first_wait_polls;
     in_o.zero0 = c->acc_qkv; in_o.zero0_n = static_cast<int64_t>(n_tok) * L.qkv.mpad();
     in_o.zero1 = c->acc_down; in_o.zero1_n = static_cast<int64_t>(n_tok) * mpad_e;
     in_o.out_order = kOrderResidual;
+    in_o.ahead = o_ahead(c, L, n_tok);
     in_o.stamp = next_stamp(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), 1, PRIMA_PROF_GEMV_O);
     LAUNCH_P(c, PRIMA_PROF_GEMV, q4k_bytes(L.o), launch_gemv_partials(L.o, in_o, n_tok, c->acc_o, c->sm_count, st), "gemv(o)");
     GemvIn in_f;                                 // gate/up: h_b + O projection -> h_a
@@ -990,6 +1021,11 @@ int prima_ctx_set_option(prima_ctx* c, int option, int64_t value) {
       }
       return PRIMA_OK;
     }
+    case PRIMA_OPT_L2_AHEAD_BYTES:
+    case PRIMA_OPT_L2_AHEAD_O_BYTES:
+      if (value < -1 || value > (int64_t(1) << 30) || (value > 0 && value % 16 != 0)) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_L2_AHEAD_*: -1 or a multiple of 16 in 0 .. 2^30");
+      (option == PRIMA_OPT_L2_AHEAD_BYTES ? c->l2_ahead_bytes : c->l2_ahead_o_bytes) = value;
+      return PRIMA_OK;
     case PRIMA_OPT_FAIL_AFTER_LAUNCHES:
       if (value < -1) return fail(c, PRIMA_ERR_ARG, "PRIMA_OPT_FAIL_AFTER_LAUNCHES: value below -1");
       c->fail_after = value;

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
                  const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
                  int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int n_chunks, int part_stride,
-                 float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp) {
+                 float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp, const L2Ahead ahead) {
   pdl_trigger();
   extern __shared__ __align__(16) float dyn_smem[];
   __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
@@ -156,6 +156,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
   load_old(chunk * kChunk + warp * 16, pre_limit);
   pdl_wait();
   stamp_begin(stamp);
+  if (threadIdx.x == 0) l2_ahead(ahead, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), gridDim.x * gridDim.y * gridDim.z);
   if (pre_limit < pos && chunk * kChunk + warp * 16 + 16 > pre_limit) load_old(chunk * kChunk + warp * 16, pos);
 
   // ---- finish the QKV product for this tile.  Items: one rotation pair of a query row of the tile, and for a CTA
@@ -414,7 +415,7 @@ attn_one_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __rest
                 const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
                 int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_chunks, int part_stride,
                 float* __restrict__ o_part, float2* __restrict__ ml_part, int* __restrict__ tickets, float* __restrict__ o,
-                const AttnSeqs seqs, const Stamp stamp) {
+                const AttnSeqs seqs, const Stamp stamp, const L2Ahead ahead) {
   pdl_trigger();
   int row_base = 0;                 // first output row (request * heads) of this CTA's request
   if (seqs.n > 0) {                 // one request per blockIdx.z: its own cache and position
@@ -633,6 +634,8 @@ attn_one_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __rest
       }
     }
   }
+  // this CTA's cache reads are over: from here on HBM has nothing to do for it
+  if (threadIdx.x == 0) l2_ahead(ahead, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), gridDim.x * gridDim.y * gridDim.z);
   if (t == 0) {
     s_m[warp][g] = m_run;
     s_l[warp][g] = l_run;
@@ -840,7 +843,7 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
     int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;
     cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
                                ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads,
-                               pos, stable_below, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, none, scr.stamp);
+                               pos, stable_below, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, none, scr.stamp, scr.ahead);
     if (e != cudaSuccess) return cuda_rc(e);
     if (tickets) return 1;
     e = launch_pdl(attn_merge_kernel, dim3(n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * grid.x) * sizeof(float), st, scr.o_part,
@@ -854,7 +857,7 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
   cudaError_t e = launch_pdl(attn_tile_kernel, tgrid, dim3(kThreads), tile_smem_bytes(n_tok), st, acc_qkv, mpad,
                              static_cast<const float*>(ssq.data), ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache,
                              kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part,
-                             scr.stamp);
+                             scr.stamp, scr.ahead);
   if (e != cudaSuccess) return cuda_rc(e);
   e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * tgrid.x) * sizeof(float), st,
                  scr.o_part, scr.ml_part, static_cast<int>(tgrid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
@@ -879,7 +882,7 @@ int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, 
   cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
                              ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps, rope_tab, rope_mode,
                              static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads, n_kv_heads, 0, stable_below,
-                             max_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, seqs, scr.stamp);
+                             max_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, seqs, scr.stamp, scr.ahead);
   if (e != cudaSuccess) return cuda_rc(e);
   if (tickets) return 1;
   e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * grid.x) * sizeof(float), st, scr.o_part,

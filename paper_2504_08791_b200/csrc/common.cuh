@@ -58,6 +58,13 @@ struct Stamp {
   unsigned long long* t1 = nullptr;
 };
 
+// Weights that a later kernel of the queue will stream, asked into L2 ahead of time by a kernel that leaves HBM idle
+// (attention and the product after it, which reads what attention had fetched).  Nothing waits for these requests.
+struct L2Ahead {
+  const uint8_t* ptr[2] = {nullptr, nullptr};      // device, 16-byte aligned
+  unsigned long long bytes[2] = {0, 0};            // multiples of 16
+};
+
 struct TiledMat {
   uint8_t* data = nullptr;   // device, n_sb * n_rt * 1152 bytes
   int64_t rows = 0;          // logical rows (of the fused matrix)
@@ -150,6 +157,7 @@ struct GemvIn {
   int* status = nullptr;           // device word: bit 0 set if a bounded wait gave up, bit 1 if a partial sum was out of range
   uint32_t first_wait_polls = 0;   // 0: the ordinary limit; otherwise the poll limit of every warp's first wait + 1 (test hook)
   Stamp stamp;
+  L2Ahead ahead;                   // requested by the CTAs once the predecessor kernel is done
 };
 int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, int sm_count, cudaStream_t st);
 
@@ -181,6 +189,7 @@ struct AttnScratch {
   int max_chunks;
   int* tickets;     // [kMaxTok][G], all zero between launches (see attn_one_kernel)
   Stamp stamp;      // of the next attention launch (both kernels share it)
+  L2Ahead ahead;    // requested by the CTAs of the next attention launch as they start
 };
 // Several independent requests in one launch: token t of the step belongs to a request with its own
 // cache (k[t], v[t]) and position pos[t]; rows, statistics, rotary table and outputs of token t are
@@ -259,6 +268,19 @@ __device__ __forceinline__ void stamp_end(const Stamp& s) {
   if (s.t1) {
     __syncthreads();
     if (threadIdx.x == 0) atomicMax(s.t1, global_ns());
+  }
+}
+
+// Called by one thread of each CTA: CTA `cta` of `n_ctas` asks for every n_ctas-th piece of 16 KiB of both spans.
+__device__ __forceinline__ void l2_ahead(const L2Ahead& a, unsigned cta, unsigned n_ctas) {
+  constexpr unsigned long long kPiece = 16384;
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+    const unsigned long long bytes = a.bytes[s];
+    for (unsigned long long off = cta * kPiece; off < bytes; off += n_ctas * kPiece) {
+      const unsigned size = static_cast<unsigned>(min(kPiece, bytes - off));
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.ptr[s] + off), "r"(size) : "memory");
+    }
   }
 }
 

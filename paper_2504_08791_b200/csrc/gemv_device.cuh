@@ -128,6 +128,7 @@ struct GemvParams {
   int out_order;
   int* status;
   Stamp stamp;
+  L2Ahead ahead;
   uint32_t first_wait_polls;   // poll limit of a warp's first wait (kWaitLimit in normal use; a test lowers it to exercise the give-up path)
 };
 

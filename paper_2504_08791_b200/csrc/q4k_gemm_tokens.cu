@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(NB * kMaxWarps * 32, TokCfg<NB>::kCtasPerSm) g
       pdl_wait();
       waited = true;
       stamp_begin(P.stamp);
+      if (threadIdx.x == 0) l2_ahead(P.ahead, blockIdx.x, gridDim.x);
       clear_arrays();
     }
     {

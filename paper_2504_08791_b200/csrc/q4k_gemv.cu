@@ -314,6 +314,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
       pdl_wait();
       waited = true;
       stamp_begin(P.stamp);
+      if (threadIdx.x == 0) l2_ahead(P.ahead, blockIdx.x, gridDim.x);
       clear_arrays();
     }
     {
@@ -482,6 +483,7 @@ int launch_gemv_partials(const TiledMat& w, GemvIn& in, int n_tok, acc_t* acc, i
   P.zero0 = in.zero0; P.zero0_n = in.zero0_n; P.zero1 = in.zero1; P.zero1_n = in.zero1_n;
   P.out_order = in.out_order;
   P.stamp = in.stamp;
+  P.ahead = in.ahead;
   P.first_wait_polls = in.first_wait_polls ? in.first_wait_polls - 1 : kWaitLimit;
   if ((in.out_order == kOrderResidual && w.mpad() % 256 != 0) || (in.out_order == kOrderSwiglu && w.mpad() % 512 != 0)) return cuda_rc(cudaErrorInvalidValue);
   int launches = 0;

@@ -299,6 +299,26 @@ def test_a_wait_that_gives_up_is_reported_once_and_the_next_step_is_clean(gpu, n
     p.close()
 
 
+def test_weights_asked_into_l2_ahead_of_time_change_no_bit(gpu):
+    """The requests that bring the head of the gate/up matrix into L2 while attention and the O product run are
+    hints: switched off, at their defaults, larger than the matrix or cut at odd places, the step gives the same bits."""
+    torch, binding = gpu
+    cfg = synth.model_config("small")
+    pos = 77
+    h0 = synth.activations(61, 1, cfg["hidden"])
+    p = Pair(gpu, cfg, seed=61, n_prefill=pos, with_globals=False)
+    base = p.gpu_window(0, cfg["n_layers"], h0, pos)
+    for ahead, ahead_o in ((0, 0), (16, 0), (0, 1 << 30), (1 << 30, 1 << 30), (16 * 1000 + 16, 48), (-1, -1)):
+        p.ctx.set_option(binding.OPT_L2_AHEAD_BYTES, ahead)
+        p.ctx.set_option(binding.OPT_L2_AHEAD_O_BYTES, ahead_o)
+        again = p.gpu_window(0, cfg["n_layers"], h0, pos)      # same position again: the cache entry is rewritten with the same bits
+        assert np.array_equal(again.view(np.uint32), base.view(np.uint32)), (ahead, ahead_o)
+    for bad in (-2, 24, (1 << 30) + 16):
+        with pytest.raises(binding.PrimaError):
+            p.ctx.set_option(binding.OPT_L2_AHEAD_BYTES, bad)
+    p.close()
+
+
 @pytest.mark.parametrize("after", [2, 5, 9])
 def test_a_launch_refused_in_mid_window_leaves_the_next_call_clean(gpu, after):
     """A launch in the middle of a window fails (injected on the host: the library is told to refuse it, nothing
