@@ -78,109 +78,140 @@ __device__ __forceinline__ int swz(int dim) { return dim ^ (((dim >> 5) & 1) << 
 //    64 hf + 16 t + [0, 16)  (element 0 of instruction b -> + b, element 1 -> + 8 + b).
 
 // ---- a step of several tokens of one sequence: up to 64 query rows per KV head --------------------------
-// The query rows of a KV head (tokens x heads of the group) are cut into tiles of 16 (one m16n8k16 tile of rows),
-// and a CTA serves ONE tile: CTA (x, KV head, tile).  It takes the chunks x, x + gridDim.x, ... of the context and
-// carries the running (max, sum, output) of its 16 rows from chunk to chunk exactly as the one-token kernel does
-// (per-warp tiles in shared memory, no barrier in the chunk loop), so it leaves one partial result per CTA and the
-// merge kernel sees gridDim.x of them instead of one per chunk.  The cache is read once per tile (the re-reads
-// come from L2).  Every CTA that meets new positions forms their keys and values itself; the CTAs of tile 0 append
-// them to the cache.
-__global__ void __launch_bounds__(kThreads, 2)
+// The query rows of a KV head (tokens x heads of the group) are cut into T tiles of 16 (one m16n8k16 tile of rows
+// each).  One CTA per SM; CTA (x, KV head) takes the chunks x, x + gridDim.x, ... of the cached positions [0, pos)
+// and serves all T tiles, so the cache is read once.  Its warps form P teams of T warps: a team takes every P-th
+// sub-chunk of 16 positions of the CTA's chunks and streams it through a ring of its own in shared memory
+// (asynchronous 16-byte copies, issued by the team's threads together, run S - 1 sub-chunks ahead of the one being
+// computed; the only synchronisation in the loop is the team's own named barrier), and warp tt of the team applies
+// the staged keys and values to tile tt.  Keys and values reach the tensor-core instructions through ldmatrix (rows
+// padded to 272 bytes, so the eight rows of a matrix fall in different banks), the rotated, scaled queries stay in
+// registers as fp16 fragments, and so does the warp's running output tile (fp32), rescaled only when a row's
+// maximum moved.  The positions of this step itself are not read from the cache: the CTA that owns them (the one
+// after the last cached chunk, round robin) forms their keys and values from the QKV accumulators, appends them to
+// the cache, and its team 0 takes them as one more sub-chunk under the causal mask.  Every CTA leaves one partial
+// result (running max, sum, output) per row; the merge kernel sees gridDim.x of them.
+constexpr int kStageRow = kHeadDim * 2 + 16;             // bytes of a staged row of 128 halfs
+constexpr int kStageHalf = 16 * kStageRow;               // keys (or values) of 16 positions
+constexpr int kStageBytes = 2 * kStageHalf;              // keys, then values
+constexpr int kSubPerChunk = kChunk / 16;
+template <int T>
+struct TileShape {
+  static constexpr int kTeams = T == 1 ? 8 : (T == 4 ? 3 : 4);
+  static constexpr int kStagesOf = T == 1 ? 3 : (T == 4 ? 6 : 5);
+  static constexpr int kWarpsOf = kTeams * T;
+  static constexpr int kRing = kTeams * kStagesOf * kStageBytes;
+  static constexpr size_t kSmem = static_cast<size_t>(kRing) + static_cast<size_t>(16 * T) * kStageRow + static_cast<size_t>(2) * kMaxStepTok * kHeadDim * sizeof(__half);
+  static_assert(kWarpsOf * 16 * kRowPad * sizeof(float) <= kRing, "the warps' output tiles go over the ring");
+};
+
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+// The T warps of team `team` meet (T == 1: the warp's own lanes).
+template <int T>
+__device__ __forceinline__ void team_sync(int team) {
+  if (T == 1) __syncwarp();
+  else asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(32 * T) : "memory");
+}
+
+template <int T>
+__global__ void __launch_bounds__(TileShape<T>::kWarpsOf * 32, 1)
 attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
                  const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
-                 int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int n_chunks, int part_stride,
+                 int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int part_stride,
                  float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp, const L2Ahead ahead) {
+  using Shape = TileShape<T>;
+  constexpr int P = Shape::kTeams, S = Shape::kStagesOf, W = Shape::kWarpsOf, kThr = W * 32;
   pdl_trigger();
-  extern __shared__ __align__(16) float dyn_smem[];
-  __shared__ float s_m[kWarps][16], s_l[kWarps][16], s_f[kWarps][16], s_big[16];
+  extern __shared__ __align__(16) uint8_t tile_smem[];
+  __shared__ float s_m[W][16], s_l[W][16], s_f[W][16], s_big[T][16];
   __shared__ float s_inv[kMaxStepTok];
 
   const int group = n_q_heads / n_kv_heads;
-  const int n_rows = n_tok * group;                  // query rows of this KV head
-  const int row0 = 16 * static_cast<int>(blockIdx.z);       // first row of this CTA's tile
-  const int tile_rows = min(16, n_rows - row0);
-  float* s_o = dyn_smem;                                               // [kWarps][16][kRowPad]
-  float* q_s = s_o + kWarps * 16 * kRowPad;                            // [16][kRowPad] rotated queries of the tile
-  __half* new_k = reinterpret_cast<__half*>(q_s + 16 * kRowPad);       // [n_tok][128] keys of the new positions
-  __half* new_v = new_k + n_tok * kHeadDim;
+  const int n_rows = n_tok * group;                  // query rows of this KV head (at most 16 T)
+  float* s_o = reinterpret_cast<float*>(tile_smem);                       // [W][16][kRowPad], over the ring once the loop is done
+  __half* q_h = reinterpret_cast<__half*>(tile_smem + Shape::kRing);      // [16 T][kStageRow / 2] rotated, scaled queries
+  __half* new_k = q_h + 16 * T * (kStageRow / 2);                         // [n_tok][128] keys of the new positions
+  __half* new_v = new_k + kMaxStepTok * kHeadDim;
 
   const int kv = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int team = warp / T, tt = warp % T, tl = tt * 32 + lane;      // thread tl of 32 T in its team
   const int g = lane >> 2, t = lane & 3;
-  const int n_ctx = pos + n_tok;
+  const int gx = static_cast<int>(gridDim.x), bx = static_cast<int>(blockIdx.x);
+  const int n_old = (pos + kChunk - 1) / kChunk;     // chunks that hold cached positions
+  const bool owns_new = bx == n_old % gx;
 
-  uint4 kreg[2][4];      // [position block of 8][32-dim slice]
-  uint4 vreg[4][2];      // [k-slot position][64-dim half]
   const __half* kbase = k_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
   const __half* vbase = v_cache + static_cast<int64_t>(kv) * kv_capacity * kHeadDim;
-  // Entries below `limit` (at most pos) are loaded from the cache, the others are left zero.
-  auto load_old = [&](int wbase, int limit) {
-#pragma unroll
-    for (int pb = 0; pb < 2; ++pb) {
-      const int p = wbase + 8 * pb + g;
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        kreg[pb][j] = p < limit ? __ldcg(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(p) * kHeadDim + 32 * j + 8 * t)) : make_uint4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int pi = 0; pi < 4; ++pi) {
-      const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf)
-        vreg[pi][hf] = p < limit ? __ldcg(reinterpret_cast<const uint4*>(vbase + static_cast<int64_t>(p) * kHeadDim + 64 * hf + 8 * g)) : make_uint4(0, 0, 0, 0);
-    }
+  uint8_t* my_ring = tile_smem + team * (S * kStageBytes);
+  const uint32_t ring_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(my_ring));
+  // Sub-chunk i of this team is the (team + i P)-th sub-chunk of the CTA's chunks; rows at or above pos are zeros.
+  const int n_cta_sub = bx < n_old ? ((n_old - 1 - bx) / gx + 1) * kSubPerChunk : 0;
+  const int n_sub = n_cta_sub > team ? (n_cta_sub - team - 1) / P + 1 : 0;
+  auto wbase_of = [&](int i) {
+    const int j = team + i * P;
+    return (bx + (j / kSubPerChunk) * gx) * kChunk + (j % kSubPerChunk) * 16;
   };
-  // Entries of this step come from shared memory.
-  auto patch_new = [&](int wbase) {
-    if (wbase + 16 <= pos || wbase >= n_ctx) return;
+  auto issue = [&](int i) {
+    if (i < n_sub) {
+      const int wbase = wbase_of(i);
+      if (wbase < pos) {
+        const uint32_t dst = ring_u32 + (i % S) * kStageBytes;
 #pragma unroll
-    for (int pb = 0; pb < 2; ++pb) {
-      const int p = wbase + 8 * pb + g;
-      if (p >= pos && p < n_ctx) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) kreg[pb][j] = *reinterpret_cast<const uint4*>(new_k + (p - pos) * kHeadDim + 32 * j + 8 * t);
+        for (int u = 0; u < (256 + 32 * T - 1) / (32 * T); ++u) {
+          const int idx = tl + 32 * T * u;
+          if (256 % (32 * T) == 0 || idx < 256) {
+            const int r = idx >> 4, piece = idx & 15;
+            const int p = wbase + r;
+            const uint32_t n = p < pos ? 16u : 0u;
+            const int64_t off = static_cast<int64_t>(p < pos ? p : 0) * kHeadDim + 8 * piece;
+            cp_async16_zfill(dst + r * kStageRow + 16 * piece, kbase + off, n);
+            cp_async16_zfill(dst + kStageHalf + r * kStageRow + 16 * piece, vbase + off, n);
+          }
+        }
       }
     }
-#pragma unroll
-    for (int pi = 0; pi < 4; ++pi) {
-      const int p = wbase + 2 * t + (pi & 1) + 8 * (pi >> 1);
-      if (p >= pos && p < n_ctx) {
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) vreg[pi][hf] = *reinterpret_cast<const uint4*>(new_v + (p - pos) * kHeadDim + 64 * hf + 8 * g);
-      }
-    }
+    cp_async_commit();
   };
-
-  int chunk = blockIdx.x;
+  // Cached positions below the watermark may be requested before the dependency wait; a sub-chunk that reaches above
+  // it, and all that follow it, after the wait.
   const int pre_limit = min(pos, stable_below);
-  load_old(chunk * kChunk + warp * 16, pre_limit);
+  int issued = 0;
+  while (issued < S - 1 && (issued >= n_sub || wbase_of(issued) + 16 <= pre_limit || wbase_of(issued) >= pos)) issue(issued++);
   pdl_wait();
   stamp_begin(stamp);
-  if (threadIdx.x == 0) l2_ahead(ahead, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), gridDim.x * gridDim.y * gridDim.z);
-  if (pre_limit < pos && chunk * kChunk + warp * 16 + 16 > pre_limit) load_old(chunk * kChunk + warp * 16, pos);
+  if (threadIdx.x == 0) l2_ahead(ahead, blockIdx.x + gridDim.x * blockIdx.y, gridDim.x * gridDim.y);
+  while (issued < S - 1) issue(issued++);
 
-  // ---- finish the QKV product for this tile.  Items: one rotation pair of a query row of the tile, and for a CTA
-  //      that meets new positions also one pair of each new key and value.
-  const int c_lo = pos / kChunk, c_hi = (n_ctx - 1) / kChunk;
-  const int gx = static_cast<int>(gridDim.x);
-  const bool meets_new = c_lo % gx == static_cast<int>(blockIdx.x) || c_hi % gx == static_cast<int>(blockIdx.x) ||
-                         (c_hi - c_lo >= 2);      // more than two chunks of new positions cannot happen (n_tok <= 8 < 128)
-  const bool appends = meets_new && blockIdx.z == 0;
-  const int n_q_items = tile_rows * (kHeadDim / 2);
-  const int n_items = n_q_items + (meets_new ? 2 * n_tok * (kHeadDim / 2) : 0);      // at most 1024 + 1024
-  constexpr int kTrip = 4;
-  for (int trip = 0; trip * kTrip * kThreads < n_items; ++trip) {      // same trip count for every thread
-    const int base = trip * kTrip * kThreads + threadIdx.x;
+  // ---- finish the QKV product for this KV head.  Items: one rotation pair of a query row, and for the CTA that owns
+  //      the new positions also one pair of each new key and value.
+  const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
+  const int n_q_items = n_rows * (kHeadDim / 2);
+  const int n_items = n_q_items + (owns_new ? 2 * n_tok * (kHeadDim / 2) : 0);      // at most 4096 + 1024
+  constexpr int kTrip = 8;
+  for (int trip = 0; trip * kTrip * kThr < n_items; ++trip) {      // same trip count for every thread
+    const int base = trip * kTrip * kThr + threadIdx.x;
     acc_t ra[kTrip], rb[kTrip];
     float2 cs[kTrip];
 #pragma unroll
     for (int u = 0; u < kTrip; ++u) {
-      const int idx = base + u * kThreads;
+      const int idx = base + u * kThr;
       if (idx < n_items) {
         int tok, rowbase;
         const int i = idx % (kHeadDim / 2);
         if (idx < n_q_items) {
-          const int r = row0 + idx / (kHeadDim / 2);
+          const int r = idx / (kHeadDim / 2);
           tok = r / group;
           rowbase = (kv * group + r % group) * kHeadDim;
         } else {
@@ -204,16 +235,16 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     }
 #pragma unroll
     for (int u = 0; u < kTrip; ++u) {
-      const int idx = base + u * kThreads;
+      const int idx = base + u * kThr;
       if (idx < n_items) {
         const int i = idx % (kHeadDim / 2);
         const int a = rope_mode == 0 ? i : 2 * i, b = rope_mode == 0 ? i + kHeadDim / 2 : 2 * i + 1;
         if (idx < n_q_items) {
-          const int rl = idx / (kHeadDim / 2);      // row inside the tile
-          const float inv = s_inv[(row0 + rl) / group];
+          const int r = idx / (kHeadDim / 2);
+          const float inv = s_inv[r / group];
           const float x = acc_value(ra[u]) * inv, y = acc_value(rb[u]) * inv;
-          q_s[rl * kRowPad + swz(a)] = x * cs[u].x - y * cs[u].y;
-          q_s[rl * kRowPad + swz(b)] = y * cs[u].x + x * cs[u].y;
+          q_h[r * (kStageRow / 2) + a] = __float2half_rn((x * cs[u].x - y * cs[u].y) * scale);
+          q_h[r * (kStageRow / 2) + b] = __float2half_rn((y * cs[u].x + x * cs[u].y) * scale);
         } else {
           const int j = (idx - n_q_items) / (kHeadDim / 2);
           const int tok = j % n_tok;
@@ -225,66 +256,51 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
           __half* sm = (is_v ? new_v : new_k) + tok * kHeadDim;
           sm[a] = ha;
           sm[b] = hb;
-          const int p = pos + tok;
-          if (appends && (p / kChunk) % gx == static_cast<int>(blockIdx.x)) {      // one CTA of tile 0 owns each new position
-            __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + p) * kHeadDim;
-            gd[a] = ha;
-            gd[b] = hb;
-          }
+          __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + pos + tok) * kHeadDim;
+          gd[a] = ha;
+          gd[b] = hb;
         }
       }
     }
   }
   __syncthreads();
 
-  const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
-  // rows g (lo) and g + 8 (hi) of the tile
+  // rows g (lo) and g + 8 (hi) of this warp's tile; a dead row has token -1 and zero queries
+  const int row0 = 16 * tt;
+  const int tile_rows = max(0, min(16, n_rows - row0));
   int row_tok[2];
-  const float* qrow[2];
+  uint32_t qa[8][4];      // A fragments of the scaled queries: k step ks covers head dims 16 ks .. 16 ks + 15
 #pragma unroll
   for (int hr = 0; hr < 2; ++hr) {
     const int rl = g + 8 * hr;
     const bool live = rl < tile_rows;
     row_tok[hr] = live ? (row0 + rl) / group : -1;
-    qrow[hr] = q_s + (live ? rl : 0) * kRowPad;
-  }
-  float* so_lo = s_o + (warp * 16 + g) * kRowPad;
-  float* so_hi = so_lo + 8 * kRowPad;
+    const __half* qrow = q_h + (live ? row0 + rl : 0) * (kStageRow / 2);
 #pragma unroll
-  for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      *reinterpret_cast<float4*>(so_lo + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
-      *reinterpret_cast<float4*>(so_hi + swz(64 * hf + 16 * t + 4 * q)) = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][hr] = live ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * t) : 0u;
+      qa[ks][2 + hr] = live ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * t) : 0u;
     }
+  }
+  float o[16][4];      // output tile: o[nb] holds head dims 8 nb + 2 t, + 1 of rows g (elements 0, 1) and g + 8 (2, 3)
+#pragma unroll
+  for (int nb = 0; nb < 16; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};      // of rows g and g + 8, the same in the four lanes of a quad
-  for (bool first = true; chunk < n_chunks; chunk += gridDim.x, first = false) {
-    const int wbase = chunk * kChunk + warp * 16;
-    if (!first) load_old(wbase, pos);
-    patch_new(wbase);
+
+  // One sub-chunk of 16 positions staged at `stage` (shared-memory address); position wbase + c is visible to row hr
+  // when it is at most last[hr].
+  auto process = [&](uint32_t stage, int wbase, const int (&last)[2]) {
     float sc[2][4];
 #pragma unroll
     for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
+    // S = Q K^T: matrices (positions 0-7 | 8-15) x (dims 16 ks .. + 7 | + 8 .. + 15)
+    const uint32_t k_addr = stage + ((lane & 7) + 8 * (lane >> 4)) * kStageRow + 16 * ((lane >> 3) & 1);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t qa[2][4];
-#pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-        if (row_tok[hr] >= 0) {
-          a = *reinterpret_cast<const float4*>(qrow[hr] + swz(32 * j + 8 * t));
-          b = *reinterpret_cast<const float4*>(qrow[hr] + swz(32 * j + 8 * t) + 4);
-        }
-        qa[0][hr] = pack_h2(a.x * scale, a.y * scale);
-        qa[0][2 + hr] = pack_h2(a.z * scale, a.w * scale);
-        qa[1][hr] = pack_h2(b.x * scale, b.y * scale);
-        qa[1][2 + hr] = pack_h2(b.z * scale, b.w * scale);
-      }
-#pragma unroll
-      for (int pb = 0; pb < 2; ++pb) {
-        mma_f16(sc[pb], qa[0][0], qa[0][1], qa[0][2], qa[0][3], kreg[pb][j].x, kreg[pb][j].y);
-        mma_f16(sc[pb], qa[1][0], qa[1][1], qa[1][2], qa[1][3], kreg[pb][j].z, kreg[pb][j].w);
-      }
+    for (int ks = 0; ks < 8; ++ks) {
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4(k_addr + 32 * ks, b0, b1, b2, b3);
+      mma_f16(sc[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+      mma_f16(sc[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
     }
     // ---- mask, row maxima, rescaling factors, exponentials
     float mx[2] = {-INFINITY, -INFINITY};
@@ -294,8 +310,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
       for (int e = 0; e < 4; ++e) {
         const int hr = e >> 1;
         const int p = wbase + 8 * pb + 2 * t + (e & 1);
-        const bool ok = row_tok[hr] >= 0 && p <= pos + row_tok[hr];
-        sc[pb][e] = ok ? sc[pb][e] : -INFINITY;
+        sc[pb][e] = p <= last[hr] ? sc[pb][e] : -INFINITY;
         mx[hr] = fmaxf(mx[hr], sc[pb][e]);
       }
     float alpha[2], lsum[2], m_new[2];
@@ -307,7 +322,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
       alpha[hr] = m_run[hr] > -INFINITY ? expf(m_run[hr] - m_new[hr]) : 1.0f;      // nothing accumulated yet: the tile is zero
       lsum[hr] = 0.f;
     }
-    uint32_t pa[4];
+    uint32_t pa[4];      // A fragment of P: rows g, g + 8 x positions 2t, 2t+1 (first block of 8) and 8 + 2t, + 1
 #pragma unroll
     for (int pb = 0; pb < 2; ++pb) {
       float pv[4];
@@ -317,8 +332,8 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
         pv[e] = m_new[hr] > -INFINITY ? expf(sc[pb][e] - m_new[hr]) : 0.f;
         lsum[hr] += pv[e];
       }
-      pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g,   k slots of this block
-      pa[2 * pb + 1] = pack_h2(pv[2], pv[3]);    // row g+8
+      pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g
+      pa[2 * pb + 1] = pack_h2(pv[2], pv[3]);    // row g + 8
     }
 #pragma unroll
     for (int hr = 0; hr < 2; ++hr) {
@@ -327,39 +342,51 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
       l_run[hr] = l_run[hr] * alpha[hr] + lsum[hr];
       m_run[hr] = m_new[hr];
     }
-    // ---- O = P V, added to the warp's own tile: per 64-dim half eight instructions of 8 head dims each
+    if (!__all_sync(0xffffffffu, alpha[0] == 1.0f && alpha[1] == 1.0f)) {      // some row's maximum moved
 #pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll
-      for (int bh = 0; bh < 2; ++bh) {      // instructions 4 bh .. 4 bh + 3 of this half
-        float oc[4][4];
-#pragma unroll
-        for (int bb = 0; bb < 4; ++bb) {
-          const int b = 4 * bh + bb, j = b >> 1;
-          const uint32_t sel = (b & 1) ? 0x7632u : 0x5410u;
-          const uint32_t* v0 = reinterpret_cast<const uint32_t*>(&vreg[0][hf]);
-          const uint32_t* v1 = reinterpret_cast<const uint32_t*>(&vreg[1][hf]);
-          const uint32_t* v2 = reinterpret_cast<const uint32_t*>(&vreg[2][hf]);
-          const uint32_t* v3 = reinterpret_cast<const uint32_t*>(&vreg[3][hf]);
-          const uint32_t b0 = __byte_perm(v0[j], v1[j], sel);
-          const uint32_t b1 = __byte_perm(v2[j], v3[j], sel);
-          oc[bb][0] = oc[bb][1] = oc[bb][2] = oc[bb][3] = 0.f;
-          mma_f16(oc[bb], pa[0], pa[1], pa[2], pa[3], b0, b1);
-        }
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int col = swz(64 * hf + 16 * t + 8 * e + 4 * bh);
-          float4* dlo = reinterpret_cast<float4*>(so_lo + col);
-          const float4 olo = *dlo;
-          *dlo = make_float4(fmaf(olo.x, alpha[0], oc[0][e]), fmaf(olo.y, alpha[0], oc[1][e]), fmaf(olo.z, alpha[0], oc[2][e]),
-                             fmaf(olo.w, alpha[0], oc[3][e]));
-          float4* dhi = reinterpret_cast<float4*>(so_hi + col);
-          const float4 ohi = *dhi;
-          *dhi = make_float4(fmaf(ohi.x, alpha[1], oc[0][2 + e]), fmaf(ohi.y, alpha[1], oc[1][2 + e]), fmaf(ohi.z, alpha[1], oc[2][2 + e]),
-                             fmaf(ohi.w, alpha[1], oc[3][2 + e]));
-        }
+      for (int nb = 0; nb < 16; ++nb) {
+        o[nb][0] *= alpha[0]; o[nb][1] *= alpha[0];
+        o[nb][2] *= alpha[1]; o[nb][3] *= alpha[1];
       }
     }
+    // ---- O += P V: transposed matrices (positions 0-7 | 8-15) x (dims 16 j .. + 7 | + 8 .. + 15)
+    const uint32_t v_addr = stage + kStageHalf + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kStageRow + 16 * (lane >> 4);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4_trans(v_addr + 32 * j, b0, b1, b2, b3);
+      mma_f16(o[2 * j], pa[0], pa[1], pa[2], pa[3], b0, b1);
+      mma_f16(o[2 * j + 1], pa[0], pa[1], pa[2], pa[3], b2, b3);
+    }
+  };
+
+  {
+    int last[2];
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) last[hr] = row_tok[hr] >= 0 ? pos - 1 : -1;      // every live row sees every cached position
+    for (int i = 0; i < n_sub; ++i) {
+      cp_async_wait<S - 2>();      // all but the newest S - 2 groups: sub-chunk i has landed (this thread's pieces)
+      team_sync<T>(team);          // ... and the team's; the stage of sub-chunk i - 1 is free
+      issue(i + S - 1);
+      const int wbase = wbase_of(i);
+      if (wbase < pos && tile_rows > 0) process(ring_u32 + (i % S) * kStageBytes, wbase, last);
+    }
+  }
+  cp_async_wait<0>();
+  if (owns_new && team == 0) {      // the positions of this step, zero rows behind them, in stage 0 of team 0's ring
+    team_sync<T>(team);
+    for (int idx = tl; idx < 256; idx += 32 * T) {
+      const int r = idx >> 4, piece = idx & 15;
+      const uint4 zero = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(my_ring + r * kStageRow + 16 * piece) = r < n_tok ? *reinterpret_cast<const uint4*>(new_k + r * kHeadDim + 8 * piece) : zero;
+      *reinterpret_cast<uint4*>(my_ring + kStageHalf + r * kStageRow + 16 * piece) =
+          r < n_tok ? *reinterpret_cast<const uint4*>(new_v + r * kHeadDim + 8 * piece) : zero;
+    }
+    team_sync<T>(team);
+    int last[2];
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) last[hr] = row_tok[hr] >= 0 ? pos + row_tok[hr] : -1;      // causal among the new positions
+    if (tile_rows > 0) process(ring_u32, pos, last);
   }
   if (t == 0) {
     s_m[warp][g] = m_run[0];
@@ -367,36 +394,42 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     s_l[warp][g] = l_run[0];
     s_l[warp][g + 8] = l_run[1];
   }
-  __syncthreads();
-  if (threadIdx.x < kWarps * 16) {
+  __syncthreads();      // every team is done with its ring: the tiles may go over it
+#pragma unroll
+  for (int nb = 0; nb < 16; ++nb) {
+    *reinterpret_cast<float2*>(s_o + (warp * 16 + g) * kRowPad + 8 * nb + 2 * t) = make_float2(o[nb][0], o[nb][1]);
+    *reinterpret_cast<float2*>(s_o + (warp * 16 + g + 8) * kRowPad + 8 * nb + 2 * t) = make_float2(o[nb][2], o[nb][3]);
+  }
+  if (threadIdx.x < W * 16) {      // weight of warp w's tile in the CTA's result for its row
     const int w = threadIdx.x >> 4, r = threadIdx.x & 15;
     float big = -INFINITY;
 #pragma unroll
-    for (int ww = 0; ww < kWarps; ++ww) big = fmaxf(big, s_m[ww][r]);
+    for (int pp = 0; pp < P; ++pp) big = fmaxf(big, s_m[pp * T + w % T][r]);
     const float mine = s_m[w][r];
     s_f[w][r] = mine > -INFINITY ? expf(mine - big) : 0.f;
-    if (w == 0) s_big[r] = big;
+    if (w < T) s_big[w][r] = big;
   }
   __syncthreads();
-  // thread (row, four head dims) adds up the eight warps' tiles: one partial result of the CTA, numbered by blockIdx.x
-  for (int idx = threadIdx.x; idx < tile_rows * (kHeadDim / 4); idx += kThreads) {
-    const int r = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
-    const int col = swz(d4);
+  // thread (row, four head dims) adds up the teams' tiles: one partial result of the CTA per row, numbered by blockIdx.x
+  for (int idx = threadIdx.x; idx < n_rows * (kHeadDim / 4); idx += kThr) {
+    const int rr = idx / (kHeadDim / 4), d4 = (idx % (kHeadDim / 4)) * 4;
+    const int tile = rr >> 4, r = rr & 15;
     float4 accum = make_float4(0.f, 0.f, 0.f, 0.f);
     float l = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
+    for (int pp = 0; pp < P; ++pp) {
+      const int w = pp * T + tile;
       const float f = s_f[w][r];
-      const float4 v = *reinterpret_cast<const float4*>(s_o + (w * 16 + r) * kRowPad + col);
+      const float4 v = *reinterpret_cast<const float4*>(s_o + (w * 16 + r) * kRowPad + d4);
       l += f * s_l[w][r];
       accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
     }
-    const int rr = row0 + r;
     const int tok = rr / group, head = kv * group + rr % group;
     const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * part_stride + blockIdx.x;
     *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
-    if (d4 == 0) ml_part[slot] = make_float2(s_big[r], l);
+    if (d4 == 0) ml_part[slot] = make_float2(s_big[tile][r], l);
   }
+  stamp_end(stamp);
 }
 
 // ---- at most eight query rows per KV head (one token per request), merge included ------------------
@@ -786,10 +819,6 @@ attn_merge_kernel(const float* __restrict__ o_part, const float2* __restrict__ m
   stamp_end(stamp);
 }
 
-size_t tile_smem_bytes(int n_tok) {
-  return static_cast<size_t>(kWarps * 16 + 16) * kRowPad * sizeof(float) + static_cast<size_t>(2) * n_tok * kHeadDim * sizeof(__half);
-}
-
 constexpr size_t kOneSmemBytes = static_cast<size_t>(kWarps * 8 + 8) * kRowPad * sizeof(float) + 2 * kHeadDim * sizeof(__half);
 static_assert(8 * kMaxParts <= kWarps * 8 * kRowPad, "the merge weights reuse the tiles");
 
@@ -813,9 +842,15 @@ static int configure_kernels() {
   static bool configured[kMaxDevices] = {};
   int dev = -1;
   if (first_launch_on_device(configured, &dev)) {
-    cudaError_t e0 = cudaFuncSetAttribute(attn_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(tile_smem_bytes(kMaxStepTok)));
-    if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_tile_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaError_t e0 = cudaSuccess;
+    auto configure_tile = [&](auto kernel, size_t bytes) {
+      if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+      if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    };
+    configure_tile(attn_tile_kernel<1>, TileShape<1>::kSmem);
+    configure_tile(attn_tile_kernel<2>, TileShape<2>::kSmem);
+    configure_tile(attn_tile_kernel<3>, TileShape<3>::kSmem);
+    configure_tile(attn_tile_kernel<4>, TileShape<4>::kSmem);
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kOneSmemBytes));
     if (e0 == cudaSuccess) e0 = cudaFuncSetAttribute(attn_one_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e0 != cudaSuccess) return cuda_rc(e0);
@@ -850,14 +885,20 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
                    scr.ml_part, static_cast<int>(grid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
     return e == cudaSuccess ? 2 : cuda_rc(e);
   }
-  // several tokens: one CTA per (slot of chunks, KV head, tile of 16 query rows); about one wave of CTAs in all
+  // several tokens: one CTA per (slot of chunks, KV head), one CTA per SM, all tiles of 16 query rows in the CTA
   const int n_tiles = (n_rows + 15) / 16;
-  const int per_tile = std::min(kMaxParts, std::max(1, 2 * sm_count / (n_kv_heads * n_tiles)));
-  dim3 tgrid(std::min(n_chunks, per_tile), n_kv_heads, n_tiles);
-  cudaError_t e = launch_pdl(attn_tile_kernel, tgrid, dim3(kThreads), tile_smem_bytes(n_tok), st, acc_qkv, mpad,
-                             static_cast<const float*>(ssq.data), ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache,
-                             kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part,
-                             scr.stamp, scr.ahead);
+  if (n_tiles > 4) return cuda_rc(cudaErrorInvalidValue);
+  const int slots = std::min(kMaxParts, std::max(1, sm_count / n_kv_heads));
+  dim3 tgrid(std::min(n_chunks, slots), n_kv_heads);
+  auto launch_tile = [&](auto kernel, int warps, size_t bytes) {
+    return launch_pdl(kernel, tgrid, dim3(warps * 32), bytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data), ssq.n_groups, inv_width,
+                      ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok,
+                      scr.max_chunks, scr.o_part, scr.ml_part, scr.stamp, scr.ahead);
+  };
+  cudaError_t e = n_tiles == 1   ? launch_tile(attn_tile_kernel<1>, TileShape<1>::kWarpsOf, TileShape<1>::kSmem)
+                  : n_tiles == 2 ? launch_tile(attn_tile_kernel<2>, TileShape<2>::kWarpsOf, TileShape<2>::kSmem)
+                  : n_tiles == 3 ? launch_tile(attn_tile_kernel<3>, TileShape<3>::kWarpsOf, TileShape<3>::kSmem)
+                                 : launch_tile(attn_tile_kernel<4>, TileShape<4>::kWarpsOf, TileShape<4>::kSmem);
   if (e != cudaSuccess) return cuda_rc(e);
   e = launch_pdl(attn_merge_kernel, dim3(n_tok * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * tgrid.x) * sizeof(float), st,
                  scr.o_part, scr.ml_part, static_cast<int>(tgrid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
