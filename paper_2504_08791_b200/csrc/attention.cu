@@ -129,10 +129,21 @@ __global__ void __launch_bounds__(TileShape<T>::kWarpsOf * 32, 1)
 attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
                  const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
                  int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int part_stride,
-                 float* __restrict__ o_part, float2* __restrict__ ml_part, const Stamp stamp, const L2Ahead ahead) {
+                 float* __restrict__ o_part, float2* __restrict__ ml_part, const AttnSeqs seqs, const Stamp stamp, const L2Ahead ahead) {
   using Shape = TileShape<T>;
   constexpr int P = Shape::kTeams, S = Shape::kStagesOf, W = Shape::kWarpsOf, kThr = W * 32;
   pdl_trigger();
+  int row_base = 0;                 // first output row (request * heads) of this CTA's request
+  if (seqs.n > 0) {                 // one request per blockIdx.z, one token each: its own cache and position
+    const int tq = blockIdx.z;
+    k_cache = seqs.k[tq];
+    v_cache = seqs.v[tq];
+    pos = seqs.pos[tq];
+    acc += tq * mpad;
+    ssq += tq * kMaxStatBlocks;
+    rope_tab += tq * (kHeadDim / 2);
+    row_base = tq * n_q_heads;
+  }
   extern __shared__ __align__(16) uint8_t tile_smem[];
   __shared__ float s_m[W][16], s_l[W][16], s_f[W][16], s_big[T][16];
   __shared__ float s_inv[kMaxStepTok];
@@ -163,21 +174,23 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     const int j = team + i * P;
     return (bx + (j / kSubPerChunk) * gx) * kChunk + (j % kSubPerChunk) * 16;
   };
+  // This thread's pieces of a sub-chunk: 16 bytes number tl % 16 of the rows tl / 16 + 2 T u.
+  const int piece = tl & 15, r_first = tl >> 4;
   auto issue = [&](int i) {
     if (i < n_sub) {
       const int wbase = wbase_of(i);
       if (wbase < pos) {
-        const uint32_t dst = ring_u32 + (i % S) * kStageBytes;
+        const uint32_t dst = ring_u32 + (i % S) * kStageBytes + r_first * kStageRow + 16 * piece;
+        const int64_t off = static_cast<int64_t>(wbase + r_first) * kHeadDim + 8 * piece;
+        const bool whole = wbase + 16 <= pos;
 #pragma unroll
-        for (int u = 0; u < (256 + 32 * T - 1) / (32 * T); ++u) {
-          const int idx = tl + 32 * T * u;
-          if (256 % (32 * T) == 0 || idx < 256) {
-            const int r = idx >> 4, piece = idx & 15;
-            const int p = wbase + r;
-            const uint32_t n = p < pos ? 16u : 0u;
-            const int64_t off = static_cast<int64_t>(p < pos ? p : 0) * kHeadDim + 8 * piece;
-            cp_async16_zfill(dst + r * kStageRow + 16 * piece, kbase + off, n);
-            cp_async16_zfill(dst + kStageHalf + r * kStageRow + 16 * piece, vbase + off, n);
+        for (int u = 0; u < (16 + 2 * T - 1) / (2 * T); ++u) {
+          const int r = r_first + 2 * T * u;
+          if (16 % (2 * T) == 0 || r < 16) {
+            const bool in = whole || wbase + r < pos;
+            const int64_t src = in ? off + u * (2 * T * kHeadDim) : 0;      // a row at or above pos: nothing is read, zeros are written
+            cp_async16_zfill(dst + u * (2 * T * kStageRow), kbase + src, in ? 16u : 0u);
+            cp_async16_zfill(dst + kStageHalf + u * (2 * T * kStageRow), vbase + src, in ? 16u : 0u);
           }
         }
       }
@@ -191,7 +204,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
   while (issued < S - 1 && (issued >= n_sub || wbase_of(issued) + 16 <= pre_limit || wbase_of(issued) >= pos)) issue(issued++);
   pdl_wait();
   stamp_begin(stamp);
-  if (threadIdx.x == 0) l2_ahead(ahead, blockIdx.x + gridDim.x * blockIdx.y, gridDim.x * gridDim.y);
+  if (threadIdx.x == 0) l2_ahead(ahead, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), gridDim.x * gridDim.y * gridDim.z);
   while (issued < S - 1) issue(issued++);
 
   // ---- finish the QKV product for this KV head.  Items: one rotation pair of a query row, and for the CTA that owns
@@ -265,7 +278,8 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
   }
   __syncthreads();
 
-  // rows g (lo) and g + 8 (hi) of this warp's tile; a dead row has token -1 and zero queries
+  // rows g (lo) and g + 8 (hi) of this warp's tile; a dead row (beyond the last query row) has zero queries and is
+  // computed like any other: its result is finite and never written
   const int row0 = 16 * tt;
   const int tile_rows = max(0, min(16, n_rows - row0));
   int row_tok[2];
@@ -289,7 +303,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
 
   // One sub-chunk of 16 positions staged at `stage` (shared-memory address); position wbase + c is visible to row hr
   // when it is at most last[hr].
-  auto process = [&](uint32_t stage, int wbase, const int (&last)[2]) {
+  auto process = [&](uint32_t stage, int wbase, const int (&last)[2], bool masked) {
     float sc[2][4];
 #pragma unroll
     for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
@@ -304,22 +318,26 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     }
     // ---- mask, row maxima, rescaling factors, exponentials
     float mx[2] = {-INFINITY, -INFINITY};
+    if (masked) {      // (the same for the whole warp)
+#pragma unroll
+      for (int pb = 0; pb < 2; ++pb)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int p = wbase + 8 * pb + 2 * t + (e & 1);
+          sc[pb][e] = p <= last[e >> 1] ? sc[pb][e] : -INFINITY;
+        }
+    }
 #pragma unroll
     for (int pb = 0; pb < 2; ++pb)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int hr = e >> 1;
-        const int p = wbase + 8 * pb + 2 * t + (e & 1);
-        sc[pb][e] = p <= last[hr] ? sc[pb][e] : -INFINITY;
-        mx[hr] = fmaxf(mx[hr], sc[pb][e]);
-      }
+      for (int e = 0; e < 4; ++e) mx[e >> 1] = fmaxf(mx[e >> 1], sc[pb][e]);
     float alpha[2], lsum[2], m_new[2];
 #pragma unroll
     for (int hr = 0; hr < 2; ++hr) {
       mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
       mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
       m_new[hr] = fmaxf(m_run[hr], mx[hr]);
-      alpha[hr] = m_run[hr] > -INFINITY ? expf(m_run[hr] - m_new[hr]) : 1.0f;      // nothing accumulated yet: the tile is zero
+      alpha[hr] = m_run[hr] > -INFINITY ? __expf(m_run[hr] - m_new[hr]) : 1.0f;      // nothing accumulated yet: the tile is zero
       lsum[hr] = 0.f;
     }
     uint32_t pa[4];      // A fragment of P: rows g, g + 8 x positions 2t, 2t+1 (first block of 8) and 8 + 2t, + 1
@@ -329,7 +347,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int hr = e >> 1;
-        pv[e] = m_new[hr] > -INFINITY ? expf(sc[pb][e] - m_new[hr]) : 0.f;
+        pv[e] = m_new[hr] > -INFINITY ? __expf(sc[pb][e] - m_new[hr]) : 0.f;
         lsum[hr] += pv[e];
       }
       pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g
@@ -363,13 +381,13 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
   {
     int last[2];
 #pragma unroll
-    for (int hr = 0; hr < 2; ++hr) last[hr] = row_tok[hr] >= 0 ? pos - 1 : -1;      // every live row sees every cached position
+    for (int hr = 0; hr < 2; ++hr) last[hr] = pos - 1;      // every row sees every cached position
     for (int i = 0; i < n_sub; ++i) {
       cp_async_wait<S - 2>();      // all but the newest S - 2 groups: sub-chunk i has landed (this thread's pieces)
       team_sync<T>(team);          // ... and the team's; the stage of sub-chunk i - 1 is free
       issue(i + S - 1);
       const int wbase = wbase_of(i);
-      if (wbase < pos && tile_rows > 0) process(ring_u32 + (i % S) * kStageBytes, wbase, last);
+      if (wbase < pos) process(ring_u32 + (i % S) * kStageBytes, wbase, last, wbase + 16 > pos);
     }
   }
   cp_async_wait<0>();
@@ -385,8 +403,8 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     team_sync<T>(team);
     int last[2];
 #pragma unroll
-    for (int hr = 0; hr < 2; ++hr) last[hr] = row_tok[hr] >= 0 ? pos + row_tok[hr] : -1;      // causal among the new positions
-    if (tile_rows > 0) process(ring_u32, pos, last);
+    for (int hr = 0; hr < 2; ++hr) last[hr] = pos + max(row_tok[hr], 0);      // causal among the new positions
+    process(ring_u32, pos, last, true);
   }
   if (t == 0) {
     s_m[warp][g] = m_run[0];
@@ -425,7 +443,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
       accum.x += f * v.x; accum.y += f * v.y; accum.z += f * v.z; accum.w += f * v.w;
     }
     const int tok = rr / group, head = kv * group + rr % group;
-    const int64_t slot = (static_cast<int64_t>(tok) * n_q_heads + head) * part_stride + blockIdx.x;
+    const int64_t slot = (static_cast<int64_t>(row_base) + static_cast<int64_t>(tok) * n_q_heads + head) * part_stride + blockIdx.x;
     *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
     if (d4 == 0) ml_part[slot] = make_float2(s_big[tile][r], l);
   }
@@ -874,7 +892,11 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
   const int per_head = std::min(kMaxParts, std::max(1, 2 * sm_count / n_kv_heads));
   dim3 grid(std::min(n_chunks, per_head), n_kv_heads);
   const AttnSeqs none{};
-  if (n_tok == 1) {
+  // one token: up to about ten thousand positions the kernel that keeps its positions in registers (two CTAs per SM,
+  // everything requested before the dependency wait) is faster; beyond, the streaming kernel (measured: 10.9 against
+  // 14.3 us per layer at 4096 positions, 25.8 against 22.3 at 16384, 40.2 against 32.4 at 32768)
+  constexpr int kLongContextChunks = 80;
+  if (n_tok == 1 && n_chunks < kLongContextChunks) {
     int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;
     cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
                                ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads,
@@ -893,7 +915,7 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
   auto launch_tile = [&](auto kernel, int warps, size_t bytes) {
     return launch_pdl(kernel, tgrid, dim3(warps * 32), bytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data), ssq.n_groups, inv_width,
                       ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok,
-                      scr.max_chunks, scr.o_part, scr.ml_part, scr.stamp, scr.ahead);
+                      scr.max_chunks, scr.o_part, scr.ml_part, none, scr.stamp, scr.ahead);
   };
   cudaError_t e = n_tiles == 1   ? launch_tile(attn_tile_kernel<1>, TileShape<1>::kWarpsOf, TileShape<1>::kSmem)
                   : n_tiles == 2 ? launch_tile(attn_tile_kernel<2>, TileShape<2>::kWarpsOf, TileShape<2>::kSmem)
@@ -915,8 +937,22 @@ int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, 
   if (max_chunks > scr.max_chunks) return cuda_rc(cudaErrorInvalidValue);
   const int rc = configure_kernels();
   if (rc != 0) return rc;
-  // The whole launch should be about one wave of CTAs (two per SM): with many requests a CTA takes several chunks of
-  // its request and carries its running state from one to the next, instead of many waves of short-lived CTAs.
+  if (seqs.n >= 2) {
+    // several requests: the streaming kernel with one tile of query rows (the heads of the group), one CTA per SM in
+    // all; a CTA beyond its request's chunks leaves an empty partial result, which the merge gives no weight
+    const int slots = std::min(kMaxParts, std::max(1, sm_count / (n_kv_heads * seqs.n)));
+    dim3 tgrid(std::min(max_chunks, slots), n_kv_heads, seqs.n);
+    cudaError_t e = launch_pdl(attn_tile_kernel<1>, tgrid, dim3(TileShape<1>::kWarpsOf * 32), TileShape<1>::kSmem, st, acc_qkv, mpad,
+                               static_cast<const float*>(ssq.data), ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps,
+                               rope_tab, rope_mode, static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads, n_kv_heads,
+                               0, stable_below, 1, scr.max_chunks, scr.o_part, scr.ml_part, seqs, scr.stamp, scr.ahead);
+    if (e != cudaSuccess) return cuda_rc(e);
+    const AttnSeqs none{};
+    e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * tgrid.x) * sizeof(float), st, scr.o_part,
+                   scr.ml_part, static_cast<int>(tgrid.x), scr.max_chunks, n_q_heads, o, none, scr.stamp);
+    return e == cudaSuccess ? 2 : cuda_rc(e);
+  }
+  // a single request: the one-token kernel, about one wave of CTAs (two per SM)
   const int per_head = std::min(kMaxParts, std::max(1, 2 * sm_count / (n_kv_heads * seqs.n)));
   dim3 grid(std::min(max_chunks, per_head), n_kv_heads, seqs.n);      // CTAs beyond a request's own chunks leave at once
   int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;

@@ -119,6 +119,8 @@ def test_window_splits_are_bit_identical_on_the_gpu(gpu, splits, n_tok):
     (dict(rope_mode=1), 129, 6),                                            # ... on the multi-token kernels
     (dict(n_q_heads=2, n_kv_heads=2, hidden=256), 33, 1),                   # no grouping, one super-block column
     (dict(n_q_heads=8, n_kv_heads=1, hidden=1024), 200, 3),                 # one KV head for eight query heads
+    (dict(n_q_heads=8, n_kv_heads=1, hidden=1024), 250, 8),                 # ... 64 query rows: four tiles in one CTA
+    (dict(n_q_heads=8, n_kv_heads=1, hidden=1024), 256, 4),                 # the step's positions open a new chunk
     (dict(n_q_heads=10, n_kv_heads=2, hidden=1280, ffn=1280), 127, 1),      # five query heads per KV head, column groups of 5
     (dict(n_q_heads=10, n_kv_heads=2, hidden=1280, ffn=1280), 128, 7),
     (dict(n_q_heads=4, n_kv_heads=4, hidden=512, ffn=3328, vocab=1000), 0, 2),   # 13 super-block columns (prime), vocab not a multiple of 8
@@ -254,13 +256,16 @@ def test_sums_outside_the_accumulator_range_are_reported_once(gpu):
     p.close()
 
 
-@pytest.mark.parametrize("n_tok", [1, 3])
-def test_long_context_with_more_chunks_than_resident_ctas(gpu, n_tok):
-    """19,100 / 39,000 cached positions on a model with two KV heads: 150 / 305 chunks per head, more than the 148
-    CTAs per head that the grid gets, so CTAs take further chunks, and the merge sees more partial results than it
-    has threads."""
-    cfg = synth.model_config("tiny", kv_capacity=40000)
-    pos = 39000 if n_tok == 1 else 19100               # 305 chunks: three per CTA, carried from chunk to chunk
+@pytest.mark.parametrize("n_tok,pos,over", [
+    (1, 39000, {}),                                                  # streaming kernel, 305 chunks on 74 CTAs per KV head
+    (3, 19100, dict(n_kv_heads=1)),                                  # ... 150 chunks on 148 CTAs: more partial results than the merge has threads
+    (1, 9500, dict(n_q_heads=8, n_kv_heads=8, hidden=1024)),         # one-token kernel, 75 chunks on 37 CTAs per KV head: two or three per CTA
+])
+def test_long_context_with_more_chunks_than_resident_ctas(gpu, n_tok, pos, over):
+    """More chunks of cached positions than CTAs per KV head, so that a CTA takes further chunks and carries its
+    running state from one to the next, in both attention kernels, and a merge over more partial results than it has
+    threads."""
+    cfg = synth.model_config("tiny", kv_capacity=40000, **over)
     p = Pair(gpu, cfg, seed=43, n_prefill=pos)
     h0 = synth.activations(43, n_tok, cfg["hidden"])
     want = p.ref.forward_window(0, cfg["n_layers"], h0, pos)
