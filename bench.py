@@ -44,7 +44,7 @@ WORKLOADS = {
 SEEDS = {"70b": 3, "32b": 2, "8b": 1}
 # dram__bytes_read.sum + dram__bytes_write.sum over the four 70B-shaped layer matrices / their Q4_K bytes
 # (one ncu capture of gemv_partials_kernel<1>, profiles/gemv_partials_70b_matrices.md)
-NCU_TRAFFIC_RATIO = 489.9 / 481.3
+NCU_TRAFFIC_RATIO = (496.9 + 7.8 - 14.2) / 481.3      # read + written, without the bytes the O product asks ahead for gate/up
 
 
 def log(*a):

@@ -287,13 +287,15 @@ int prima_gemv_plan_destroy(prima_gemv_plan* plan);
  *   PRIMA_FMT_Q4_K  the 144-byte super-block described at the top (the calls below forward to the _q4k calls)
  * Matrices are row-major, cols a multiple of 256.  prima_dequant_fmt: n_blocks blocks (dev) -> fp32 (dev), the exact
  * value (no rounding is needed: it fits binary32).  prima_gemv_fmt: y[c][r] = sum_k W[r][k] x[c][k], 1 <= n_cols <= 4;
- * dev_w in its standard layout, read in place (nothing is allocated or re-tiled), at an even address; the activations
- * of all columns (4 bytes a value for FP16 matrices; for the block formats 16-bit integers with one fp32 step per 32
- * values, as in the Q4_K path, 2.625 bytes a value) plus two rows of the matrix must fit 200 KiB of shared memory
+ * dev_w in its standard layout, read in place (nothing is allocated or re-tiled), at an even address.  Shared
+ * memory must hold the activations of all columns (4 bytes a value for FP16 matrices; for the block formats 16-bit
+ * integers with one fp32 step per 32 values, as in the Q4_K path, 3 bytes a value with cols rounded up to 2048) plus
+ * two rows of the matrix (FP16) or the warps' copy rings (block formats: 35 KiB at least) within 200 KiB
  * (PRIMA_ERR_ARG otherwise, with a message in prima_fmt_last_error).  dev_w must lie in an allocation whose size is
  * a multiple of 16 bytes, as every cudaMalloc allocation is: rows are fetched in 16-byte pieces from the boundary at
- * or below their first byte.  Per row |y - y_ref| <= 1e-3 * sum |w x| (activation step <= 2^-15 of a block's largest
- * value, exact integer sums per group, fp32 accumulation over groups).  Queued on `stream`, no waiting. */
+ * or below their first byte to the boundary at or above their last.  Per row |y - y_ref| <= 1e-3 * sum |w x|
+ * (activation step <= 2^-15 of a block's largest value, exact integer sums per group, fp32 accumulation over
+ * groups).  Queued on `stream`, no waiting. */
 #define PRIMA_FMT_Q4_K 0
 #define PRIMA_FMT_Q6_K 1
 #define PRIMA_FMT_Q8_0 2

@@ -13,13 +13,15 @@
 // brought into shared memory with 16-byte asynchronous copies (the copy starts at the 16-byte boundary at or
 // below the row's first byte, since rows of these formats need not start on one), the next row is requested
 // before the current one is used, and the activations of all columns sit in shared memory as fp32 for the
-// whole kernel.  FP16 weights are multiplied in fp32.  For the two block formats the activations are held as in the
-// Q4_K kernels: 16-bit integers x_q = round(x / s_b) with one fp32 step s_b per block of 32, cut into a high and a
-// low signed byte, so that the sum over a group of weights is an exact integer from 4-way byte dot products
-// (Q8_0: q * x_q; Q6_K: v * x_q - 32 * sum(x_q), v the unsigned 6-bit value), scaled once per group by
-// d * s_b (* sc for Q6_K) in fp32.  A CTA takes several consecutive rows per iteration when rows are short (their
-// bytes are contiguous: one copy range), each row worked on by its own team of threads; the threads' sums are
-// added in a fixed order, so the result is the same from run to run.  Bound: HBM (0.82 / 1.06 / 2 bytes per weight).
+// whole kernel.  FP16 weights are multiplied in fp32 (one CTA per row, double-buffered 16-byte copies).  For the two
+// block formats the activations are held as in the Q4_K kernels: 16-bit integers x_q = round(x / s_b) with one fp32
+// step s_b per block of 32, cut into a high and a low signed byte, so that the sum over a group of weights is an exact
+// integer from 4-way byte dot products (Q8_0: q * x_q; Q6_K: v * x_q - 32 * sum(x_q), v the unsigned 6-bit value),
+// scaled once per group by d * s_b (* sc for Q6_K) in fp32.  Every CTA quantises the activations once into shared
+// memory; then every warp takes rows of its own and streams them in segments of 2048 weights through a ring of
+// 16-byte asynchronous copies of its own (no barrier between warps), a lane working on 64 weights of a segment; the
+// lanes' sums are added by shuffles, so the result is the same from run to run.
+// Bound: HBM (0.82 / 1.06 / 2 bytes per weight).
 #include <cstdio>
 
 #include "../../include/prima.h"
@@ -194,74 +196,100 @@ __device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {      // 
   asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-// Eight bytes at an even offset `a` of shared memory: three aligned words, shifted by 0 or 16 bits.
-__device__ __forceinline__ uint2 lds8_even(const uint8_t* smem, int a) {
+// N consecutive words starting at an even byte offset `a` of shared memory: N + 1 aligned words, shifted by 0 or 16 bits.
+template <int N>
+__device__ __forceinline__ void lds_even(const uint8_t* smem, int a, uint32_t (&out)[N]) {
   const uint32_t* p = reinterpret_cast<const uint32_t*>(smem + (a & ~3));
-  const uint32_t w0 = p[0], w1 = p[1], w2 = p[2], sh = (a & 2) * 8;
-  return make_uint2(__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh));
-}
-
-// The shared-memory image of one column of activations is cut into chunks of eight consecutive values; chunk j has
-// its eight high bytes at 8 j, its low bytes at P + 8 j and the pair (sum of its eight x_q, step of its block of 32
-// as fp32 bits) at 2 P + 8 j, P = cols rounded up to 1024.  For Q8_0 chunk j holds values 8 j ..; for Q6_K the chunk
-// of values 256 s + 128 n + 32 i + 8 o .. is j = 128 (s / 4) + 32 i + 8 (s % 4) + 4 n + o, so that the 32 lanes of a
-// warp (four super-blocks s, halves n, octets o) read 256 consecutive bytes at each i.
-template <int FMT>
-__device__ __forceinline__ int chunk_slot(int kc) {
-  if (FMT != PRIMA_FMT_Q6_K) return kc;
-  const int s = kc >> 5, n = (kc >> 4) & 1, i = (kc >> 2) & 3, o = kc & 3;
-  return 128 * (s >> 2) + 32 * i + 8 * (s & 3) + 4 * n + o;
-}
-
-template <int FMT, int NC>
-__device__ __forceinline__ void row_partial_q(const uint8_t* smem, int rowoff, int col_bytes, int padded, int cols, int tl, int tpr,
-                                              float (&acc)[NC]) {
-  if (FMT == PRIMA_FMT_Q8_0) {
-    // two threads per block of 32 weights, sixteen consecutive weights each
-    const int n_blk = cols >> 5, j = tl & 1;
-    for (int b = tl >> 1; b < n_blk; b += tpr >> 1) {
-      const int blk = rowoff + 34 * b;
-      const float d = half_bits_to_float(lds_u16(smem + blk));
-      const int a = blk + 2 + 16 * j;
-      const uint32_t* p = reinterpret_cast<const uint32_t*>(smem + (a & ~3));
-      const uint32_t sh = (a & 2) * 8, w0 = p[0], w1 = p[1], w2 = p[2], w3 = p[3], w4 = p[4];
-      const uint32_t q0 = __funnelshift_r(w0, w1, sh), q1 = __funnelshift_r(w1, w2, sh), q2 = __funnelshift_r(w2, w3, sh), q3 = __funnelshift_r(w3, w4, sh);
-      const int ch = 16 * (2 * b + j);
+  const uint32_t sh = (a & 2) * 8;
+  uint32_t w[N + 1];
 #pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        const uint8_t* xc = smem + c * col_bytes + ch;
-        const uint4 xh = *reinterpret_cast<const uint4*>(xc);
-        const uint4 xl = *reinterpret_cast<const uint4*>(xc + padded);
-        const float step = *reinterpret_cast<const float*>(xc + 2 * padded + 4);
-        const int h = dp4a_ss(q3, xh.w, dp4a_ss(q2, xh.z, dp4a_ss(q1, xh.y, dp4a_ss(q0, xh.x, 0))));
-        const int l = dp4a_ss(q3, xl.w, dp4a_ss(q2, xl.z, dp4a_ss(q1, xl.y, dp4a_ss(q0, xl.x, 0))));
-        acc[c] = fmaf(static_cast<float>(h * 256 + l), d * step, acc[c]);
+  for (int i = 0; i <= N; ++i) w[i] = p[i];
+#pragma unroll
+  for (int i = 0; i < N; ++i) out[i] = __funnelshift_r(w[i], w[i + 1], sh);
+}
+
+// A row is cut into segments of 2048 weights (8 Q6_K super-blocks, 1680 bytes; 64 Q8_0 blocks, 2176 bytes; the last
+// segment of a row may be shorter).  The shared-memory image of one column of activations is cut into pieces of 16
+// consecutive values: piece j has its 16 high bytes at 16 j, its low bytes at P + 16 j and two pairs (sum of eight
+// x_q, step of their block of 32 as fp32 bits) at 2 P + 16 j; P = cols rounded up to 2048.  The pieces of a segment
+// are ordered so that the 32 lanes of a warp read 512 consecutive bytes with every 16-byte load:
+//   Q8_0: lane = block b of 32 within the half segment; piece (b, first / second 16 values) -> 64 (b / 32) + 32 half + b % 32
+//   Q6_K: lane = (super-block s, half n, 16 positions h); piece of values 256 s + 128 n + 32 i + 16 h .. -> 32 i + 4 s + 2 n + h
+template <int FMT>
+__device__ __forceinline__ int piece_slot(int piece) {      // piece = index of 16 consecutive values within the row
+  const int seg = piece >> 7, in = piece & 127;
+  if (FMT == PRIMA_FMT_Q8_0) {
+    const int b = in >> 1, half = in & 1;
+    return 128 * seg + 64 * (b >> 5) + 32 * half + (b & 31);
+  }
+  const int s = in >> 4, n = (in >> 3) & 1, i = (in >> 1) & 3, h = in & 1;
+  return 128 * seg + 32 * i + 4 * s + 2 * n + h;
+}
+
+constexpr int kSegWeights = 2048;
+template <int FMT>
+struct SegShape {
+  static constexpr int kBytes = FMT == PRIMA_FMT_Q8_0 ? 64 * 34 : 8 * 210;      // a full segment
+  static constexpr int kBuf = kBytes + 32;                                      // + the bytes around an unaligned start and end
+  static constexpr int kUnit = FMT == PRIMA_FMT_Q8_0 ? 272 : 210;               // bytes of 256 weights
+};
+
+// One segment of one row, staged at shared-memory offset `seg` (its first byte): this lane's share of sum w x.
+template <int FMT, int NC>
+__device__ __forceinline__ void segment_partial(const uint8_t* smem, int seg, int n_units, int xseg, int col_bytes, int padded, int lane, float (&acc)[NC]) {
+  if (FMT == PRIMA_FMT_Q8_0) {
+    // lane = block within a half segment of 32 blocks (8 units of 256 weights = 64 blocks)
+#pragma unroll
+    for (int hs = 0; hs < 2; ++hs) {
+      const int b = 32 * hs + lane;
+      if (b < 8 * n_units) {
+        const int blk = seg + 34 * b;
+        const float d = half_bits_to_float(lds_u16(smem + blk));
+        uint32_t q[8];
+        lds_even<8>(smem, blk + 2, q);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          const uint8_t* xc = smem + c * col_bytes + xseg + 1024 * hs + 16 * lane;
+          const uint4 h0 = *reinterpret_cast<const uint4*>(xc), h1 = *reinterpret_cast<const uint4*>(xc + 512);
+          const uint4 l0 = *reinterpret_cast<const uint4*>(xc + padded), l1 = *reinterpret_cast<const uint4*>(xc + padded + 512);
+          const float step = *reinterpret_cast<const float*>(xc + 2 * padded + 4);
+          int h = dp4a_ss(q[3], h0.w, dp4a_ss(q[2], h0.z, dp4a_ss(q[1], h0.y, dp4a_ss(q[0], h0.x, 0))));
+          h = dp4a_ss(q[7], h1.w, dp4a_ss(q[6], h1.z, dp4a_ss(q[5], h1.y, dp4a_ss(q[4], h1.x, h))));
+          int l = dp4a_ss(q[3], l0.w, dp4a_ss(q[2], l0.z, dp4a_ss(q[1], l0.y, dp4a_ss(q[0], l0.x, 0))));
+          l = dp4a_ss(q[7], l1.w, dp4a_ss(q[6], l1.z, dp4a_ss(q[5], l1.y, dp4a_ss(q[4], l1.x, l))));
+          acc[c] = fmaf(static_cast<float>(h * 256 + l), d * step, acc[c]);
+        }
       }
     }
   } else {
-    // eight threads per super-block: thread = (half n, eight consecutive positions 8 o .. 8 o + 7), 32 weights each
-    const int n_sb = cols >> 8, n = (tl >> 2) & 1, o = tl & 3;
-    for (int s = tl >> 3; s < n_sb; s += tpr >> 3) {
-      const int sb = rowoff + 210 * s;
-      const uint2 qa = lds8_even(smem, sb + 64 * n + 8 * o), qb = lds8_even(smem, sb + 64 * n + 32 + 8 * o);
-      const uint2 qh = lds8_even(smem, sb + 128 + 32 * n + 8 * o);
+    // lane = (super-block s of the segment, half n, 16 positions 16 h ..): 64 weights
+    const int s = lane >> 2, n = (lane >> 1) & 1, h16 = lane & 1;
+    if (s < n_units) {
+      const int sb = seg + 210 * s;
+      uint32_t qa[4], qb[4], qh[4];
+      lds_even<4>(smem, sb + 64 * n + 16 * h16, qa);
+      lds_even<4>(smem, sb + 64 * n + 32 + 16 * h16, qb);
+      lds_even<4>(smem, sb + 128 + 32 * n + 16 * h16, qh);
       const float d = half_bits_to_float(lds_u16(smem + sb + 208));
-      const int8_t* scp = reinterpret_cast<const int8_t*>(smem + sb + 192 + 8 * n + (o >> 1));
-      const int ch0 = 8 * (128 * (s >> 2) + 8 * (s & 3) + 4 * n + o);
+      const int8_t* scp = reinterpret_cast<const int8_t*>(smem + sb + 192 + 8 * n + h16);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint2 src = (i & 1) ? qb : qa;
-        const uint32_t v0 = (i < 2 ? (src.x & 0x0f0f0f0fu) : ((src.x >> 4) & 0x0f0f0f0fu)) | (((qh.x >> (2 * i)) & 0x03030303u) << 4);
-        const uint32_t v1 = (i < 2 ? (src.y & 0x0f0f0f0fu) : ((src.y >> 4) & 0x0f0f0f0fu)) | (((qh.y >> (2 * i)) & 0x03030303u) << 4);
+        uint32_t v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t src = (i & 1) ? qb[k] : qa[k];
+          v[k] = (i < 2 ? (src & 0x0f0f0f0fu) : ((src >> 4) & 0x0f0f0f0fu)) | (((qh[k] >> (2 * i)) & 0x03030303u) << 4);
+        }
         const float dsc = d * static_cast<float>(scp[2 * i]);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
-          const uint8_t* xc = smem + c * col_bytes + ch0 + 256 * i;
-          const uint2 xh = *reinterpret_cast<const uint2*>(xc);
-          const uint2 xl = *reinterpret_cast<const uint2*>(xc + padded);
-          const int2 ss = *reinterpret_cast<const int2*>(xc + 2 * padded);
-          const int h = dp4a_us(v1, xh.y, dp4a_us(v0, xh.x, 0)), l = dp4a_us(v1, xl.y, dp4a_us(v0, xl.x, 0));
-          acc[c] = fmaf(static_cast<float>(h * 256 + l - 32 * ss.x), dsc * __int_as_float(ss.y), acc[c]);
+          const uint8_t* xc = smem + c * col_bytes + xseg + 512 * i + 16 * lane;
+          const uint4 xh = *reinterpret_cast<const uint4*>(xc);
+          const uint4 xl = *reinterpret_cast<const uint4*>(xc + padded);
+          const int4 ss = *reinterpret_cast<const int4*>(xc + 2 * padded);      // (sum, step, sum, step): one block of 32, one step
+          const int hh = dp4a_us(v[3], xh.w, dp4a_us(v[2], xh.z, dp4a_us(v[1], xh.y, dp4a_us(v[0], xh.x, 0))));
+          const int ll = dp4a_us(v[3], xl.w, dp4a_us(v[2], xl.z, dp4a_us(v[1], xl.y, dp4a_us(v[0], xl.x, 0))));
+          acc[c] = fmaf(static_cast<float>(hh * 256 + ll - 32 * (ss.x + ss.z)), dsc * __int_as_float(ss.y), acc[c]);
         }
       }
     }
@@ -270,31 +298,44 @@ __device__ __forceinline__ void row_partial_q(const uint8_t* smem, int rowoff, i
 
 constexpr int kMaxQThreads = 512;
 
-// rows_per_it (1, 2, 4 or 8) consecutive rows per iteration, blockDim.x / rows_per_it threads per row; a ring of
-// `depth` (2..6) buffers of buf_bytes each holds the rows on their way in.
+// Every warp takes rows of its own (global warp number, then every total-warps-th row) and streams their segments
+// through a ring of `depth` buffers of its own in shared memory: no barrier between warps after the prologue.
 template <int FMT, int NC>
-__global__ void __launch_bounds__(kMaxQThreads) gemv_fmtq_kernel(const uint8_t* __restrict__ w, int64_t rows, int cols, int row_bytes, int rows_per_it,
-                                                                  int buf_bytes, int depth, const float* __restrict__ x, float* __restrict__ y) {
+__global__ void __launch_bounds__(kMaxQThreads) gemv_fmtq_kernel(const uint8_t* __restrict__ w, int64_t rows, int cols, int row_bytes, int depth,
+                                                                  const float* __restrict__ x, float* __restrict__ y) {
+  using Seg = SegShape<FMT>;
   extern __shared__ __align__(16) uint8_t smem[];
-  __shared__ float s_part[kMaxQThreads / 32][NC];
-  const int padded = (cols + 1023) & ~1023, col_bytes = 3 * padded;
-  const int ring = NC * col_bytes;      // offset of the ring of buffers
-  const int t = threadIdx.x, nthr = blockDim.x, lane = t & 31, warp = t >> 5;
-  const int64_t n_groups = (rows + rows_per_it - 1) / rows_per_it;
-  auto request = [&](int64_t grp, int slot) {
-    const int64_t r0 = grp * rows_per_it;
-    const int nr = static_cast<int>(min(static_cast<int64_t>(rows_per_it), rows - r0));
-    const uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(r0 * row_bytes);
-    const uintptr_t a0 = first & ~static_cast<uintptr_t>(15);
-    const int n16 = static_cast<int>((first + static_cast<uintptr_t>(nr) * row_bytes + 15 - a0) >> 4);
-    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem + ring + slot * buf_bytes));
-    for (int k = t; k < n16; k += nthr) cp_async16(dst + 16 * k, reinterpret_cast<const void*>(a0 + 16 * static_cast<uintptr_t>(k)));
-  };
-  int64_t grp = blockIdx.x;
-  for (int j = 0; j < depth - 1; ++j) {
-    if (grp + j * static_cast<int64_t>(gridDim.x) < n_groups) request(grp + j * static_cast<int64_t>(gridDim.x), j);
+  const int padded = (cols + kSegWeights - 1) / kSegWeights * kSegWeights, col_bytes = 3 * padded;
+  const int t = threadIdx.x, nthr = blockDim.x, lane = t & 31, warp = t >> 5, n_warps = nthr >> 5;
+  const int ring = NC * col_bytes + warp * depth * Seg::kBuf;      // offset of this warp's ring
+  const uint32_t ring_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem + ring));
+  const int segs_per_row = (cols + kSegWeights - 1) / kSegWeights;
+  const int64_t gw = static_cast<int64_t>(blockIdx.x) * n_warps + warp, total_warps = static_cast<int64_t>(gridDim.x) * n_warps;
+  const int64_t my_rows = gw < rows ? (rows - 1 - gw) / total_warps + 1 : 0;
+  const int64_t n_flat = my_rows * segs_per_row;      // this warp's segments, row after row
+  // running description of the next segment to request: its first byte, its number within the row, its ring slot
+  const uintptr_t row_step = static_cast<uintptr_t>(total_warps) * row_bytes - static_cast<uintptr_t>(segs_per_row - 1) * Seg::kBytes;
+  uintptr_t rq_first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(gw) * row_bytes;
+  int rq_seg = 0, rq_slot = 0;
+  int64_t rq_left = n_flat;
+  const int tail_units = (cols >> 8) - 8 * (segs_per_row - 1);      // units of a row's last segment (1..8)
+  auto request = [&]() {
+    if (rq_left > 0) {
+      const bool last = rq_seg == segs_per_row - 1;
+      const int units = last ? tail_units : 8;
+      const uint32_t lead = static_cast<uint32_t>(rq_first) & 15u;
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(rq_first - lead) + 16 * lane;
+      const int n16 = static_cast<int>((lead + units * Seg::kUnit + 15) >> 4);
+      const uint32_t dst = ring_u32 + rq_slot * Seg::kBuf + 16 * lane;
+      for (int k = lane; k < n16; k += 32) cp_async16(dst + 16 * (k - lane), src + 16 * (k - lane));
+      rq_first += last ? row_step : static_cast<uintptr_t>(Seg::kBytes);
+      rq_seg = last ? 0 : rq_seg + 1;
+      --rq_left;
+    }
+    rq_slot = rq_slot + 1 == depth ? 0 : rq_slot + 1;
     cp_async_commit();
-  }
+  };
+  for (int j = 0; j < depth - 1; ++j) request();
   // quantise the activations: one thread per chunk of eight values, four neighbouring lanes per block of 32
   // (the number of chunks is a multiple of 32 and so is the stride: a warp is in a pass as a whole)
   const int n_chunks = cols >> 3;
@@ -327,50 +368,48 @@ __global__ void __launch_bounds__(kMaxQThreads) gemv_fmtq_kernel(const uint8_t* 
       hi[e >> 2] |= static_cast<uint32_t>(h & 255) << (8 * (e & 3));
       lo[e >> 2] |= static_cast<uint32_t>(l & 255) << (8 * (e & 3));
     }
-    uint8_t* xc = smem + c * col_bytes + 8 * chunk_slot<FMT>(kc);
+    uint8_t* xc = smem + c * col_bytes + 16 * piece_slot<FMT>(kc >> 1) + 8 * (kc & 1);
     *reinterpret_cast<uint2*>(xc) = make_uint2(hi[0], hi[1]);
     *reinterpret_cast<uint2*>(xc + padded) = make_uint2(lo[0], lo[1]);
     *reinterpret_cast<int2*>(xc + 2 * padded) = make_int2(sum, __float_as_int(ok ? amax * (1.0f / 32639.0f) : 0.f));
   }
-  const int tpr = nthr / rows_per_it;      // threads per row (>= 32)
-  const int row_in = t / tpr, tl = t - row_in * tpr;
-  const int warps_per_row = tpr >> 5;
-  int slot = 0;      // iteration number modulo depth
-  for (; grp < n_groups; grp += gridDim.x, slot = slot + 1 == depth ? 0 : slot + 1) {
-    const int64_t nxt = grp + static_cast<int64_t>(depth - 1) * gridDim.x;
-    if (nxt < n_groups) request(nxt, slot == 0 ? depth - 1 : slot - 1);      // the buffer read in the iteration before this one
-    cp_async_commit();
-    // this group's copies of this thread (all but the depth-1 newest groups); the barrier makes everybody's (and the
-    // activations) visible
+  __syncthreads();      // the image is complete; from here on the warps go their own ways
+
+  float acc[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) acc[c] = 0.f;
+  int64_t row = gw;
+  int seg = 0, slot = 0;
+  uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(gw) * row_bytes;
+  for (int64_t q = 0; q < n_flat; ++q) {
+    // this segment's copies of this lane (all but the depth-1 newest groups), then everybody's
     switch (depth) {
-      case 2: cp_async_wait<1>(); break;
-      case 3: cp_async_wait<2>(); break;
-      case 4: cp_async_wait<3>(); break;
-      case 5: cp_async_wait<4>(); break;
-      default: cp_async_wait<5>(); break;
+      case 2: cp_async_wait<0>(); break;
+      case 3: cp_async_wait<1>(); break;
+      case 4: cp_async_wait<2>(); break;
+      case 5: cp_async_wait<3>(); break;
+      default: cp_async_wait<4>(); break;
     }
-    __syncthreads();
-    const int64_t r0 = grp * rows_per_it;
-    const uintptr_t first = reinterpret_cast<uintptr_t>(w) + static_cast<uintptr_t>(r0 * row_bytes);
-    const int rowoff = ring + slot * buf_bytes + static_cast<int>(first & 15) + row_in * row_bytes;
-    float acc[NC];
+    __syncwarp();      // also: every lane is done with the buffer of segment q - 1, which the next request overwrites
+    request();
+    const bool last = seg == segs_per_row - 1;
+    const int at = ring + slot * Seg::kBuf + static_cast<int>(static_cast<uint32_t>(first) & 15u);
+    segment_partial<FMT, NC>(smem, at, last ? tail_units : 8, 16 * 128 * seg, col_bytes, padded, lane, acc);
+    slot = slot + 1 == depth ? 0 : slot + 1;
+    if (last) {
 #pragma unroll
-    for (int c = 0; c < NC; ++c) acc[c] = 0.f;
-    if (r0 + row_in < rows) row_partial_q<FMT, NC>(smem, rowoff, col_bytes, padded, cols, tl, tpr, acc);
+      for (int c = 0; c < NC; ++c) {
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
-      if (lane == 0) s_part[warp][c] = acc[c];
-    }
-    __syncthreads();      // also: everybody is done with this group's buffer before the request after next overwrites it
-    if (t < rows_per_it * NC) {
-      const int rr = t / NC, c = t - rr * NC;
-      if (r0 + rr < rows) {
-        float sum = 0.f;
-        for (int wp = 0; wp < warps_per_row; ++wp) sum += s_part[rr * warps_per_row + wp][c];
-        y[static_cast<int64_t>(c) * rows + r0 + rr] = sum;
+        for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+        if (lane == 0) y[static_cast<int64_t>(c) * rows + row] = acc[c];
+        acc[c] = 0.f;
       }
+      seg = 0;
+      row += total_warps;
+      first += row_step;
+    } else {
+      ++seg;
+      first += Seg::kBytes;
     }
   }
   cp_async_wait<0>();
@@ -399,19 +438,27 @@ int launch_gemv_fmt(const uint8_t* w, int64_t rows, int64_t cols, int64_t row_by
     return e == cudaSuccess ? 1 : cuda_rc(e);
   }
   constexpr int F = FMT == PRIMA_FMT_F16 ? PRIMA_FMT_Q8_0 : FMT;      // (the block formats only; keeps the F16 instantiation out)
-  // two CTAs of 256 threads a SM while the activations are small, one of 512 otherwise; what is left of a CTA's share
-  // of shared memory holds the ring: groups of 1..8 rows of up to 56 KiB, small enough for a ring of three
-  const size_t x_bytes = static_cast<size_t>(n_cols) * 3 * static_cast<size_t>((cols + 1023) / 1024 * 1024);
-  if (x_bytes + 2 * (static_cast<size_t>(row_bytes) + 32) > 215 * 1024) return cuda_rc(cudaErrorInvalidValue);
-  const int per_sm = x_bytes <= 40 * 1024 && x_bytes + 3 * (static_cast<size_t>(row_bytes) + 32) <= 107 * 1024 ? 2 : 1;
-  const size_t share = (216 * 1024) / per_sm - 1024;
-  const size_t max_group = std::min<size_t>(56 * 1024, (share - x_bytes) / 3);
-  int rows_per_it = 1;
-  while (rows_per_it < 8 && static_cast<size_t>(row_bytes) * rows_per_it * 2 + 32 <= max_group) rows_per_it *= 2;
-  const int64_t buf_bytes = ((row_bytes * rows_per_it + 15) / 16 + 1) * 16;
-  const int depth = static_cast<int>(std::min<size_t>(6, (share - x_bytes) / static_cast<size_t>(buf_bytes)));      // >= 2 by the check above
-  const size_t smem = x_bytes + static_cast<size_t>(depth) * buf_bytes;
-  void (*kern)(const uint8_t*, int64_t, int, int, int, int, int, const float*, float*) = nullptr;
+  // one CTA per SM: the activations' image once, the rest of shared memory for the warps' rings (2..6 buffers each);
+  // 16 warps, or 8 when the image leaves too little room
+  const size_t x_bytes = static_cast<size_t>(n_cols) * 3 * static_cast<size_t>((cols + kSegWeights - 1) / kSegWeights * kSegWeights);
+  const size_t room = 215 * 1024;
+  // 8..16 warps a CTA: as many as leave every warp a ring of three buffers (two at least), and among those the count
+  // that wastes the fewest warp-rows in the last round (8192 rows on 148 SMs: 14 warps, 98.8 % against 86.5 % with 16)
+  int warps = 0;
+  double best = -1.0;
+  for (int cand = kMaxQThreads / 32; cand >= 8; --cand) {
+    if (x_bytes + static_cast<size_t>(cand) * (cand > 8 ? 3 : 2) * SegShape<F>::kBuf > room) continue;
+    const int64_t all = static_cast<int64_t>(sm_count) * cand;
+    const double eff = static_cast<double>(rows) / static_cast<double>((rows + all - 1) / all * all);
+    if (eff > best + 0.02) {
+      best = eff;
+      warps = cand;
+    }
+  }
+  if (warps == 0) return cuda_rc(cudaErrorInvalidValue);
+  const int depth = static_cast<int>(std::min<size_t>(6, (room - x_bytes) / (static_cast<size_t>(warps) * SegShape<F>::kBuf)));
+  const size_t smem = x_bytes + static_cast<size_t>(warps) * depth * SegShape<F>::kBuf;
+  void (*kern)(const uint8_t*, int64_t, int, int, int, const float*, float*) = nullptr;
   switch (n_cols) {
     case 1: kern = gemv_fmtq_kernel<F, 1>; break;
     case 2: kern = gemv_fmtq_kernel<F, 2>; break;
@@ -420,10 +467,8 @@ int launch_gemv_fmt(const uint8_t* w, int64_t rows, int64_t cols, int64_t row_by
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return cuda_rc(e);
-  const int64_t n_groups = (rows + rows_per_it - 1) / rows_per_it;
-  const int64_t grid = std::min<int64_t>(n_groups, static_cast<int64_t>(sm_count) * per_sm);
-  kern<<<static_cast<unsigned>(grid), kMaxQThreads / per_sm, smem, st>>>(w, rows, static_cast<int>(cols), static_cast<int>(row_bytes), rows_per_it,
-                                                                                   static_cast<int>(buf_bytes), depth, x, y);
+  const int64_t grid = std::min<int64_t>((rows + warps - 1) / warps, sm_count);
+  kern<<<static_cast<unsigned>(grid), warps * 32, smem, st>>>(w, rows, static_cast<int>(cols), static_cast<int>(row_bytes), depth, x, y);
   e = cudaGetLastError();
   return e == cudaSuccess ? 1 : cuda_rc(e);
 }
@@ -471,9 +516,9 @@ int prima_gemv_fmt(int fmt, const void* dev_w, int64_t rows, int64_t cols, const
     return fmt_fail("prima_gemv_fmt: rows >= 1, cols a positive multiple of 256 and 1 <= n_cols <= 4 are required");
   if (reinterpret_cast<uintptr_t>(dev_w) & 1) return fmt_fail("prima_gemv_fmt: dev_w must be at an even address");
   const int64_t row_bytes = cols / prima_fmt_block_weights(fmt) * prima_fmt_block_bytes(fmt);
-  const int64_t x_bytes = fmt == PRIMA_FMT_F16 ? cols * 4 : 3 * ((cols + 1023) / 1024 * 1024);
-  if (static_cast<int64_t>(n_cols) * x_bytes + 2 * (row_bytes + 32) > 200 * 1024)
-    return fmt_fail("prima_gemv_fmt: the activations of all columns and two rows of the matrix must fit 200 KiB of shared memory");
+  const int64_t x_bytes = fmt == PRIMA_FMT_F16 ? cols * 4 : 3 * ((cols + 2047) / 2048 * 2048);
+  if (static_cast<int64_t>(n_cols) * x_bytes + (fmt == PRIMA_FMT_F16 ? 2 * (row_bytes + 32) : 8 * 2 * 2208) > 200 * 1024)
+    return fmt_fail("prima_gemv_fmt: the activations of all columns and the copy buffers must fit 200 KiB of shared memory");
   int dev = 0, sm_count = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
