@@ -1,31 +1,34 @@
 // Grouped-query decode attention over the fp16 KV cache, split along the context.
 //
-// One CTA of 8 warps per (context chunk of 128 positions, KV head); each warp owns 16 positions.
-// The query rows that share the KV head -- the H/G heads of every token of the step, at most 64
-// rows -- are processed 16 at a time (one m16n8k16 tile of rows).  Per tile a warp computes
+// The context is cut into chunks of 128 positions, 16 positions per warp.  The query rows that share a KV head --
+// the H/G heads of every token of the step, at most 64 rows -- are processed 16 at a time (one m16n8k16 tile of
+// rows).  Per tile a warp computes
 //   S = Q K^T   with  A = Q (16 rows x 16 dims, fp16, pre-scaled by 1/sqrt(128)),  B = K,
 //   P = exp(S - max),   O = P V   with  A = P (fp16),  B = V,
-// all with fp32 accumulation on the tensor cores.  K and V go from global memory straight into
-// the B-operand registers with fully used 16-byte loads: the instruction's k index is only a
-// label, so each lane is given the head dimensions (for K) or positions (for V) that make its
-// bytes contiguous in the cache, and Q / P are arranged to match.  The eight warps' (max, sum, O)
-// are combined through shared memory, giving per query row and chunk the running maximum m, the
-// sum l of exp(s - m) and the un-normalised output.  A second kernel merges the chunks of a row in
-// ascending order:  M = max m_c,  o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c.
+// all with fp32 accumulation on the tensor cores, and keeps per query row the running maximum m, the sum l of
+// exp(s - m) and the un-normalised output.  A CTA combines its warps through shared memory and leaves one partial
+// result per row; attn_merge_kernel merges the partial results of a row in ascending order:
+//   M = max m_c,  o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c.
 // Token t of the step attends positions 0 .. pos + t (causal inside the step).
 //
-// The kernel also finishes the fused QKV product that precedes it: every CTA forms the queries of
-// its KV head from that product's accumulators (RMSNorm factor, rotation); a CTA that owns a chunk
-// with new positions also forms the new keys and values, rounds them to binary16, appends them to
-// the cache and keeps a copy in shared memory, from which its warps take them (the cache is never
-// read back inside the kernel).
+// The kernels also finish the fused QKV product that precedes them: every CTA forms the queries it needs from that
+// product's accumulators (RMSNorm factor, rotation); the CTA that owns the step's new positions also forms the new
+// keys and values, rounds them to binary16, appends them to the cache and keeps a copy in shared memory, from which
+// they are used (the cache is never read back inside the kernel).
 //
-// Two kernels.  attn_one_kernel serves at most eight query rows per KV head (one token per request):
-// a CTA that takes several chunks carries its running state from chunk to chunk and leaves ONE partial
-// result, and the merge is part of the same kernel: every CTA of a (request, KV head) takes a ticket
-// after it has written its partial result, and the CTA that draws the last ticket -- nobody waits for
-// anybody -- combines all of them in ascending order and writes the output rows.  attn_partial_kernel
-// + attn_merge_kernel serve a step of several tokens of one sequence (up to 64 query rows per KV head).
+// Two kernels.
+//  * attn_one_kernel: at most eight query rows per KV head (one token), fewer than about ten thousand positions.
+//    Two CTAs per SM, one per (slot of chunks, KV head).  K and V go from global memory straight into the B-operand
+//    registers with fully used 16-byte loads: the instruction's k index is only a label, so each lane is given the
+//    head dimensions (for K) or positions (for V) that make its bytes contiguous in the cache, and Q / P are
+//    arranged to match.  A CTA that takes several chunks carries its running state from chunk to chunk in per-warp
+//    tiles in shared memory.  Optionally (PRIMA_ATTN_MERGE=fused) the merge is part of the kernel: every CTA of a
+//    KV head takes a ticket after it has written its partial result, and the CTA that draws the last ticket --
+//    nobody waits for anybody -- combines all of them in ascending order and writes the output rows.
+//  * attn_tile_kernel<T>: steps of several tokens (T tiles of 16 rows per KV head), steps of several requests (one
+//    tile per request, grid.z = request, its own cache and position) and one-token steps on long contexts.  One CTA
+//    per SM; keys and values are streamed through shared-memory rings of asynchronous copies and read with
+//    ldmatrix; queries and the running output tile stay in registers (see the comment at the kernel).
 //
 // Cache entries below `stable_below` were written before the host last waited for the stream, or by a
 // kernel at least one full step upstream whose completion the host has observed; only those are read
@@ -33,13 +36,10 @@
 // still be in flight when this kernel starts (programmatic dependent launch orders nothing before the
 // wait), so they are read after it.
 //
-// With several independent requests per step (one token each) the grid gets a third dimension: CTA
-// (chunk, KV head, request) works on that request's own cache and position, all in one launch.
-//
-// Latency matters more than bandwidth here (the whole cache of a layer is a few microseconds of
-// HBM time): every warp requests the old entries of its positions before it waits for the
-// predecessor kernel, all loads of the finishing step are issued together, and the shared-memory
-// tiles are padded and swizzled so that neither their 16-byte stores nor their reads conflict.
+// At short contexts latency matters more than bandwidth (the whole cache of a layer is a few microseconds of HBM
+// time): old entries are requested before the wait for the predecessor kernel, all loads of the finishing step are
+// issued together, and the shared-memory tiles are padded (and in attn_one_kernel swizzled) so that neither their
+// stores nor their reads conflict.
 #include <cstdlib>
 
 #include "common.cuh"
