@@ -271,7 +271,7 @@ struct Walk {
 
 }  // namespace gemv_detail
 
-// Launches the 5..16-token kernel on `grid` CTAs (defined in q4k_gemm_tokens.cu); CTAs of that kernel per SM.
+// Launches the 4..16-token kernel on `grid` CTAs (defined in q4k_gemm_tokens.cu); CTAs of that kernel per SM.
 int gemv_tokens_ctas_per_sm(int n_tok);
 cudaError_t launch_gemv_tokens(const gemv_detail::GemvParams& P, int64_t grid, cudaStream_t st);
 

@@ -122,7 +122,7 @@ def test_gemv_activation_scales_and_special_vectors(gpu):
 
 @pytest.mark.parametrize("n", [6, 11])
 def test_gemv_several_tokens_with_outliers_and_mixed_scales(gpu, n):
-    # 5..16 columns go through the kernel that quantises a column's 256 activations with one step
+    # 4..16 columns go through the kernel that quantises a column's 256 activations with one step
     rows, cols = 264, 2048
     w = synth.model_tensor(8, 0, synth.WQ, rows, cols)
     x = synth.activations(8, n, cols)
