@@ -196,14 +196,34 @@ __device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {      // 
   asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-// N consecutive words starting at an even byte offset `a` of shared memory: N + 1 aligned words, shifted by 0 or 16 bits.
+// Loads from shared memory by 32-bit shared-space address (volatile: they stay behind the wait that precedes them).
+__device__ __forceinline__ uint32_t sld32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t sld16(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ int sld8s(uint32_t a) {
+  int v;
+  asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint4 sld128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+// N consecutive words starting at an even shared-memory address `a`: N + 1 aligned words, shifted by 0 or 16 bits.
 template <int N>
-__device__ __forceinline__ void lds_even(const uint8_t* smem, int a, uint32_t (&out)[N]) {
-  const uint32_t* p = reinterpret_cast<const uint32_t*>(smem + (a & ~3));
-  const uint32_t sh = (a & 2) * 8;
+__device__ __forceinline__ void lds_even(uint32_t a, uint32_t (&out)[N]) {
+  const uint32_t base = a & ~3u, sh = (a & 2u) * 8u;
   uint32_t w[N + 1];
 #pragma unroll
-  for (int i = 0; i <= N; ++i) w[i] = p[i];
+  for (int i = 0; i <= N; ++i) w[i] = sld32(base + 4 * i);
 #pragma unroll
   for (int i = 0; i < N; ++i) out[i] = __funnelshift_r(w[i], w[i + 1], sh);
 }
@@ -234,25 +254,26 @@ struct SegShape {
   static constexpr int kUnit = FMT == PRIMA_FMT_Q8_0 ? 272 : 210;               // bytes of 256 weights
 };
 
-// One segment of one row, staged at shared-memory offset `seg` (its first byte): this lane's share of sum w x.
+// One segment of one row, staged at shared-memory address `seg` (its first byte): this lane's share of sum w x.
+// `ximg` is the address of the activations' image of column 0 at this segment (+ 16 * lane).
 template <int FMT, int NC>
-__device__ __forceinline__ void segment_partial(const uint8_t* smem, int seg, int n_units, int xseg, int col_bytes, int padded, int lane, float (&acc)[NC]) {
+__device__ __forceinline__ void segment_partial(uint32_t seg, int n_units, uint32_t ximg, uint32_t col_bytes, uint32_t padded, int lane, float (&acc)[NC]) {
   if (FMT == PRIMA_FMT_Q8_0) {
     // lane = block within a half segment of 32 blocks (8 units of 256 weights = 64 blocks)
 #pragma unroll
     for (int hs = 0; hs < 2; ++hs) {
       const int b = 32 * hs + lane;
       if (b < 8 * n_units) {
-        const int blk = seg + 34 * b;
-        const float d = half_bits_to_float(lds_u16(smem + blk));
+        const uint32_t blk = seg + 34 * b;
+        const float d = half_bits_to_float(sld16(blk));
         uint32_t q[8];
-        lds_even<8>(smem, blk + 2, q);
+        lds_even<8>(blk + 2, q);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
-          const uint8_t* xc = smem + c * col_bytes + xseg + 1024 * hs + 16 * lane;
-          const uint4 h0 = *reinterpret_cast<const uint4*>(xc), h1 = *reinterpret_cast<const uint4*>(xc + 512);
-          const uint4 l0 = *reinterpret_cast<const uint4*>(xc + padded), l1 = *reinterpret_cast<const uint4*>(xc + padded + 512);
-          const float step = *reinterpret_cast<const float*>(xc + 2 * padded + 4);
+          const uint32_t xc = ximg + c * col_bytes + 1024 * hs;
+          const uint4 h0 = sld128(xc), h1 = sld128(xc + 512);
+          const uint4 l0 = sld128(xc + padded), l1 = sld128(xc + padded + 512);
+          const float step = __uint_as_float(sld32(xc + 2 * padded + 4));
           int h = dp4a_ss(q[3], h0.w, dp4a_ss(q[2], h0.z, dp4a_ss(q[1], h0.y, dp4a_ss(q[0], h0.x, 0))));
           h = dp4a_ss(q[7], h1.w, dp4a_ss(q[6], h1.z, dp4a_ss(q[5], h1.y, dp4a_ss(q[4], h1.x, h))));
           int l = dp4a_ss(q[3], l0.w, dp4a_ss(q[2], l0.z, dp4a_ss(q[1], l0.y, dp4a_ss(q[0], l0.x, 0))));
@@ -265,31 +286,32 @@ __device__ __forceinline__ void segment_partial(const uint8_t* smem, int seg, in
     // lane = (super-block s of the segment, half n, 16 positions 16 h ..): 64 weights
     const int s = lane >> 2, n = (lane >> 1) & 1, h16 = lane & 1;
     if (s < n_units) {
-      const int sb = seg + 210 * s;
+      const uint32_t sb = seg + 210 * s;
       uint32_t qa[4], qb[4], qh[4];
-      lds_even<4>(smem, sb + 64 * n + 16 * h16, qa);
-      lds_even<4>(smem, sb + 64 * n + 32 + 16 * h16, qb);
-      lds_even<4>(smem, sb + 128 + 32 * n + 16 * h16, qh);
-      const float d = half_bits_to_float(lds_u16(smem + sb + 208));
-      const int8_t* scp = reinterpret_cast<const int8_t*>(smem + sb + 192 + 8 * n + h16);
+      lds_even<4>(sb + 64 * n + 16 * h16, qa);
+      lds_even<4>(sb + 64 * n + 32 + 16 * h16, qb);
+      lds_even<4>(sb + 128 + 32 * n + 16 * h16, qh);
+      const float d = half_bits_to_float(sld16(sb + 208));
+      const uint32_t scp = sb + 192 + 8 * n + h16;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         uint32_t v[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const uint32_t src = (i & 1) ? qb[k] : qa[k];
-          v[k] = (i < 2 ? (src & 0x0f0f0f0fu) : ((src >> 4) & 0x0f0f0f0fu)) | (((qh[k] >> (2 * i)) & 0x03030303u) << 4);
+          const uint32_t hi2 = (i < 2 ? (qh[k] << (4 - 2 * i)) : (qh[k] >> (2 * i - 4))) & 0x30303030u;
+          v[k] = ((i < 2 ? src : (src >> 4)) & 0x0f0f0f0fu) | hi2;
         }
-        const float dsc = d * static_cast<float>(scp[2 * i]);
+        const float dsc = d * static_cast<float>(sld8s(scp + 2 * i));
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
-          const uint8_t* xc = smem + c * col_bytes + xseg + 512 * i + 16 * lane;
-          const uint4 xh = *reinterpret_cast<const uint4*>(xc);
-          const uint4 xl = *reinterpret_cast<const uint4*>(xc + padded);
-          const int4 ss = *reinterpret_cast<const int4*>(xc + 2 * padded);      // (sum, step, sum, step): one block of 32, one step
+          const uint32_t xc = ximg + c * col_bytes + 512 * i;
+          const uint4 xh = sld128(xc);
+          const uint4 xl = sld128(xc + padded);
+          const uint4 ss = sld128(xc + 2 * padded);      // (sum, step, sum, step): one block of 32, one step
           const int hh = dp4a_us(v[3], xh.w, dp4a_us(v[2], xh.z, dp4a_us(v[1], xh.y, dp4a_us(v[0], xh.x, 0))));
           const int ll = dp4a_us(v[3], xl.w, dp4a_us(v[2], xl.z, dp4a_us(v[1], xl.y, dp4a_us(v[0], xl.x, 0))));
-          acc[c] = fmaf(static_cast<float>(hh * 256 + ll - 32 * (ss.x + ss.z)), dsc * __int_as_float(ss.y), acc[c]);
+          acc[c] = fmaf(static_cast<float>(hh * 256 + ll - 32 * (static_cast<int>(ss.x) + static_cast<int>(ss.z))), dsc * __uint_as_float(ss.y), acc[c]);
         }
       }
     }
@@ -309,6 +331,7 @@ __global__ void __launch_bounds__(kMaxQThreads) gemv_fmtq_kernel(const uint8_t* 
   const int t = threadIdx.x, nthr = blockDim.x, lane = t & 31, warp = t >> 5, n_warps = nthr >> 5;
   const int ring = NC * col_bytes + warp * depth * Seg::kBuf;      // offset of this warp's ring
   const uint32_t ring_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem + ring));
+  const uint32_t img_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + 16 * lane;      // this lane's piece of a segment's image
   const int segs_per_row = (cols + kSegWeights - 1) / kSegWeights;
   const int64_t gw = static_cast<int64_t>(blockIdx.x) * n_warps + warp, total_warps = static_cast<int64_t>(gridDim.x) * n_warps;
   const int64_t my_rows = gw < rows ? (rows - 1 - gw) / total_warps + 1 : 0;
@@ -393,8 +416,8 @@ __global__ void __launch_bounds__(kMaxQThreads) gemv_fmtq_kernel(const uint8_t* 
     __syncwarp();      // also: every lane is done with the buffer of segment q - 1, which the next request overwrites
     request();
     const bool last = seg == segs_per_row - 1;
-    const int at = ring + slot * Seg::kBuf + static_cast<int>(static_cast<uint32_t>(first) & 15u);
-    segment_partial<FMT, NC>(smem, at, last ? tail_units : 8, 16 * 128 * seg, col_bytes, padded, lane, acc);
+    const uint32_t at = ring_u32 + slot * Seg::kBuf + (static_cast<uint32_t>(first) & 15u);
+    segment_partial<FMT, NC>(at, last ? tail_units : 8, img_u32 + 2048 * seg, col_bytes, padded, lane, acc);
     slot = slot + 1 == depth ? 0 : slot + 1;
     if (last) {
 #pragma unroll
