@@ -124,6 +124,13 @@ __device__ __forceinline__ void team_sync(int team) {
   else asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(32 * T) : "memory");
 }
 
+// 2^x by the special-function unit (2 ulp; 2^-inf = 0).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 template <int T>
 __global__ void __launch_bounds__(TileShape<T>::kWarpsOf * 32, 1)
 attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
@@ -209,7 +216,9 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
 
   // ---- finish the QKV product for this KV head.  Items: one rotation pair of a query row, and for the CTA that owns
   //      the new positions also one pair of each new key and value.
-  const float scale = 0.08838834764831845f;   // 1 / sqrt(128)
+  // 1 / sqrt(128) times log2(e): scores come out in units of log2, so that every exponential is a bare ex2; the
+  // running maximum handed to the merge is converted back
+  const float scale = 0.08838834764831845f * 1.4426950408889634f;
   const int n_q_items = n_rows * (kHeadDim / 2);
   const int n_items = n_q_items + (owns_new ? 2 * n_tok * (kHeadDim / 2) : 0);      // at most 4096 + 1024
   constexpr int kTrip = 8;
@@ -304,18 +313,25 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
   // One sub-chunk of 16 positions staged at `stage` (shared-memory address); position wbase + c is visible to row hr
   // when it is at most last[hr].
   auto process = [&](uint32_t stage, int wbase, const int (&last)[2], bool masked) {
-    float sc[2][4];
+    float sc[2][4], sd[2][4];      // even and odd k steps apart: four chains of four dependent instructions instead of two of eight
 #pragma unroll
-    for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = 0.f;
+    for (int pb = 0; pb < 2; ++pb) sc[pb][0] = sc[pb][1] = sc[pb][2] = sc[pb][3] = sd[pb][0] = sd[pb][1] = sd[pb][2] = sd[pb][3] = 0.f;
     // S = Q K^T: matrices (positions 0-7 | 8-15) x (dims 16 ks .. + 7 | + 8 .. + 15)
     const uint32_t k_addr = stage + ((lane & 7) + 8 * (lane >> 4)) * kStageRow + 16 * ((lane >> 3) & 1);
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      uint32_t b0, b1, b2, b3;
+    for (int ks = 0; ks < 8; ks += 2) {
+      uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
       ldmatrix_x4(k_addr + 32 * ks, b0, b1, b2, b3);
+      ldmatrix_x4(k_addr + 32 * ks + 32, c0, c1, c2, c3);
       mma_f16(sc[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
       mma_f16(sc[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+      mma_f16(sd[0], qa[ks + 1][0], qa[ks + 1][1], qa[ks + 1][2], qa[ks + 1][3], c0, c1);
+      mma_f16(sd[1], qa[ks + 1][0], qa[ks + 1][1], qa[ks + 1][2], qa[ks + 1][3], c2, c3);
     }
+#pragma unroll
+    for (int pb = 0; pb < 2; ++pb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sc[pb][e] += sd[pb][e];
     // ---- mask, row maxima, rescaling factors, exponentials
     float mx[2] = {-INFINITY, -INFINITY};
     if (masked) {      // (the same for the whole warp)
@@ -336,8 +352,10 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     for (int hr = 0; hr < 2; ++hr) {
       mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
       mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
-      m_new[hr] = fmaxf(m_run[hr], mx[hr]);
-      alpha[hr] = m_run[hr] > -INFINITY ? __expf(m_run[hr] - m_new[hr]) : 1.0f;      // nothing accumulated yet: the tile is zero
+      // the reference point of a row moves only when a score exceeds it by more than 2^8: until then the exponentials
+      // are at most 256 (exact enough in fp16, harmless in the fp32 sums) and the output tile needs no rescaling
+      m_new[hr] = mx[hr] > m_run[hr] + 8.0f ? mx[hr] : m_run[hr];
+      alpha[hr] = m_run[hr] > -INFINITY ? fast_exp2(m_run[hr] - m_new[hr]) : 1.0f;      // nothing accumulated yet: the tile is zero
       lsum[hr] = 0.f;
     }
     uint32_t pa[4];      // A fragment of P: rows g, g + 8 x positions 2t, 2t+1 (first block of 8) and 8 + 2t, + 1
@@ -347,7 +365,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int hr = e >> 1;
-        pv[e] = m_new[hr] > -INFINITY ? __expf(sc[pb][e] - m_new[hr]) : 0.f;
+        pv[e] = m_new[hr] > -INFINITY ? fast_exp2(sc[pb][e] - m_new[hr]) : 0.f;
         lsum[hr] += pv[e];
       }
       pa[2 * pb] = pack_h2(pv[0], pv[1]);        // row g
@@ -406,9 +424,9 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     for (int hr = 0; hr < 2; ++hr) last[hr] = pos + max(row_tok[hr], 0);      // causal among the new positions
     process(ring_u32, pos, last, true);
   }
-  if (t == 0) {
-    s_m[warp][g] = m_run[0];
-    s_m[warp][g + 8] = m_run[1];
+  if (t == 0) {      // (back to natural units: the merge and the one-token kernel use e^x)
+    s_m[warp][g] = m_run[0] * 0.6931471805599453f;
+    s_m[warp][g + 8] = m_run[1] * 0.6931471805599453f;
     s_l[warp][g] = l_run[0];
     s_l[warp][g + 8] = l_run[1];
   }
