@@ -10,6 +10,12 @@ random-init Q4_K tensors of the named shape; the KV cache is prefilled with N(0,
 
 With --n-tok T > 1 a step is one verification pass of speculative decoding: T tokens at consecutive
 positions go through the model together (causal among themselves) and the time is reported per step.
+Other lines: --requests R (one token of each of R concurrent requests per step, own caches), --ctx N (cached
+positions), --speculative 8b (speculative cycles with a draft model), --resident-layers N (the layers from N on
+are streamed from pinned host memory every token; reported against the host-link rate measured in the same run),
+--gemv-fmt q6_k|q8_0|f16 (the single product in another weight format), --l2-ahead-mb / --l2-ahead-o-mb (how much
+of the gate/up matrix is asked into L2 during attention and the O product), --repeats (timed regions; the value is
+their median).
 
 With N > 1 (launched by torch.distributed.run) every rank decodes its own request on its own
 GPU: the path does not shard, ranks are independent replicas and no collective is on the data
