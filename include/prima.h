@@ -161,7 +161,8 @@ int prima_kv_load_seq(prima_ctx* ctx, int seq, int layer, int pos_begin, int n_p
 int prima_kv_read_seq(prima_ctx* ctx, int seq, int layer, int pos_begin, int n_pos, uint16_t* k, uint16_t* v);
 
 /* Wait for all queued work; returns PRIMA_ERR_DEVICE if a kernel raised the status word (a
- * partial sum outside the accumulator range, or a bounded wait inside a kernel that gave up) and
+ * partial sum outside the accumulator range, a bounded wait inside a kernel that gave up, or, in the
+ * library built with -DPRIMA_BOUNDS, an index outside its array: that access is skipped) and
  * PRIMA_ERR_CUDA if the stream reports an error.  A raised status word is reported once; the
  * outputs of the steps queued since the previous prima_sync are then invalid, and before it returns
  * prima_sync clears the status word and the library's internal accumulators, so the context can go

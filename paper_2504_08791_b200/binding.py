@@ -12,7 +12,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libprima.so")
+# PRIMA_LIB=bounds selects the range-checked build of the same sources (tests)
+LIB_PATH = os.path.join(_HERE, "libprima_bounds.so" if os.environ.get("PRIMA_LIB") == "bounds" else "libprima.so")
 
 OK, ERR_ARG, ERR_STATE, ERR_CUDA, ERR_NOMEM, ERR_DEVICE = 0, -1, -2, -3, -4, -5
 ATTN_NORM, WQ, WK, WV, WO, FFN_NORM, W_GATE, W_UP, W_DOWN, OUT_NORM, W_HEAD, TOK_EMBD = range(12)
@@ -57,7 +58,7 @@ def lib():
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2504_08791_b200.build` "
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2504_08791_b200.build` (`--bounds` for the range-checked one) "
                                "(there is no CPU fallback)")
         L = C.CDLL(LIB_PATH)
         vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int

@@ -525,6 +525,7 @@ int prima_ctx_create(const prima_model_config* cfg, void* cuda_stream, prima_ctx
   A(dev_alloc(c, &c->am_idx, static_cast<size_t>(kMaxTok) * kArgmaxBlocks));
   A(dev_alloc(c, &c->am_out, static_cast<size_t>(kMaxTok)));
   A(dev_alloc(c, &c->status, 1, true));
+  c->attn.status = c->status;
   if (rc != PRIMA_OK) {
     g_tls_error = c->err;
     for (void* p : c->allocs) cudaFree(p);
@@ -995,7 +996,8 @@ int prima_sync(prima_ctx* c) {
     if (e != cudaSuccess) return cuda_fail(c, e, "prima_sync(reset)");
   }
   if (status != 0)
-    return fail(c, PRIMA_ERR_DEVICE, !(status & 1) ? "a partial sum was outside the accumulator range (+-2^27); results of this step are invalid"
+    return fail(c, PRIMA_ERR_DEVICE, (status & 4) ? "an index was outside its array (range-checked build); results of this step are invalid (status " + std::to_string(status) + ")"
+                                     : !(status & 1) ? "a partial sum was outside the accumulator range (+-2^27); results of this step are invalid"
                                                  : "a bounded wait inside a kernel gave up (status " + std::to_string(status) + ")");
   return PRIMA_OK;
 }

@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(TileShape<T>::kWarpsOf * 32, 1)
 attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __restrict__ ssq, int n_groups, float inv_width, float eps,
                  const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
                  int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_tok, int part_stride,
-                 float* __restrict__ o_part, float2* __restrict__ ml_part, const AttnSeqs seqs, const Stamp stamp, const L2Ahead ahead) {
+                 float* __restrict__ o_part, float2* __restrict__ ml_part, const AttnSeqs seqs, const Stamp stamp, const L2Ahead ahead, int* status) {
   using Shape = TileShape<T>;
   constexpr int P = Shape::kTeams, S = Shape::kStagesOf, W = Shape::kWarpsOf, kThr = W * 32;
   pdl_trigger();
@@ -278,9 +278,11 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
           __half* sm = (is_v ? new_v : new_k) + tok * kHeadDim;
           sm[a] = ha;
           sm[b] = hb;
-          __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + pos + tok) * kHeadDim;
-          gd[a] = ha;
-          gd[b] = hb;
+          if (in_range(pos + tok >= 0 && pos + tok < kv_capacity, status)) {
+            __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + pos + tok) * kHeadDim;
+            gd[a] = ha;
+            gd[b] = hb;
+          }
         }
       }
     }
@@ -462,6 +464,7 @@ attn_tile_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __res
     }
     const int tok = rr / group, head = kv * group + rr % group;
     const int64_t slot = (static_cast<int64_t>(row_base) + static_cast<int64_t>(tok) * n_q_heads + head) * part_stride + blockIdx.x;
+    if (!in_range(static_cast<int>(blockIdx.x) < part_stride, status)) continue;
     *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
     if (d4 == 0) ml_part[slot] = make_float2(s_big[tile][r], l);
   }
@@ -484,7 +487,7 @@ attn_one_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __rest
                 const float2* __restrict__ rope_tab, int rope_mode, __half* __restrict__ k_cache, __half* __restrict__ v_cache,
                 int kv_capacity, int n_q_heads, int n_kv_heads, int pos, int stable_below, int n_chunks, int part_stride,
                 float* __restrict__ o_part, float2* __restrict__ ml_part, int* __restrict__ tickets, float* __restrict__ o,
-                const AttnSeqs seqs, const Stamp stamp, const L2Ahead ahead) {
+                const AttnSeqs seqs, const Stamp stamp, const L2Ahead ahead, int* status) {
   pdl_trigger();
   int row_base = 0;                 // first output row (request * heads) of this CTA's request
   if (seqs.n > 0) {                 // one request per blockIdx.z: its own cache and position
@@ -609,9 +612,11 @@ attn_one_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __rest
           __half* sm = is_v ? new_v : new_k;
           sm[a] = ha;
           sm[b] = hb;
-          __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + pos) * kHeadDim;
-          gd[a] = ha;
-          gd[b] = hb;
+          if (in_range(pos >= 0 && pos < kv_capacity, status)) {
+            __half* gd = (is_v ? v_cache : k_cache) + (static_cast<int64_t>(kv) * kv_capacity + pos) * kHeadDim;
+            gd[a] = ha;
+            gd[b] = hb;
+          }
         }
       }
     }
@@ -740,7 +745,7 @@ attn_one_kernel(const acc_t* __restrict__ acc, int64_t mpad, const float* __rest
     stamp_end(stamp);
     return;
   }
-  if (r < group) {
+  if (r < group && in_range(static_cast<int>(blockIdx.x) < part_stride, status)) {
     const int64_t slot = out_row * part_stride + blockIdx.x;
     *reinterpret_cast<float4*>(o_part + slot * kHeadDim + d4) = accum;
     if (lane == 0) ml_part[slot] = make_float2(s_big[r], l);
@@ -918,7 +923,7 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
     int* tickets = attention_merge_is_fused() ? scr.tickets : nullptr;
     cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
                                ssq.n_groups, inv_width, ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads,
-                               pos, stable_below, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, none, scr.stamp, scr.ahead);
+                               pos, stable_below, n_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, none, scr.stamp, scr.ahead, scr.status);
     if (e != cudaSuccess) return cuda_rc(e);
     if (tickets) return 1;
     e = launch_pdl(attn_merge_kernel, dim3(n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * grid.x) * sizeof(float), st, scr.o_part,
@@ -933,7 +938,7 @@ int launch_attention(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, const
   auto launch_tile = [&](auto kernel, int warps, size_t bytes) {
     return launch_pdl(kernel, tgrid, dim3(warps * 32), bytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data), ssq.n_groups, inv_width,
                       ssq.eps, rope_tab, rope_mode, k_cache, v_cache, kv_capacity, n_q_heads, n_kv_heads, pos, stable_below, n_tok,
-                      scr.max_chunks, scr.o_part, scr.ml_part, none, scr.stamp, scr.ahead);
+                      scr.max_chunks, scr.o_part, scr.ml_part, none, scr.stamp, scr.ahead, scr.status);
   };
   cudaError_t e = n_tiles == 1   ? launch_tile(attn_tile_kernel<1>, TileShape<1>::kWarpsOf, TileShape<1>::kSmem)
                   : n_tiles == 2 ? launch_tile(attn_tile_kernel<2>, TileShape<2>::kWarpsOf, TileShape<2>::kSmem)
@@ -963,7 +968,7 @@ int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, 
     cudaError_t e = launch_pdl(attn_tile_kernel<1>, tgrid, dim3(TileShape<1>::kWarpsOf * 32), TileShape<1>::kSmem, st, acc_qkv, mpad,
                                static_cast<const float*>(ssq.data), ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps,
                                rope_tab, rope_mode, static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads, n_kv_heads,
-                               0, stable_below, 1, scr.max_chunks, scr.o_part, scr.ml_part, seqs, scr.stamp, scr.ahead);
+                               0, stable_below, 1, scr.max_chunks, scr.o_part, scr.ml_part, seqs, scr.stamp, scr.ahead, scr.status);
     if (e != cudaSuccess) return cuda_rc(e);
     const AttnSeqs none{};
     e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * tgrid.x) * sizeof(float), st, scr.o_part,
@@ -977,7 +982,7 @@ int launch_attention_seqs(const acc_t* acc_qkv, int64_t mpad, const SumSq& ssq, 
   cudaError_t e = launch_pdl(attn_one_kernel, grid, dim3(kThreads), kOneSmemBytes, st, acc_qkv, mpad, static_cast<const float*>(ssq.data),
                              ssq.n_groups, ssq.width > 0 ? 1.0f / static_cast<float>(ssq.width) : 0.f, ssq.eps, rope_tab, rope_mode,
                              static_cast<__half*>(nullptr), static_cast<__half*>(nullptr), kv_capacity, n_q_heads, n_kv_heads, 0, stable_below,
-                             max_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, seqs, scr.stamp, scr.ahead);
+                             max_chunks, scr.max_chunks, scr.o_part, scr.ml_part, tickets, o, seqs, scr.stamp, scr.ahead, scr.status);
   if (e != cudaSuccess) return cuda_rc(e);
   if (tickets) return 1;
   e = launch_pdl(attn_merge_kernel, dim3(seqs.n * n_q_heads), dim3(kHeadDim), static_cast<size_t>(2 * grid.x) * sizeof(float), st, scr.o_part,

@@ -190,6 +190,7 @@ struct AttnScratch {
   int* tickets;     // [kMaxTok][G], all zero between launches (see attn_one_kernel)
   Stamp stamp;      // of the next attention launch (both kernels share it)
   L2Ahead ahead;    // requested by the CTAs of the next attention launch as they start
+  int* status = nullptr;      // the context's status word (range-checked build: bit 2)
 };
 // Several independent requests in one launch: token t of the step belongs to a request with its own
 // cache (k[t], v[t]) and position pos[t]; rows, statistics, rotary table and outputs of token t are
@@ -283,6 +284,17 @@ __device__ __forceinline__ void l2_ahead(const L2Ahead& a, unsigned cta, unsigne
     }
   }
 }
+
+// Range-checked build (-DPRIMA_BOUNDS): an index outside its array raises bit 2 of the status word and the access is
+// skipped; nothing traps.  In the ordinary build the check costs nothing.
+#ifdef PRIMA_BOUNDS
+__device__ __forceinline__ bool in_range(bool ok, int* status) {
+  if (!ok && status) atomicOr(status, 4);
+  return ok;
+}
+#else
+__device__ __forceinline__ bool in_range(bool, int*) { return true; }
+#endif
 
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -199,8 +199,11 @@ __global__ void __launch_bounds__(NB * kMaxWarps * 32, TokCfg<NB>::kCtasPerSm) g
     const int nb = pf.batch();
     if (lane == 0 && tb == 0) {
       const uint8_t* src = w + (static_cast<int64_t>(pf.grp * sg + warp) * n_rt + pf.rt) * kUnitBytes;
-      mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
-      bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot, stream_once_policy());
+      // (range-checked build: the batch lies inside the matrix; a request that does not is left out and its wait runs out)
+      if (in_range(src >= w && src + nb * kUnitBytes <= w + static_cast<int64_t>(n_sb) * n_rt * kUnitBytes && nb >= 1 && nb <= kBatch, status)) {
+        mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
+        bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot, stream_once_policy());
+      }
     }
     pf.next(nb);
     ++n_in_flight;
@@ -398,7 +401,8 @@ __global__ void __launch_bounds__(NB * kMaxWarps * 32, TokCfg<NB>::kCtasPerSm) g
           for (int ww = 1; ww < kMaxWarps; ++ww)
             if (ww < sg) sum += src[ww * kBatch * kRowsPerTile * kCols];
           if (!(fabsf(sum) < kAccLimit)) atomicOr(status, 2);
-          atomicAdd(acc_out + static_cast<int64_t>(tok) * mpad + acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row), acc_from(sum));
+          const int64_t at = acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row);
+          if (in_range(at >= 0 && at < mpad && tok < P.n_tok_total, status)) atomicAdd(acc_out + static_cast<int64_t>(tok) * mpad + at, acc_from(sum));
         }
       }
       parity ^= 1;

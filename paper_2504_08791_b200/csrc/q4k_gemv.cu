@@ -280,8 +280,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
     const int nb = pf.batch();
     if (lane == 0) {
       const uint8_t* src = w + (static_cast<int64_t>(pf.grp * sg + warp) * n_rt + pf.rt) * kUnitBytes;
-      mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
-      bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot, stream_once_policy());
+      // (range-checked build: the batch lies inside the matrix; a request that does not is left out and its wait runs out)
+      if (in_range(src >= w && src + nb * kUnitBytes <= w + static_cast<int64_t>(n_sb) * n_rt * kUnitBytes && nb >= 1 && nb <= kBatch, status)) {
+        mbar_expect_tx(bar_u32 + 8 * rslot, nb * kUnitBytes);
+        bulk_load(ring_u32 + rslot * kBatchBytes, src, nb * kUnitBytes, bar_u32 + 8 * rslot, stream_once_policy());
+      }
     }
     pf.next(nb);
     ++n_in_flight;
@@ -409,7 +412,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, (NTOK == 1 ? 2 : 1)) gemv_part
         float sum = src[0];
         for (int ww = 1; ww < sg; ++ww) sum += src[ww * kBatch * kRowsPerTile];
         if (!(fabsf(sum) < kAccLimit)) atomicOr(status, 2);
-        atomicAdd(acc_out + static_cast<int64_t>(tok0 + k) * mpad + acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row), acc_from(sum));
+        const int64_t at = acc_position(P.out_order, (cur.rt + i) * kRowsPerTile + row);
+        if (in_range(at >= 0 && at < mpad && tok0 + k < P.n_tok_total, status)) atomicAdd(acc_out + static_cast<int64_t>(tok0 + k) * mpad + at, acc_from(sum));
       }
     }
     parity ^= 1;

@@ -370,3 +370,67 @@ def test_merge_inside_the_attention_kernel_matches_checker():
     env = dict(os.environ, PRIMA_ATTN_MERGE="fused", PYTHONPATH=root)
     out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "fused merge ok" in out.stdout, out.stdout + out.stderr
+
+
+def test_range_checked_build_gives_the_same_bits_and_raises_nothing(gpu):
+    """The library built with -DPRIMA_BOUNDS (every weight request, accumulator index, cache append and partial-result
+    slot checked against its array; a violation would raise bit 2 of the status word and skip the access) runs the
+    same steps in a child process: no status is raised (prima_sync succeeds) and the hidden states and logits have the
+    bits of the ordinary build.  Shapes with ragged tails, several tokens, several requests, a long context."""
+    import os
+    import subprocess
+    import sys
+    import tempfile
+    torch, binding = gpu
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    if not os.path.exists(os.path.join(root, "paper_2504_08791_b200", "libprima_bounds.so")):
+        from paper_2504_08791_b200 import build as _build
+        _build.build(bounds=True)
+    code = (
+        "import sys, numpy as np, torch\n"
+        "from paper_2504_08791_b200 import binding, synth\n"
+        "out = {}\n"
+        "cases = [('tiny', {}, 37, 1), ('small', {}, 255, 5), ('small', dict(n_q_heads=10, n_kv_heads=2, hidden=1280, ffn=1280), 128, 7),\n"
+        "         ('small', dict(n_q_heads=4, n_kv_heads=4, hidden=512, ffn=3328, vocab=1000), 0, 2), ('tiny', dict(kv_capacity=12000), 11000, 1)]\n"
+        "for i, (name, over, pos, n_tok) in enumerate(cases):\n"
+        "    cfg = synth.model_config(name, max_n_tok=16, **over)\n"
+        "    ctx = binding.Context(cfg)\n"
+        "    for layer, tid, rows, cols, data in synth.iter_model_tensors(71, cfg):\n"
+        "        ctx.load(layer, tid, data, rows, cols)\n"
+        "    for l in range(cfg['n_layers']):\n"
+        "        if pos:\n"
+        "            k, v = synth.kv_prefill(71, l, pos, cfg['n_kv_heads'], cfg['head_dim'])\n"
+        "            ctx.kv_load(l, 0, k, v)\n"
+        "            ctx.kv_load(l, 0, k[:min(pos, 90)], v[:min(pos, 90)], seq=3)\n"
+        "    h = torch.from_numpy(synth.activations(71, n_tok, cfg['hidden'])).cuda()\n"
+        "    o = torch.empty_like(h)\n"
+        "    ctx.forward_window(0, cfg['n_layers'], h, o, pos, n_tok)\n"
+        "    lg = torch.empty((n_tok, cfg['vocab']), dtype=torch.float32, device='cuda')\n"
+        "    ctx.logits(o, n_tok, lg)\n"
+        "    ctx.sync()\n"
+        "    out['h%d' % i] = o.cpu().numpy(); out['l%d' % i] = lg.cpu().numpy()\n"
+        "    if pos:\n"
+        "        h2 = torch.from_numpy(synth.activations(72, 2, cfg['hidden'])).cuda()\n"
+        "        o2 = torch.empty_like(h2)\n"
+        "        ctx.forward_window_seqs(0, cfg['n_layers'], h2, o2, [0, 3], [pos, min(pos, 90)])\n"
+        "        ctx.sync()\n"
+        "        out['s%d' % i] = o2.cpu().numpy()\n"
+        "    ctx.close()\n"
+        "np.savez(sys.argv[1], **out)\n"
+        "print('steps ok')\n")
+    got = {}
+    with tempfile.TemporaryDirectory() as tmp:
+        for which in ("plain", "bounds"):
+            env = dict(os.environ, PYTHONPATH=root)
+            env.pop("PRIMA_LIB", None)
+            if which == "bounds":
+                env["PRIMA_LIB"] = "bounds"
+            path = os.path.join(tmp, which + ".npz")
+            run = subprocess.run([sys.executable, "-c", code, path], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+            assert run.returncode == 0 and "steps ok" in run.stdout, which + ": " + run.stdout + run.stderr
+            with np.load(path) as z:
+                got[which] = {k: z[k] for k in z.files}
+    assert sorted(got["plain"]) == sorted(got["bounds"]) and len(got["plain"]) >= 14
+    for k, a in got["plain"].items():
+        assert np.isfinite(a).all(), k
+        assert np.array_equal(a.view(np.uint32), got["bounds"][k].view(np.uint32)), k
